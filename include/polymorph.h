@@ -1,0 +1,187 @@
+/*
+ * polymorph.h -- C ABI of the B200 (sm_100a) Polymorph forward library.
+ *
+ * The library runs the data-parallel hot path of Polymorph (arXiv 2507.14959): the batched
+ * forward pass of a shared ViT/DeiT backbone whose every linear layer computes
+ *
+ *        y = x W + b + sum_{a in S(frame)} s_a (x A_a) B_a            (Sec. 3.1)
+ *
+ * for each frame's own set S of active LoRA adapters (nothing is ever merged into W), followed by
+ * the active adapters' class-subset heads, sigmoid scoring, the per-frame merge of the active
+ * heads (Fig. 5b) and the greedy adapter-set (context) selection of Algorithm 2.
+ *
+ * Conventions
+ *   - Every function returns PM_OK (0) or a negative pm_error; nothing aborts, nothing traps on
+ *     the device.  pm_last_error() gives a text for the last failure on a handle.
+ *   - "host" / "dev" in a comment says where a pointer must live.  All matrices are row-major;
+ *     weights use the paper's row-vector convention W[in, out] (h = x W).
+ *   - Ownership: pm_create / pm_register_adapter / pm_linear_* copy and convert what they are
+ *     given (the caller may free it on return).  Frames, set lists, score and state buffers stay
+ *     caller-owned and must outlive the stream work that uses them.
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and is asynchronous, except where a comment says it synchronises.
+ *   - dtype 0: bf16 storage, fp32 accumulation, tensor-core kernels.  dtype 1: an all-fp32
+ *     debug build of the same path on plain CUDA-core kernels.
+ *   - Device-side waits are bounded; if one expires the kernel records PM_ERR_TIMEOUT in the
+ *     handle's device status word (read it with pm_status) and returns normally.
+ */
+#ifndef POLYMORPH_H_
+#define POLYMORPH_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PM_OK = 0,
+    PM_ERR_ARG = -1,       /* NULL / out-of-range / malformed argument (e.g. non-monotone CSR)  */
+    PM_ERR_STATE = -2,     /* adapter id not registered, cover table not built                  */
+    PM_ERR_CAPACITY = -3,  /* more frames / adapters per frame / rank than the handle was sized  */
+    PM_ERR_CUDA = -4,      /* a CUDA runtime or driver call failed                              */
+    PM_ERR_TIMEOUT = -5,   /* a bounded device-side wait expired                                */
+    PM_ERR_OOM = -6        /* device or host allocation failed                                  */
+} pm_error;
+
+typedef struct pm_handle_s* pm_handle;   /* opaque: owns every device copy of the model   */
+typedef struct pm_linear_s* pm_linear;   /* opaque: one isolated base+multi-LoRA linear   */
+
+/* Model geometry and capacities.  tokens = (img/patch)^2 + 1 (CLS first).  d / heads must be 64. */
+typedef struct {
+    int img, patch, d, layers, heads, mlp, n_classes;
+    float ln_eps;
+    int max_adapters;   /* adapter ids are in [0, max_adapters)                          */
+    int max_rank;       /* largest LoRA rank that will be registered                     */
+    int max_set;        /* largest |S| of a frame                                        */
+    int max_frames;     /* largest batch passed to pm_forward / pm_select                */
+    int dtype;          /* 0 = bf16 tensor-core build, 1 = fp32 debug build              */
+} pm_config;
+
+/* Backbone weights, host fp32.  Per-layer tensors are stacked on a leading [layers] axis. */
+typedef struct {
+    const float *patch_w;   /* [3*patch*patch, d], input order (channel, y, x)  */
+    const float *patch_b;   /* [d]                                               */
+    const float *cls;       /* [d]                                               */
+    const float *pos;       /* [tokens, d]                                       */
+    const float *ln1_g, *ln1_b;     /* [layers, d]                               */
+    const float *qkv_w, *qkv_b;     /* [layers, d, 3d], [layers, 3d]; output columns [3][heads][64] */
+    const float *proj_w, *proj_b;   /* [layers, d, d], [layers, d]               */
+    const float *ln2_g, *ln2_b;     /* [layers, d]                               */
+    const float *fc1_w, *fc1_b;     /* [layers, d, mlp], [layers, mlp]           */
+    const float *fc2_w, *fc2_b;     /* [layers, mlp, d], [layers, d]             */
+    const float *lnf_g, *lnf_b;     /* [d]                                       */
+    const float *head_w, *head_b;   /* base head over all classes: [d, n_classes], [n_classes] */
+} pm_backbone;
+
+/* One LoRA adapter = one context C of the paper (Sec. 3.3): low-rank pairs for the adapted
+ * linears, a head over its class subset, and its per-class accuracies a_{C,l} (Sec. 3.5). */
+typedef struct {
+    int rank;
+    float scale;                 /* alpha / rank (Sec. 4: rank 16, alpha 32 -> 2)                  */
+    const float* const* A;       /* host [layers*4] pointers, index l*4 + {0 qkv,1 proj,2 fc1,3 fc2}: */
+    const float* const* B;       /*   A[in, rank], B[rank, out]; NULL pair = linear not adapted    */
+    int n_cls;
+    const int32_t* class_ids;    /* host [n_cls], distinct, each in [0, n_classes)                 */
+    const float* head_w;         /* host [d, n_cls]                                                */
+    const float* head_b;         /* host [n_cls]                                                   */
+    const float* acc;            /* host [n_cls] accuracies a_{C,l}; NULL = all 1                  */
+} pm_adapter;
+
+/* ---- model lifetime -------------------------------------------------------------------- */
+
+/* Builds the device model from host weights (ViT/DeiT encoder cited in Sec. 1; pre-LN blocks).
+ * Allocates all activation and scratch memory for max_frames.  Synchronises the device. */
+int pm_create(const pm_config* cfg, const pm_backbone* weights, pm_handle* out);
+
+/* Registers (or replaces) adapter `adapter_id` (Sec. 3.1 low-rank pairs, Sec. 4 head).  The
+ * handle's stream work must be idle.  Adapter ids order the tie-breaks of Algorithm 2. */
+int pm_register_adapter(pm_handle h, int adapter_id, const pm_adapter* adapter);
+
+/* Builds the class -> adapter cover tables used by pm_select from the registered adapters and
+ * the accuracy threshold tau of Algorithm 2: for every class its first provider in Algorithm 2's
+ * visiting order (fewest classes first, then lowest id) among adapters with a_{C,l} >= tau, and
+ * the bit mask of all such providers.  Call after the last pm_register_adapter. */
+int pm_set_cover(pm_handle h, float tau);
+
+void pm_destroy(pm_handle h);
+
+/* ---- the hot path ---------------------------------------------------------------------- */
+
+/* Forward pass of n_frames frames (Sec. 3.1, Sec. 3.2, Fig. 5b).
+ *   frames        dev, [n_frames, 3, img, img]; bf16 (dtype 0) or fp32 (dtype 1)
+ *   set_offsets   host or dev int32 [n_frames+1], CSR over frames, set_offsets[0] = 0
+ *   set_ids       host or dev int32 [set_offsets[n_frames]]: adapter ids, distinct per frame (any
+ *                 order; they are applied in ascending id).  Device lists are copied to the host
+ *                 first, which synchronises the stream.
+ *   scores_out    dev fp32 [n_frames, n_classes]: sigmoid scores of the active adapters' heads,
+ *                 scattered to class ids, maximum where several active adapters list a class,
+ *                 0 for classes no active adapter lists
+ *   base_out      dev fp32 [n_frames, n_classes] or NULL: sigmoid scores of the base head
+ * Errors: PM_ERR_ARG (NULL, bad CSR, duplicate id), PM_ERR_STATE (unregistered id),
+ * PM_ERR_CAPACITY (n_frames > max_frames, |S| > max_set).  No kernel is launched on error. */
+int pm_forward(pm_handle h, const void* frames, int n_frames,
+               const int32_t* set_offsets, const int32_t* set_ids,
+               float* scores_out, float* base_out, void* cuda_stream);
+
+/* Algorithm 2 (greedy context detection with conditional context copy) for n_frames streams.
+ *   scores        dev fp32 [n_frames, n_classes]; Y_t = {k : scores[k] > score_thr}
+ *   context_copy  Algorithm 2's flag
+ *   has_prev      0: first frame of every stream (no Y_{t-1}, S_{t-1}: the greedy branch runs);
+ *                 1: prev_labels / prev_offsets / prev_ids hold Y_{t-1} and S_{t-1}
+ *   prev_labels   dev uint32 [n_frames, ceil(n_classes/32)] bit sets; read if has_prev, always
+ *                 overwritten with Y_t; may be NULL only if has_prev == 0 (then nothing is kept)
+ *   prev_offsets, prev_ids   dev int32 CSR of S_{t-1} (ascending ids); read only if has_prev
+ *   next_offsets  dev int32 [n_frames+1]; next_ids dev int32 [ids_capacity]: CSR of S_t,
+ *                 ascending ids.  If the result needs more than ids_capacity entries the lists are
+ *                 truncated and PM_ERR_CAPACITY is recorded in the status word.
+ * Needs pm_set_cover.  prev_* and next_* must not alias. */
+int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, int context_copy,
+              int has_prev, uint32_t* prev_labels,
+              const int32_t* prev_offsets, const int32_t* prev_ids,
+              int32_t* next_offsets, int32_t* next_ids, int ids_capacity, void* cuda_stream);
+
+/* Synchronises the stream and returns the device status word (PM_OK or the first recorded
+ * error), then clears it. */
+int pm_status(pm_handle h, void* cuda_stream);
+
+const char* pm_last_error(pm_handle h);
+
+/* Number of kernels the library has launched on this handle since creation. */
+long long pm_launch_count(pm_handle h);
+
+/* ---- single operators (the same kernels pm_forward uses), for unit tests and sweeps ----- */
+
+/* One base + multi-LoRA linear y = epilogue(x W + b + sum_a s_a (x A_a) B_a)   (Sec. 3.1).
+ *   w host fp32 [k_in, n_out]; bias host fp32 [n_out]
+ *   epilogue 0: none, 1: exact-erf GELU, 2: y += residual
+ * k_in and n_out must be multiples of 64. */
+int pm_linear_create(int k_in, int n_out, const float* w, const float* bias,
+                     int max_adapters, int max_rank, int max_set, int max_frames, int tokens,
+                     int epilogue, int dtype, pm_linear* out);
+/* A host fp32 [k_in, rank], B host fp32 [rank, n_out]. */
+int pm_linear_register(pm_linear lin, int adapter_id, int rank, float scale,
+                       const float* A, const float* B);
+/* x dev [n_frames*tokens, k_in], residual dev [n_frames*tokens, n_out] or NULL (epilogue 2 only),
+ * y dev [n_frames*tokens, n_out]; element type per dtype.  set_offsets / set_ids: host CSR. */
+int pm_linear_forward(pm_linear lin, const void* x, int n_frames,
+                      const int32_t* set_offsets, const int32_t* set_ids,
+                      const void* residual, void* y, void* cuda_stream);
+int pm_linear_status(pm_linear lin, void* cuda_stream);
+const char* pm_linear_last_error(pm_linear lin);
+void pm_linear_destroy(pm_linear lin);
+
+/* Row-wise LayerNorm of x[rows, d] (biased variance, fp32 statistics); gamma/beta dev fp32 [d].
+ * d must be a multiple of 8 and at most 1024. */
+int pm_layernorm(const void* x, const float* gamma, const float* beta, void* y,
+                 int rows, int d, float eps, int dtype, void* cuda_stream);
+
+/* softmax(q k^T / 8) v per (frame, head), head dim 64; qkv dev [n_frames*tokens, 3*heads*64]
+ * with columns ordered [3][heads][64]; out dev [n_frames*tokens, heads*64]. */
+int pm_attention(const void* qkv, void* out, int n_frames, int tokens, int heads, int dtype,
+                 void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POLYMORPH_H_ */

@@ -1,0 +1,780 @@
+// C ABI of the Polymorph library: model upload, adapter arenas, per-batch routing plan
+// (bucketing of frames by adapter set, tile -> LoRA slab lists) and the launch sequences.
+#include <algorithm>
+#include <array>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+
+#include "common.cuh"
+
+int gemm_tile_n(int n_out);   // gemm_tcgen05.cu
+
+namespace {
+
+#define CK(expr)                                                                        \
+    do {                                                                                \
+        cudaError_t _e = (expr);                                                        \
+        if (_e != cudaSuccess) {                                                        \
+            err = std::string(#expr) + ": " + cudaGetErrorString(_e);                   \
+            return _e == cudaErrorMemoryAllocation ? PM_ERR_OOM : PM_ERR_CUDA;          \
+        }                                                                               \
+    } while (0)
+
+template <typename T> T host_cvt(float v);
+template <> float host_cvt<float>(float v) { return v; }
+template <> bf16 host_cvt<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+struct DevBuf {              // owning device allocation
+    void* p = nullptr;
+    size_t bytes = 0;
+    ~DevBuf() { if (p) cudaFree(p); }
+    cudaError_t alloc(size_t n) {
+        if (p) { cudaFree(p); p = nullptr; }
+        bytes = n;
+        if (n == 0) return cudaSuccess;
+        return cudaMalloc(&p, n);
+    }
+    template <typename T> T* as() const { return reinterpret_cast<T*>(p); }
+};
+
+template <typename T>
+cudaError_t upload(DevBuf& buf, const float* host, size_t n) {
+    cudaError_t e = buf.alloc(n * sizeof(T));
+    if (e != cudaSuccess) return e;
+    std::vector<T> tmp(n);
+    for (size_t i = 0; i < n; ++i) tmp[i] = host_cvt<T>(host[i]);
+    return cudaMemcpy(buf.p, tmp.data(), n * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+// [k_in, n_out] row-major -> [n_out, k_in]
+template <typename T>
+cudaError_t upload_transposed(DevBuf& buf, const float* w, int k_in, int n_out) {
+    cudaError_t e = buf.alloc((size_t)k_in * n_out * sizeof(T));
+    if (e != cudaSuccess) return e;
+    std::vector<T> tmp((size_t)k_in * n_out);
+    for (int k = 0; k < k_in; ++k)
+        for (int n = 0; n < n_out; ++n) tmp[(size_t)n * k_in + k] = host_cvt<T>(w[(size_t)k * n_out + n]);
+    return cudaMemcpy(buf.p, tmp.data(), tmp.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+size_t esize(int dtype) { return dtype == 0 ? 2 : 4; }
+
+// One linear with its LoRA arenas.
+struct LinearObj {
+    LinearDev dev;
+    DevBuf wt, bias, at, bt;
+    int slabs_max = 0, max_adapters = 0, dtype = 0;
+
+    int init(int k_in, int n_out, const float* w, const float* b, int max_adapters_, int slabs_max_,
+             int dtype_, std::string& err) {
+        dev.k_in = k_in; dev.n_out = n_out;
+        slabs_max = slabs_max_; max_adapters = max_adapters_; dtype = dtype_;
+        if (dtype == 0) CK(upload_transposed<bf16>(wt, w, k_in, n_out));
+        else CK(upload_transposed<float>(wt, w, k_in, n_out));
+        CK(upload<float>(bias, b, n_out));
+        dev.Wt = wt.p; dev.bias = bias.as<float>();
+        if (max_adapters > 0 && slabs_max > 0) {
+            const size_t RS = (size_t)slabs_max * PM_SLAB;
+            CK(at.alloc((size_t)max_adapters * RS * k_in * esize(dtype)));
+            CK(bt.alloc((size_t)max_adapters * RS * n_out * esize(dtype)));
+            CK(cudaMemset(at.p, 0, at.bytes));
+            CK(cudaMemset(bt.p, 0, bt.bytes));
+            dev.lora.At = at.p; dev.lora.Bt = bt.p;
+        }
+        if (dtype == 0) {
+            const int bn = gemm_tile_n(n_out);
+            bool ok = tm_encode_2d(&dev.tm_w, wt.p, k_in, n_out, (uint64_t)k_in * 2, 64, bn, 128);
+            if (ok && dev.lora.At) {
+                ok = tm_encode_2d(&dev.tm_bt, bt.p, PM_SLAB, (uint64_t)max_adapters * slabs_max * n_out,
+                                  PM_SLAB * 2, PM_SLAB, bn, 32);
+            }
+            if (!ok) { err = "cuTensorMapEncodeTiled failed (static operands)"; return PM_ERR_CUDA; }
+            dev.has_tm = true;
+        }
+        return PM_OK;
+    }
+
+    template <typename T>
+    int set_adapter_t(int a, int rank, const float* A, const float* B, std::string& err) {
+        const int k_in = dev.k_in, n_out = dev.n_out;
+        const size_t RS = (size_t)slabs_max * PM_SLAB;
+        std::vector<T> ha(RS * k_in, host_cvt<T>(0.f)), hb(RS * n_out, host_cvt<T>(0.f));
+        if (A && B) {
+            for (int k = 0; k < k_in; ++k)
+                for (int j = 0; j < rank; ++j) ha[(size_t)j * k_in + k] = host_cvt<T>(A[(size_t)k * rank + j]);
+            for (int j = 0; j < rank; ++j)
+                for (int n = 0; n < n_out; ++n)
+                    hb[((size_t)(j / PM_SLAB) * n_out + n) * PM_SLAB + (j % PM_SLAB)] =
+                        host_cvt<T>(B[(size_t)j * n_out + n]);
+        }
+        CK(cudaMemcpy(at.as<T>() + (size_t)a * RS * k_in, ha.data(), ha.size() * sizeof(T), cudaMemcpyHostToDevice));
+        CK(cudaMemcpy(bt.as<T>() + (size_t)a * RS * n_out, hb.data(), hb.size() * sizeof(T), cudaMemcpyHostToDevice));
+        return PM_OK;
+    }
+    int set_adapter(int a, int rank, const float* A, const float* B, std::string& err) {
+        return dtype == 0 ? set_adapter_t<bf16>(a, rank, A, B, err) : set_adapter_t<float>(a, rank, A, B, err);
+    }
+};
+
+// Per-batch routing: validation, bucketing, tile plan, upload.
+struct Router {
+    int max_frames = 0, max_set = 0, max_adapters = 0, slabs_max = 0, tokens = 0;
+    int slab_cap = 0, max_tiles = 0;
+    DevBuf blob;
+    void* stage = nullptr;          // pinned host copy of the blob
+    size_t blob_bytes = 0;
+    size_t off_perm = 0, off_soff = 0, off_sids = 0, off_tn = 0, off_ts = 0, off_tsc = 0, off_tm = 0;
+    cudaEvent_t uploaded = nullptr;
+    bool upload_pending = false;
+    RouteDev dev;
+    std::vector<int32_t> last_off, last_ids;
+    int last_frames = -1;
+    bool last_sorted = false;
+    std::vector<int> perm_host;
+
+    ~Router() {
+        if (stage) cudaFreeHost(stage);
+        if (uploaded) cudaEventDestroy(uploaded);
+    }
+
+    int init(int max_frames_, int max_set_, int max_adapters_, int slabs_max_, int tokens_, std::string& err) {
+        max_frames = max_frames_; max_set = max_set_; max_adapters = max_adapters_;
+        slabs_max = slabs_max_; tokens = tokens_;
+        const int frames_per_tile = (PM_TILE_M - 1) / tokens + 2;
+        slab_cap = std::min(frames_per_tile * max_set, max_adapters) * slabs_max;
+        max_tiles = (int)(((size_t)max_frames * tokens + PM_TILE_M - 1) / PM_TILE_M);
+        auto take = [&](size_t& off, size_t bytes) { off = blob_bytes; blob_bytes += (bytes + 255) & ~(size_t)255; };
+        take(off_perm, sizeof(int) * max_frames);
+        take(off_soff, sizeof(int) * (max_frames + 1));
+        take(off_sids, sizeof(int) * std::max(1, max_frames * max_set));
+        take(off_tn, sizeof(int) * max_tiles);
+        take(off_ts, sizeof(int) * std::max(1, max_tiles * slab_cap));
+        take(off_tsc, sizeof(float) * std::max(1, max_tiles * slab_cap));
+        take(off_tm, sizeof(uint32_t) * 4 * std::max(1, max_tiles * slab_cap));
+        CK(blob.alloc(blob_bytes));
+        CK(cudaMemset(blob.p, 0, blob_bytes));
+        CK(cudaMallocHost(&stage, blob_bytes));
+        memset(stage, 0, blob_bytes);
+        CK(cudaEventCreateWithFlags(&uploaded, cudaEventDisableTiming));
+        uint8_t* b = blob.as<uint8_t>();
+        dev.perm = (int*)(b + off_perm); dev.slot_off = (int*)(b + off_soff); dev.slot_ids = (int*)(b + off_sids);
+        dev.tile_nslabs = (int*)(b + off_tn); dev.tile_slab = (int*)(b + off_ts);
+        dev.tile_scale = (float*)(b + off_tsc); dev.tile_mask = (uint32_t*)(b + off_tm);
+        dev.tokens = tokens; dev.slab_cap = slab_cap;
+        return PM_OK;
+    }
+
+    // offsets/ids: host CSR.  ranks[a] == 0 means "not registered".
+    int build(int n_frames, const int32_t* offsets, const int32_t* ids, const std::vector<int>& ranks,
+              const std::vector<float>& scales, bool sort_frames, cudaStream_t st, std::string& err) {
+        if (n_frames < 0 || (n_frames > 0 && (!offsets))) { err = "bad frame count or NULL set_offsets"; return PM_ERR_ARG; }
+        if (n_frames > max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
+        if (n_frames > 0 && offsets[0] != 0) { err = "set_offsets[0] must be 0"; return PM_ERR_ARG; }
+        for (int f = 0; f < n_frames; ++f) {
+            if (offsets[f + 1] < offsets[f]) { err = "set_offsets not monotone"; return PM_ERR_ARG; }
+            if (offsets[f + 1] - offsets[f] > max_set) { err = "a frame has more adapters than max_set"; return PM_ERR_CAPACITY; }
+        }
+        const int nnz = n_frames > 0 ? offsets[n_frames] : 0;
+        if (nnz > 0 && !ids) { err = "NULL set_ids"; return PM_ERR_ARG; }
+        // unchanged sets (the common case: temporal continuity) reuse the uploaded plan
+        if (n_frames == last_frames && sort_frames == last_sorted && (int)last_ids.size() == nnz &&
+            std::equal(offsets, offsets + n_frames + 1, last_off.begin()) &&
+            std::equal(ids, ids + nnz, last_ids.begin()))
+            return PM_OK;
+        std::vector<std::vector<int>> sets(n_frames);
+        int widest = 0;
+        for (int f = 0; f < n_frames; ++f) {
+            sets[f].assign(ids + offsets[f], ids + offsets[f + 1]);
+            std::sort(sets[f].begin(), sets[f].end());
+            for (size_t i = 0; i < sets[f].size(); ++i) {
+                const int a = sets[f][i];
+                if (a < 0 || a >= max_adapters) { err = "adapter id out of range"; return PM_ERR_ARG; }
+                if (i > 0 && sets[f][i - 1] == a) { err = "duplicate adapter id in a frame's set"; return PM_ERR_ARG; }
+                if (ranks[a] == 0) { err = "adapter id not registered"; return PM_ERR_STATE; }
+            }
+            widest = std::max(widest, (int)sets[f].size());
+        }
+        perm_host.resize(n_frames);
+        for (int f = 0; f < n_frames; ++f) perm_host[f] = f;
+        if (sort_frames)
+            std::stable_sort(perm_host.begin(), perm_host.end(),
+                             [&](int a, int b) { return sets[a] < sets[b]; });
+        if (upload_pending) { CK(cudaEventSynchronize(uploaded)); upload_pending = false; }
+        uint8_t* s = (uint8_t*)stage;
+        int* h_perm = (int*)(s + off_perm); int* h_soff = (int*)(s + off_soff); int* h_sids = (int*)(s + off_sids);
+        int* h_tn = (int*)(s + off_tn); int* h_ts = (int*)(s + off_ts);
+        float* h_tsc = (float*)(s + off_tsc); uint32_t* h_tm = (uint32_t*)(s + off_tm);
+        h_soff[0] = 0;
+        for (int i = 0; i < n_frames; ++i) {
+            const std::vector<int>& st_ = sets[perm_host[i]];
+            h_perm[i] = perm_host[i];
+            std::copy(st_.begin(), st_.end(), h_sids + h_soff[i]);
+            h_soff[i + 1] = h_soff[i] + (int)st_.size();
+        }
+        const long long rows = (long long)n_frames * tokens;
+        const int n_tiles = (int)((rows + PM_TILE_M - 1) / PM_TILE_M);
+        for (int t = 0; t < n_tiles; ++t) {
+            const long long r0 = (long long)t * PM_TILE_M, r1 = std::min(rows, r0 + PM_TILE_M);
+            std::map<int, std::array<uint32_t, 4>> slabs;      // arena slab -> row mask, ascending
+            for (int slot = (int)(r0 / tokens); slot <= (int)((r1 - 1) / tokens); ++slot) {
+                const long long a0 = std::max(r0, (long long)slot * tokens);
+                const long long a1 = std::min(r1, (long long)(slot + 1) * tokens);
+                for (int a : sets[perm_host[slot]]) {
+                    const int ns = (ranks[a] + PM_SLAB - 1) / PM_SLAB;
+                    for (int j = 0; j < ns; ++j) {
+                        auto& m = slabs[a * slabs_max + j];
+                        for (long long r = a0; r < a1; ++r) m[(r - r0) >> 5] |= 1u << ((r - r0) & 31);
+                    }
+                }
+            }
+            if ((int)slabs.size() > slab_cap) { err = "tile needs more LoRA slabs than the plan capacity"; return PM_ERR_CAPACITY; }
+            h_tn[t] = (int)slabs.size();
+            int i = 0;
+            for (auto& kv : slabs) {
+                const size_t at = (size_t)t * slab_cap + i++;
+                h_ts[at] = kv.first;
+                h_tsc[at] = scales[kv.first / slabs_max];
+                for (int q = 0; q < 4; ++q) h_tm[at * 4 + q] = kv.second[q];
+            }
+        }
+        CK(cudaMemcpyAsync(blob.p, stage, blob_bytes, cudaMemcpyHostToDevice, st));
+        CK(cudaEventRecord(uploaded, st));
+        upload_pending = true;
+        dev.n_frames = n_frames; dev.n_tiles = n_tiles; dev.max_set = widest;
+        last_off.assign(offsets, offsets + n_frames + 1);
+        last_ids.assign(ids, ids + nnz);
+        last_frames = n_frames; last_sorted = sort_frames;
+        return PM_OK;
+    }
+    void invalidate() { last_frames = -1; }
+};
+
+// Copies a CSR that may live on the device to the host (synchronising the stream if it does).
+int fetch_csr(const int32_t* offsets, const int32_t* ids, int n_frames, cudaStream_t st,
+              std::vector<int32_t>& hoff, std::vector<int32_t>& hids, const int32_t** o, const int32_t** i,
+              std::string& err) {
+    *o = offsets; *i = ids;
+    if (!offsets || n_frames <= 0) return PM_OK;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, offsets) != cudaSuccess) { cudaGetLastError(); return PM_OK; }
+    if (at.type != cudaMemoryTypeDevice) return PM_OK;
+    hoff.resize(n_frames + 1);
+    CK(cudaMemcpyAsync(hoff.data(), offsets, sizeof(int32_t) * (n_frames + 1), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    const int nnz = hoff[n_frames];
+    if (nnz < 0) { err = "negative set_offsets"; return PM_ERR_ARG; }
+    hids.resize(std::max(nnz, 1));
+    if (nnz > 0) {
+        if (!ids) { err = "NULL set_ids"; return PM_ERR_ARG; }
+        CK(cudaMemcpyAsync(hids.data(), ids, sizeof(int32_t) * nnz, cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+    }
+    *o = hoff.data(); *i = hids.data();
+    return PM_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// handles
+// ---------------------------------------------------------------------------------------
+struct pm_linear_s {
+    int k_in = 0, n_out = 0, max_adapters = 0, max_rank = 0, slabs_max = 0, max_set = 0, max_frames = 0;
+    int tokens = 0, epilogue = 0, dtype = 0, n_sms = 148;
+    LinearObj lin;
+    Router router;
+    std::vector<int> ranks;
+    std::vector<float> scales;
+    DevBuf scale_dev, rank_dev, t32, tbuf, status;
+    AdapterMeta meta;
+    CUtensorMap tm_t;
+    long long launches = 0;
+    std::string err;
+};
+
+struct pm_handle_s {
+    pm_config cfg;
+    int tokens = 0, g2 = 0, patch_dim = 0, slabs_max = 0, n_sms = 148;
+    LinearObj patch;                         // no LoRA
+    std::vector<LinearObj> lin;              // [layers*4]
+    DevBuf cls, pos, ln1_g, ln1_b, ln2_g, ln2_b, lnf_g, lnf_b, head_wt, head_b;
+    // activations
+    DevBuf X, U, QKV, ATT, H, PATCH, Z, t32, tbuf, status;
+    CUtensorMap tm_patch, tm_u, tm_att, tm_h, tm_t;
+    int tm_rows = -1;
+    Router router;
+    // adapters
+    std::vector<int> ranks;
+    std::vector<float> scales;
+    std::vector<std::vector<int32_t>> cls_ids;
+    std::vector<std::vector<float>> head_w, head_b_host, acc;
+    DevBuf scale_dev, rank_dev, hcat, hbias, hcls, hoff;
+    AdapterMeta meta;
+    bool heads_dirty = true;
+    // cover tables
+    DevBuf first, provider, mask_scratch;
+    bool cover_ready = false;
+    long long launches = 0;
+    std::string err;
+};
+
+namespace {
+
+int slabs_for(int max_rank) { return (max_rank + PM_SLAB - 1) / PM_SLAB; }
+
+int sync_meta(DevBuf& scale_dev, DevBuf& rank_dev, const std::vector<float>& scales,
+              const std::vector<int>& ranks, std::string& err) {
+    CK(cudaMemcpy(scale_dev.p, scales.data(), scales.size() * sizeof(float), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(rank_dev.p, ranks.data(), ranks.size() * sizeof(int), cudaMemcpyHostToDevice));
+    return PM_OK;
+}
+
+template <typename T>
+int rebuild_heads(pm_handle_s* h) {
+    std::string& err = h->err;
+    const int d = h->cfg.d, na = h->cfg.max_adapters;
+    std::vector<int> hoff(na + 1, 0);
+    for (int a = 0; a < na; ++a) hoff[a + 1] = hoff[a] + (h->ranks[a] ? (int)h->cls_ids[a].size() : 0);
+    const int total = hoff[na];
+    std::vector<T> hc((size_t)std::max(total, 1) * d);
+    std::vector<float> hb(std::max(total, 1));
+    std::vector<int> hk(std::max(total, 1));
+    for (int a = 0; a < na; ++a) {
+        if (!h->ranks[a]) continue;
+        const int n = (int)h->cls_ids[a].size();
+        for (int j = 0; j < n; ++j) {
+            const int r = hoff[a] + j;
+            for (int c = 0; c < d; ++c) hc[(size_t)r * d + c] = host_cvt<T>(h->head_w[a][(size_t)c * n + j]);
+            hb[r] = h->head_b_host[a][j];
+            hk[r] = h->cls_ids[a][j];
+        }
+    }
+    CK(h->hcat.alloc(hc.size() * sizeof(T)));
+    CK(h->hbias.alloc(hb.size() * sizeof(float)));
+    CK(h->hcls.alloc(hk.size() * sizeof(int)));
+    CK(h->hoff.alloc(hoff.size() * sizeof(int)));
+    CK(cudaMemcpy(h->hcat.p, hc.data(), hc.size() * sizeof(T), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(h->hbias.p, hb.data(), hb.size() * sizeof(float), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(h->hcls.p, hk.data(), hk.size() * sizeof(int), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(h->hoff.p, hoff.data(), hoff.size() * sizeof(int), cudaMemcpyHostToDevice));
+    h->heads_dirty = false;
+    return PM_OK;
+}
+
+int encode_activation_maps(pm_handle_s* h, int rows) {
+    if (h->tm_rows == rows) return PM_OK;
+    const int d = h->cfg.d;
+    const int prow = rows / h->tokens * h->g2;
+    bool ok = tm_encode_2d(&h->tm_patch, h->PATCH.p, h->patch_dim, prow, (uint64_t)h->patch_dim * 2, 64, PM_TILE_M, 128)
+           && tm_encode_2d(&h->tm_u, h->U.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
+           && tm_encode_2d(&h->tm_att, h->ATT.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
+           && tm_encode_2d(&h->tm_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 64, PM_TILE_M, 128);
+    if (!ok) { h->err = "cuTensorMapEncodeTiled failed (activations)"; return PM_ERR_CUDA; }
+    h->tm_rows = rows;
+    return PM_OK;
+}
+
+template <typename T>
+int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_out, float* base_out,
+              cudaStream_t st) {
+    std::string& err = h->err;
+    const pm_config& c = h->cfg;
+    const int T_ = h->tokens, d = c.d, rows = n_frames * T_;
+    Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>();
+    const RouteDev& R = h->router.dev;
+    constexpr bool TC = sizeof(T) == 2;
+    if (TC) { int rc = encode_activation_maps(h, rows); if (rc) return rc; }
+    PatchEpi pe; pe.g2 = h->g2; pe.tokens = T_; pe.pos = h->pos.as<float>();
+    PatchEpi none;
+    T* X = h->X.as<T>(); T* U = h->U.as<T>(); T* QKV = h->QKV.as<T>(); T* ATT = h->ATT.as<T>();
+    T* Hb = h->H.as<T>(); T* P = h->PATCH.as<T>();
+
+    auto linear = [&](LinearObj& lo, const T* x, const CUtensorMap* tmx, int nrows, int tokens_pf, bool lora,
+                      int epi, const T* residual, const PatchEpi& pep, T* y) -> cudaError_t {
+        if constexpr (TC) {
+            const bool use_lora = lora && R.max_set > 0;
+            if (use_lora) {
+                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>());
+                if (e != cudaSuccess) return e;
+            }
+            return launch_lora_gemm(L, lo.dev, use_lora ? &R : nullptr, *tmx, &h->tm_t, nrows, epi,
+                                    (const bf16*)residual, pep, (bf16*)y, h->n_sms);
+        } else {
+            return launch_naive_linear<T>(L, lo.dev, R, h->meta, h->slabs_max, x, nrows, tokens_pf,
+                                          lora ? h->t32.as<float>() : nullptr, epi, residual, pep, y);
+        }
+    };
+
+    CK(launch_im2col<T>(L, (const T*)frames, R.perm, P, n_frames, c.img, c.patch));
+    CK(linear(h->patch, P, &h->tm_patch, n_frames * h->g2, h->g2, false, EPI_PATCH, nullptr, pe, X));
+    CK(launch_cls_rows<T>(L, h->cls.as<float>(), h->pos.as<float>(), X, n_frames, T_, d));
+    for (int l = 0; l < c.layers; ++l) {
+        CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
+        CK(linear(h->lin[l * 4 + 0], U, &h->tm_u, rows, T_, true, EPI_NONE, nullptr, none, QKV));
+        if constexpr (TC) CK(launch_attention_mma(L, (const bf16*)QKV, (bf16*)ATT, n_frames, T_, c.heads));
+        else CK(launch_attention_simple<T>(L, QKV, ATT, n_frames, T_, c.heads));
+        CK(linear(h->lin[l * 4 + 1], ATT, &h->tm_att, rows, T_, true, EPI_RESIDUAL, X, none, X));
+        CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
+        CK(linear(h->lin[l * 4 + 2], U, &h->tm_u, rows, T_, true, EPI_GELU, nullptr, none, Hb));
+        CK(linear(h->lin[l * 4 + 3], Hb, &h->tm_h, rows, T_, true, EPI_RESIDUAL, X, none, X));
+    }
+    CK(launch_heads<T>(L, X, n_frames, T_, d, c.ln_eps, h->lnf_g.as<float>(), h->lnf_b.as<float>(),
+                       h->Z.as<float>(), h->head_wt.as<T>(), h->head_b.as<float>(), c.n_classes,
+                       h->hcat.as<T>(), h->hbias.as<float>(), h->hcls.as<int>(), h->hoff.as<int>(), R,
+                       scores_out, base_out));
+    return PM_OK;
+}
+
+template <typename T>
+int create_t(pm_handle_s* h, const pm_backbone* w) {
+    std::string& err = h->err;
+    const pm_config& c = h->cfg;
+    const int d = c.d, L = c.layers, m = c.mlp, K = c.n_classes, T_ = h->tokens;
+    int rc = h->patch.init(h->patch_dim, d, w->patch_w, w->patch_b, 0, 0, c.dtype, err);
+    if (rc) return rc;
+    h->lin.resize((size_t)L * 4);
+    for (int l = 0; l < L; ++l) {
+        const float* ws[4] = {w->qkv_w + (size_t)l * d * 3 * d, w->proj_w + (size_t)l * d * d,
+                              w->fc1_w + (size_t)l * d * m, w->fc2_w + (size_t)l * m * d};
+        const float* bs[4] = {w->qkv_b + (size_t)l * 3 * d, w->proj_b + (size_t)l * d,
+                              w->fc1_b + (size_t)l * m, w->fc2_b + (size_t)l * d};
+        const int kin[4] = {d, d, d, m}, nout[4] = {3 * d, d, m, d};
+        for (int p = 0; p < 4; ++p) {
+            rc = h->lin[l * 4 + p].init(kin[p], nout[p], ws[p], bs[p], c.max_adapters, h->slabs_max, c.dtype, err);
+            if (rc) return rc;
+        }
+    }
+    CK(upload<float>(h->cls, w->cls, d));
+    CK(upload<float>(h->pos, w->pos, (size_t)T_ * d));
+    CK(upload<float>(h->ln1_g, w->ln1_g, (size_t)L * d)); CK(upload<float>(h->ln1_b, w->ln1_b, (size_t)L * d));
+    CK(upload<float>(h->ln2_g, w->ln2_g, (size_t)L * d)); CK(upload<float>(h->ln2_b, w->ln2_b, (size_t)L * d));
+    CK(upload<float>(h->lnf_g, w->lnf_g, d)); CK(upload<float>(h->lnf_b, w->lnf_b, d));
+    CK(upload_transposed<T>(h->head_wt, w->head_w, d, K));
+    CK(upload<float>(h->head_b, w->head_b, K));
+    const size_t rows = (size_t)c.max_frames * T_;
+    const size_t rows_pad = (rows + PM_TILE_M - 1) / PM_TILE_M * PM_TILE_M;
+    CK(h->X.alloc(rows_pad * d * sizeof(T))); CK(h->U.alloc(rows_pad * d * sizeof(T)));
+    CK(h->QKV.alloc(rows_pad * 3 * d * sizeof(T))); CK(h->ATT.alloc(rows_pad * d * sizeof(T)));
+    CK(h->H.alloc(rows_pad * m * sizeof(T)));
+    CK(h->PATCH.alloc(rows_pad * h->patch_dim * sizeof(T)));
+    CK(h->Z.alloc((size_t)c.max_frames * d * sizeof(float)));
+    CK(cudaMemset(h->X.p, 0, h->X.bytes)); CK(cudaMemset(h->U.p, 0, h->U.bytes));
+    CK(cudaMemset(h->QKV.p, 0, h->QKV.bytes)); CK(cudaMemset(h->ATT.p, 0, h->ATT.bytes));
+    CK(cudaMemset(h->H.p, 0, h->H.bytes)); CK(cudaMemset(h->PATCH.p, 0, h->PATCH.bytes));
+    rc = h->router.init(c.max_frames, c.max_set, c.max_adapters, h->slabs_max, T_, err);
+    if (rc) return rc;
+    if (c.dtype == 0) {
+        const size_t tb = (size_t)h->router.max_tiles * std::max(1, h->router.slab_cap) * PM_TILE_M * PM_SLAB;
+        CK(h->tbuf.alloc(tb * sizeof(bf16)));
+        CK(cudaMemset(h->tbuf.p, 0, h->tbuf.bytes));
+        if (!tm_encode_2d(&h->tm_t, h->tbuf.p, PM_SLAB, tb / PM_SLAB, PM_SLAB * 2, PM_SLAB, PM_TILE_M, 32)) {
+            err = "cuTensorMapEncodeTiled failed (slab buffer)"; return PM_ERR_CUDA;
+        }
+    } else {
+        CK(h->t32.alloc(rows * std::max(1, c.max_set) * h->slabs_max * PM_SLAB * sizeof(float)));
+    }
+    return PM_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// exported functions
+// ---------------------------------------------------------------------------------------
+extern "C" {
+
+int pm_create(const pm_config* cfg, const pm_backbone* w, pm_handle* out) {
+    if (!cfg || !w || !out) return PM_ERR_ARG;
+    *out = nullptr;
+    const pm_config& c = *cfg;
+    if (c.patch != 16 || c.img <= 0 || c.img % c.patch || c.d <= 0 || c.d % 64 || c.heads <= 0 ||
+        c.d != c.heads * 64 || c.mlp <= 0 || c.mlp % 64 || c.layers <= 0 || c.n_classes <= 0 ||
+        c.d > 1024 || c.max_adapters < 0 || c.max_adapters > 256 || c.max_rank < 0 || c.max_set < 0 ||
+        c.max_frames <= 0 || (c.dtype != 0 && c.dtype != 1))
+        return PM_ERR_ARG;
+    const float* const* fields = reinterpret_cast<const float* const*>(w);
+    for (size_t i = 0; i < sizeof(pm_backbone) / sizeof(const float*); ++i)
+        if (!fields[i]) return PM_ERR_ARG;
+    pm_handle_s* h = new (std::nothrow) pm_handle_s();
+    if (!h) return PM_ERR_OOM;
+    h->cfg = c;
+    const int g = c.img / c.patch;
+    h->g2 = g * g; h->tokens = g * g + 1; h->patch_dim = 3 * c.patch * c.patch;
+    h->slabs_max = slabs_for(c.max_rank);
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        delete h; return PM_ERR_CUDA;
+    }
+    h->ranks.assign(std::max(1, c.max_adapters), 0);
+    h->scales.assign(std::max(1, c.max_adapters), 0.f);
+    h->cls_ids.resize(c.max_adapters); h->head_w.resize(c.max_adapters);
+    h->head_b_host.resize(c.max_adapters); h->acc.resize(c.max_adapters);
+    int rc = c.dtype == 0 ? create_t<bf16>(h, w) : create_t<float>(h, w);
+    std::string& err = h->err;
+    auto fail = [&](int code) { fprintf(stderr, "pm_create: %s\n", h->err.c_str()); delete h; return code; };
+    if (rc) return fail(rc);
+    if (h->scale_dev.alloc(h->scales.size() * sizeof(float)) != cudaSuccess ||
+        h->rank_dev.alloc(h->ranks.size() * sizeof(int)) != cudaSuccess ||
+        h->status.alloc(sizeof(int)) != cudaSuccess ||
+        cudaMemset(h->status.p, 0, sizeof(int)) != cudaSuccess) { err = "allocation failed"; return fail(PM_ERR_OOM); }
+    rc = sync_meta(h->scale_dev, h->rank_dev, h->scales, h->ranks, err);
+    if (rc) return fail(rc);
+    h->meta.scale = h->scale_dev.as<float>(); h->meta.rank = h->rank_dev.as<int>();
+    if (cudaDeviceSynchronize() != cudaSuccess) { err = "device synchronize failed"; return fail(PM_ERR_CUDA); }
+    *out = h;
+    return PM_OK;
+}
+
+int pm_register_adapter(pm_handle h, int id, const pm_adapter* a) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    const pm_config& c = h->cfg;
+    if (!a || id < 0 || id >= c.max_adapters) { err = "adapter id out of range"; return PM_ERR_ARG; }
+    if (a->rank <= 0 || a->rank > c.max_rank) { err = "adapter rank exceeds max_rank"; return PM_ERR_CAPACITY; }
+    if (!a->A || !a->B || a->n_cls < 0 || (a->n_cls > 0 && (!a->class_ids || !a->head_w || !a->head_b))) {
+        err = "NULL adapter field"; return PM_ERR_ARG;
+    }
+    std::vector<char> seen(c.n_classes, 0);
+    for (int j = 0; j < a->n_cls; ++j) {
+        const int k = a->class_ids[j];
+        if (k < 0 || k >= c.n_classes || seen[k]) { err = "class ids must be distinct and in range"; return PM_ERR_ARG; }
+        seen[k] = 1;
+    }
+    for (int i = 0; i < c.layers * 4; ++i)
+        if ((a->A[i] == nullptr) != (a->B[i] == nullptr)) { err = "A and B must both be given or both NULL"; return PM_ERR_ARG; }
+    for (int i = 0; i < c.layers * 4; ++i) {
+        int rc = h->lin[i].set_adapter(id, a->rank, a->A[i], a->B[i], err);
+        if (rc) return rc;
+    }
+    h->ranks[id] = a->rank; h->scales[id] = a->scale;
+    h->cls_ids[id].assign(a->class_ids, a->class_ids + a->n_cls);
+    h->head_w[id].assign(a->head_w, a->head_w + (size_t)c.d * a->n_cls);
+    h->head_b_host[id].assign(a->head_b, a->head_b + a->n_cls);
+    if (a->acc) h->acc[id].assign(a->acc, a->acc + a->n_cls);
+    else h->acc[id].assign(a->n_cls, 1.f);
+    h->heads_dirty = true; h->cover_ready = false;
+    h->router.invalidate();
+    return sync_meta(h->scale_dev, h->rank_dev, h->scales, h->ranks, err);
+}
+
+int pm_set_cover(pm_handle h, float tau) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    const int K = h->cfg.n_classes, na = h->cfg.max_adapters;
+    const int AW = std::max(1, (na + 63) / 64);
+    // Algorithm 2 visits contexts by increasing size |C| (all listed classes), ties by id
+    std::vector<int> order;
+    for (int a = 0; a < na; ++a) if (h->ranks[a]) order.push_back(a);
+    std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
+        return h->cls_ids[x].size() < h->cls_ids[y].size();
+    });
+    std::vector<int> first(K, -1);
+    std::vector<uint64_t> prov((size_t)K * AW, 0);
+    for (int a : order)
+        for (size_t j = 0; j < h->cls_ids[a].size(); ++j) {
+            if (!(h->acc[a][j] >= tau)) continue;
+            const int k = h->cls_ids[a][j];
+            if (first[k] < 0) first[k] = a;
+            prov[(size_t)k * AW + (a >> 6)] |= 1ull << (a & 63);
+        }
+    CK(h->first.alloc(first.size() * sizeof(int)));
+    CK(h->provider.alloc(prov.size() * sizeof(uint64_t)));
+    CK(h->mask_scratch.alloc((size_t)h->cfg.max_frames * AW * sizeof(uint64_t)));
+    CK(cudaMemcpy(h->first.p, first.data(), first.size() * sizeof(int), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(h->provider.p, prov.data(), prov.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
+    h->cover_ready = true;
+    return PM_OK;
+}
+
+void pm_destroy(pm_handle h) {
+    if (!h) return;
+    cudaDeviceSynchronize();
+    delete h;
+}
+
+int pm_forward(pm_handle h, const void* frames, int n_frames, const int32_t* set_offsets,
+               const int32_t* set_ids, float* scores_out, float* base_out, void* cuda_stream) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (n_frames < 0 || (n_frames > 0 && (!frames || !set_offsets || !scores_out))) { err = "NULL argument"; return PM_ERR_ARG; }
+    if (n_frames == 0) return PM_OK;
+    if (n_frames > h->cfg.max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
+    std::vector<int32_t> hoff, hids;
+    const int32_t *o, *i;
+    int rc = fetch_csr(set_offsets, set_ids, n_frames, st, hoff, hids, &o, &i, err);
+    if (rc) return rc;
+    rc = h->router.build(n_frames, o, i, h->ranks, h->scales, true, st, err);
+    if (rc) return rc;
+    if (h->heads_dirty) {
+        rc = h->cfg.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
+        if (rc) return rc;
+    }
+    return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, scores_out, base_out, st)
+                             : forward_t<float>(h, frames, n_frames, scores_out, base_out, st);
+}
+
+int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, int context_copy,
+              int has_prev, uint32_t* prev_labels, const int32_t* prev_offsets, const int32_t* prev_ids,
+              int32_t* next_offsets, int32_t* next_ids, int ids_capacity, void* cuda_stream) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    if (!h->cover_ready) { err = "pm_set_cover has not been called since the last registration"; return PM_ERR_STATE; }
+    if (n_frames < 0 || !scores || !next_offsets || (!next_ids && ids_capacity > 0) || ids_capacity < 0) { err = "NULL argument"; return PM_ERR_ARG; }
+    if (has_prev && (!prev_labels || !prev_offsets || !prev_ids)) { err = "has_prev needs prev_labels, prev_offsets and prev_ids"; return PM_ERR_ARG; }
+    if (n_frames > h->cfg.max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
+    Launch L; L.st = (cudaStream_t)cuda_stream; L.launches = &h->launches; L.status = h->status.as<int>();
+    CK(launch_select(L, scores, n_frames, h->cfg.n_classes, h->cfg.max_adapters, score_thr, context_copy,
+                     has_prev, prev_labels, prev_offsets, prev_ids, h->first.as<int>(),
+                     h->provider.as<uint64_t>(), h->mask_scratch.as<uint64_t>(), next_offsets, next_ids,
+                     ids_capacity));
+    return PM_OK;
+}
+
+static int read_status(DevBuf& status, cudaStream_t st, std::string& err) {
+    int v = 0;
+    CK(cudaStreamSynchronize(st));
+    CK(cudaMemcpy(&v, status.p, sizeof(int), cudaMemcpyDeviceToHost));
+    if (v != 0) {
+        CK(cudaMemset(status.p, 0, sizeof(int)));
+        err = v == PM_ERR_TIMEOUT ? "a bounded device-side wait expired" : "device status word set";
+    }
+    return v;
+}
+
+int pm_status(pm_handle h, void* cuda_stream) {
+    if (!h) return PM_ERR_ARG;
+    return read_status(h->status, (cudaStream_t)cuda_stream, h->err);
+}
+
+const char* pm_last_error(pm_handle h) { return h ? h->err.c_str() : "NULL handle"; }
+long long pm_launch_count(pm_handle h) { return h ? h->launches : 0; }
+
+// ---- single operators -------------------------------------------------------------------
+int pm_linear_create(int k_in, int n_out, const float* w, const float* bias, int max_adapters,
+                     int max_rank, int max_set, int max_frames, int tokens, int epilogue, int dtype,
+                     pm_linear* out) {
+    if (!out) return PM_ERR_ARG;
+    *out = nullptr;
+    if (!w || !bias || k_in <= 0 || n_out <= 0 || k_in % 64 || n_out % 64 || max_adapters < 0 ||
+        max_adapters > 256 || max_rank < 0 || max_set < 0 || max_frames <= 0 || tokens <= 0 ||
+        epilogue < 0 || epilogue > 2 || (dtype != 0 && dtype != 1))
+        return PM_ERR_ARG;
+    pm_linear_s* l = new (std::nothrow) pm_linear_s();
+    if (!l) return PM_ERR_OOM;
+    std::string& err = l->err;
+    l->k_in = k_in; l->n_out = n_out; l->max_adapters = max_adapters; l->max_rank = max_rank;
+    l->slabs_max = slabs_for(max_rank); l->max_set = max_set; l->max_frames = max_frames;
+    l->tokens = tokens; l->epilogue = epilogue; l->dtype = dtype;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&l->n_sms, cudaDevAttrMultiProcessorCount, dev);
+    auto fail = [&](int code) { fprintf(stderr, "pm_linear_create: %s\n", l->err.c_str()); delete l; return code; };
+    int rc = l->lin.init(k_in, n_out, w, bias, max_adapters, l->slabs_max, dtype, err);
+    if (rc) return fail(rc);
+    rc = l->router.init(max_frames, max_set, std::max(1, max_adapters), l->slabs_max, tokens, err);
+    if (rc) return fail(rc);
+    l->ranks.assign(std::max(1, max_adapters), 0);
+    l->scales.assign(std::max(1, max_adapters), 0.f);
+    const size_t rows = (size_t)max_frames * tokens;
+    cudaError_t e = l->scale_dev.alloc(l->scales.size() * sizeof(float));
+    if (e == cudaSuccess) e = l->rank_dev.alloc(l->ranks.size() * sizeof(int));
+    if (e == cudaSuccess) e = l->status.alloc(sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(l->status.p, 0, sizeof(int));
+    if (e == cudaSuccess && dtype == 1)
+        e = l->t32.alloc(rows * std::max(1, max_set) * std::max(1, l->slabs_max) * PM_SLAB * sizeof(float));
+    size_t tb = 0;
+    if (e == cudaSuccess && dtype == 0) {
+        tb = (size_t)l->router.max_tiles * std::max(1, l->router.slab_cap) * PM_TILE_M * PM_SLAB;
+        e = l->tbuf.alloc(tb * sizeof(bf16));
+        if (e == cudaSuccess) e = cudaMemset(l->tbuf.p, 0, l->tbuf.bytes);
+    }
+    if (e != cudaSuccess) { err = cudaGetErrorString(e); return fail(e == cudaErrorMemoryAllocation ? PM_ERR_OOM : PM_ERR_CUDA); }
+    if (dtype == 0 && !tm_encode_2d(&l->tm_t, l->tbuf.p, PM_SLAB, tb / PM_SLAB, PM_SLAB * 2, PM_SLAB, PM_TILE_M, 32)) {
+        err = "cuTensorMapEncodeTiled failed (slab buffer)"; return fail(PM_ERR_CUDA);
+    }
+    rc = sync_meta(l->scale_dev, l->rank_dev, l->scales, l->ranks, err);
+    if (rc) return fail(rc);
+    l->meta.scale = l->scale_dev.as<float>(); l->meta.rank = l->rank_dev.as<int>();
+    if (cudaDeviceSynchronize() != cudaSuccess) { err = "device synchronize failed"; return fail(PM_ERR_CUDA); }
+    *out = l;
+    return PM_OK;
+}
+
+int pm_linear_register(pm_linear l, int id, int rank, float scale, const float* A, const float* B) {
+    if (!l) return PM_ERR_ARG;
+    std::string& err = l->err;
+    if (id < 0 || id >= l->max_adapters || !A || !B) { err = "bad adapter id or NULL matrices"; return PM_ERR_ARG; }
+    if (rank <= 0 || rank > l->max_rank) { err = "adapter rank exceeds max_rank"; return PM_ERR_CAPACITY; }
+    int rc = l->lin.set_adapter(id, rank, A, B, err);
+    if (rc) return rc;
+    l->ranks[id] = rank; l->scales[id] = scale;
+    l->router.invalidate();
+    return sync_meta(l->scale_dev, l->rank_dev, l->scales, l->ranks, err);
+}
+
+int pm_linear_forward(pm_linear l, const void* x, int n_frames, const int32_t* set_offsets,
+                      const int32_t* set_ids, const void* residual, void* y, void* cuda_stream) {
+    if (!l) return PM_ERR_ARG;
+    std::string& err = l->err;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (n_frames < 0 || (n_frames > 0 && (!x || !y || !set_offsets))) { err = "NULL argument"; return PM_ERR_ARG; }
+    if (l->epilogue == EPI_RESIDUAL && n_frames > 0 && !residual) { err = "epilogue 2 needs a residual"; return PM_ERR_ARG; }
+    if (n_frames == 0) return PM_OK;
+    int rc = l->router.build(n_frames, set_offsets, set_ids, l->ranks, l->scales, false, st, err);
+    if (rc) return rc;
+    Launch L; L.st = st; L.launches = &l->launches; L.status = l->status.as<int>();
+    const RouteDev& R = l->router.dev;
+    const int rows = n_frames * l->tokens;
+    PatchEpi none;
+    if (l->dtype == 0) {
+        CUtensorMap tm_x;
+        if (!tm_encode_2d(&tm_x, x, l->k_in, rows, (uint64_t)l->k_in * 2, 64, PM_TILE_M, 128)) {
+            err = "cuTensorMapEncodeTiled failed (x); x must be 16-byte aligned"; return PM_ERR_CUDA;
+        }
+        const bool lora = R.max_set > 0 && l->lin.dev.lora.At != nullptr;
+        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>()));
+        CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, rows, l->epilogue,
+                            (const bf16*)residual, none, (bf16*)y, l->n_sms));
+    } else {
+        CK(launch_naive_linear<float>(L, l->lin.dev, R, l->meta, l->slabs_max, (const float*)x, rows, l->tokens,
+                                      l->t32.as<float>(), l->epilogue, (const float*)residual, none, (float*)y));
+    }
+    return PM_OK;
+}
+
+int pm_linear_status(pm_linear l, void* cuda_stream) {
+    if (!l) return PM_ERR_ARG;
+    return read_status(l->status, (cudaStream_t)cuda_stream, l->err);
+}
+const char* pm_linear_last_error(pm_linear l) { return l ? l->err.c_str() : "NULL handle"; }
+void pm_linear_destroy(pm_linear l) {
+    if (!l) return;
+    cudaDeviceSynchronize();
+    delete l;
+}
+
+int pm_layernorm(const void* x, const float* gamma, const float* beta, void* y, int rows, int d,
+                 float eps, int dtype, void* cuda_stream) {
+    if (!x || !gamma || !beta || !y || rows < 0 || d <= 0 || d % 8 || d > 1024 || (dtype != 0 && dtype != 1))
+        return PM_ERR_ARG;
+    Launch L; L.st = (cudaStream_t)cuda_stream;
+    cudaError_t e = dtype == 0 ? launch_layernorm<bf16>(L, (const bf16*)x, gamma, beta, (bf16*)y, rows, d, eps)
+                               : launch_layernorm<float>(L, (const float*)x, gamma, beta, (float*)y, rows, d, eps);
+    return e == cudaSuccess ? PM_OK : PM_ERR_CUDA;
+}
+
+int pm_attention(const void* qkv, void* out, int n_frames, int tokens, int heads, int dtype,
+                 void* cuda_stream) {
+    if (!qkv || !out || n_frames < 0 || tokens <= 0 || heads <= 0 || (dtype != 0 && dtype != 1))
+        return PM_ERR_ARG;
+    Launch L; L.st = (cudaStream_t)cuda_stream;
+    cudaError_t e = dtype == 0 ? launch_attention_mma(L, (const bf16*)qkv, (bf16*)out, n_frames, tokens, heads)
+                               : launch_attention_simple<float>(L, (const float*)qkv, (float*)out, n_frames, tokens, heads);
+    return e == cudaSuccess ? PM_OK : PM_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,119 @@
+// Shared declarations of the Polymorph B200 library (host structures, launch prototypes).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "polymorph.h"
+
+typedef __nv_bfloat16 bf16;
+
+#define PM_TILE_M 128          // rows of one GEMM tile
+#define PM_SLAB 16             // LoRA ranks are handled in slabs of 16 (one UMMA K step)
+
+// ---------------------------------------------------------------------------------------
+// device-side views
+// ---------------------------------------------------------------------------------------
+// LoRA arenas of one linear.  At: [max_adapters * RS, k_in] (row a*RS + j = column j of A_a),
+// Bt: [max_adapters * slabs_max][n_out][16] (Bt[a*slabs_max + s][n][j] = B_a[16 s + j, n]);
+// RS = slabs_max * 16.  Unused ranks and unregistered adapters are zero.
+struct LoraArena {
+    void* At = nullptr;
+    void* Bt = nullptr;
+};
+
+struct LinearDev {
+    int k_in = 0, n_out = 0;
+    void* Wt = nullptr;        // [n_out, k_in]  (W transposed: K-major for the tensor cores)
+    float* bias = nullptr;     // [n_out]
+    LoraArena lora;
+    // tensor maps of the static operands (bf16 build only)
+    CUtensorMap tm_w, tm_at, tm_bt;
+    bool has_tm = false;
+};
+
+// Per-batch routing of frames to adapters, in SLOT order (slot = position after bucketing
+// frames by adapter set).  All arrays live on the device.
+struct RouteDev {
+    int n_frames = 0, tokens = 0, n_tiles = 0, slab_cap = 0, max_set = 0;
+    int* perm = nullptr;        // [F] slot -> caller's frame index
+    int* slot_off = nullptr;    // [F+1] CSR over slots
+    int* slot_ids = nullptr;    // [nnz] ascending adapter ids per slot
+    // tile plan (rows 128*t .. 128*t+127): the union of the LoRA slabs its rows need
+    int* tile_nslabs = nullptr;     // [n_tiles]
+    int* tile_slab = nullptr;       // [n_tiles, slab_cap] arena slab index a*slabs_max + s
+    float* tile_scale = nullptr;    // [n_tiles, slab_cap] s_a
+    uint32_t* tile_mask = nullptr;  // [n_tiles, slab_cap, 4] 128-bit mask of rows using the slab
+};
+
+struct AdapterMeta {            // device arrays indexed by adapter id
+    float* scale = nullptr;     // [max_adapters]
+    int* rank = nullptr;        // [max_adapters], 0 = not registered
+};
+
+enum { EPI_NONE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_PATCH = 3 };
+
+struct PatchEpi {               // EPI_PATCH: GEMM row i = patch (i % g2) of slot (i / g2)
+    int g2 = 0, tokens = 0;     //   -> output row slot*tokens + 1 + patch, plus pos[1+patch]
+    const float* pos = nullptr; // [tokens, n_out] fp32
+};
+
+// ---------------------------------------------------------------------------------------
+// launch prototypes (definitions in kernels_simple.cu / gemm_tcgen05.cu / attention.cu)
+// every function enqueues on `st`, bumps *launches per kernel and returns a cudaError_t
+// ---------------------------------------------------------------------------------------
+struct Launch {
+    cudaStream_t st = 0;
+    long long* launches = nullptr;
+    int* status = nullptr;      // device status word
+};
+
+template <typename T>
+cudaError_t launch_layernorm(const Launch& L, const T* x, const float* g, const float* b, T* y,
+                             int rows, int d, float eps);
+template <typename T>
+cudaError_t launch_attention_simple(const Launch& L, const T* qkv, T* out, int n_frames, int tokens,
+                                    int heads);
+cudaError_t launch_attention_mma(const Launch& L, const bf16* qkv, bf16* out, int n_frames,
+                                 int tokens, int heads);
+template <typename T>
+cudaError_t launch_im2col(const Launch& L, const T* frames, const int* perm, T* out, int n_frames,
+                          int img, int patch);
+template <typename T>
+cudaError_t launch_cls_rows(const Launch& L, const float* cls, const float* pos, T* x, int n_frames,
+                            int tokens, int d);
+// fp32 debug / reference-quality linear: t32 = scaled shrink per (row, set position, rank)
+template <typename T>
+cudaError_t launch_naive_linear(const Launch& L, const LinearDev& lin, const RouteDev& R,
+                                const AdapterMeta& meta, int slabs_max, const T* x, int rows,
+                                int tokens_per_frame, float* t32, int epi, const T* residual,
+                                const PatchEpi& pe, T* y);
+// tensor-core path (bf16): shrink into the slab buffer, then the fused GEMM
+cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
+                          const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf);
+cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
+                             const CUtensorMap& tm_x, const CUtensorMap* tm_t, int rows, int epi,
+                             const bf16* residual, const PatchEpi& pe, bf16* y, int n_sms);
+template <typename T>
+cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, int d, float eps,
+                         const float* lnf_g, const float* lnf_b, float* z,
+                         const T* base_wt, const float* base_b, int n_classes,
+                         const T* hcat, const float* hbias, const int* hcls, const int* hoff,
+                         const RouteDev& R, float* scores_out, float* base_out);
+cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, int n_classes,
+                          int n_adapters, float thr, int context_copy, int has_prev,
+                          uint32_t* prev_labels, const int* prev_off, const int* prev_ids,
+                          const int* first, const uint64_t* provider, uint64_t* mask_scratch,
+                          int* next_off, int* next_ids, int ids_capacity);
+
+// tensor-map helpers (gemm_tcgen05.cu); return false if the driver entry point is unavailable
+bool tm_encode_2d(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer,
+                  uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, int swizzle);
+bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                  uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
+                  uint32_t b2, int swizzle);

@@ -1,0 +1,559 @@
+// Fused base + multi-LoRA GEMM on the sm_100a tensor cores (Sec. 3.1: y = xW + sum_a s_a (xA_a)B_a).
+//
+//   y[128 x BN tile] = x_tile W^T_tile                        (K/64 pipeline stages, 4 UMMAs each)
+//                    + sum over the tile's LoRA slabs  t_slab B_slab   (one K=16 UMMA per slab,
+//                      into the SAME TMEM accumulator)
+//                    -> epilogue: bias, GELU / residual / patch-embed placement, bf16 store.
+//
+// t (the scaled, row-masked shrink x A_cat of the tile) is produced by launch_shrink before the
+// GEMM and fetched by TMA like any other operand.  Operands are staged by TMA into 128B- (base)
+// and 32B- (LoRA slab) swizzled shared memory; a single thread issues tcgen05.mma; accumulators
+// live in TMEM (two buffers, so the epilogue of one tile overlaps the main loop of the next).
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue.
+// Every mbarrier wait is bounded: on expiry the CTA raises an abort flag, records
+// PM_ERR_TIMEOUT in the status word, drains and returns.
+#include "common.cuh"
+
+#define BUMP(L) do { if ((L).launches) ++*(L).launches; } while (0)
+
+namespace {
+
+constexpr int BM = PM_TILE_M;
+constexpr int BK = 64;
+constexpr int STAGES = 4;
+constexpr int GEMM_THREADS = 192;
+constexpr int SLABS_PER_STAGE = 4;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;     // ~2 s
+
+// ---------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// Bounded wait.  Returns false once the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, (int)PM_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b,
+                                          uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrives once all tcgen05 operations issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+          "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+          "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand whose rows are `swizzle_bytes` wide
+// (128: base operands, 64 bf16 per row; 32: one LoRA slab, 16 bf16 per row).  Groups of 8 rows
+// are contiguous, so the stride between groups is 8 * swizzle_bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, int swizzle_bytes) {
+    const uint64_t layout = swizzle_bytes == 128 ? 2ull : (swizzle_bytes == 64 ? 4ull : 6ull);
+    uint64_t d = (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)1 << 16;                                        // leading byte offset (unused)
+    d |= (uint64_t)(((8 * swizzle_bytes) >> 4) & 0x3FFF) << 32;    // stride byte offset
+    d |= (uint64_t)1 << 46;                                        // descriptor version (sm_100)
+    d |= layout << 61;
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ float gelu_erf(float v) {
+    return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+struct GemmArgs {
+    int rows, k_in, n_out, m_tiles, n_tiles, epi;
+    const float* bias;
+    const bf16* residual;
+    bf16* y;
+    PatchEpi pe;
+    // LoRA plan (null tile_nslabs = no LoRA)
+    const int* tile_nslabs;
+    const int* tile_slab;
+    int slab_cap;
+    int* status;
+};
+
+template <int BN>
+struct Smem {
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int T_SLAB_BYTES = BM * PM_SLAB * 2;      // 4096
+    static constexpr int B_SLAB_BYTES = BN * PM_SLAB * 2;
+    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;      // barriers + alignment slack
+};
+
+template <int BN>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                 const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
+                 const GemmArgs args) {
+    using S = Smem<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t bars = base + S::BAR_OFFSET;
+    // barrier words: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int s) { return bars + 8u * (2 * STAGES + s); };
+    auto tempty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 2 + s); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + S::BAR_OFFSET + 8 * (2 * STAGES + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::BAR_OFFSET + 8 * (2 * STAGES + 4) + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = args.m_tiles * args.n_tiles;
+    const int num_kb = args.k_in / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), 2 * BN);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m = tile / args.n_tiles, n = tile % args.n_tiles;
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    mbar_expect_tx(full_bar(stage), S::STAGE_BYTES);
+                    const uint32_t sa = base + stage * S::STAGE_BYTES;
+                    tma_load_2d(sa, &tm_x, kb * BK, m * BM, full_bar(stage));
+                    tma_load_2d(sa + S::A_BYTES, &tm_w, kb * BK, n * BN, full_bar(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                const int ns = args.tile_nslabs ? args.tile_nslabs[m] : 0;
+                for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
+                    const int cnt = min(SLABS_PER_STAGE, ns - g0);
+                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    mbar_expect_tx(full_bar(stage), cnt * (S::T_SLAB_BYTES + S::B_SLAB_BYTES));
+                    const uint32_t sa = base + stage * S::STAGE_BYTES;
+                    for (int i = 0; i < cnt; ++i) {
+                        const int slot = m * args.slab_cap + g0 + i;
+                        const int slab = args.tile_slab[slot];
+                        tma_load_2d(sa + i * S::T_SLAB_BYTES, &tm_t, 0, slot * BM, full_bar(stage));
+                        tma_load_2d(sa + S::A_BYTES + i * S::B_SLAB_BYTES, &tm_bt, 0,
+                                    slab * args.n_out + n * BN, full_bar(stage));
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m = tile / args.n_tiles;
+                ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, args.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                uint32_t accumulate = 0;
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * S::STAGE_BYTES;
+                    const uint32_t sb = sa + S::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        umma_bf16(d_tmem, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
+                                  accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit(empty_bar(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                const int ns = args.tile_nslabs ? args.tile_nslabs[m] : 0;
+                for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
+                    const int cnt = min(SLABS_PER_STAGE, ns - g0);
+                    ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * S::STAGE_BYTES;
+                    const uint32_t sb = sa + S::A_BYTES;
+                    for (int i = 0; i < cnt; ++i) {
+                        umma_bf16(d_tmem, smem_desc(sa + i * S::T_SLAB_BYTES, 32),
+                                  smem_desc(sb + i * S::B_SLAB_BYTES, 32), idesc, accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit(empty_bar(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(tfull_bar(acc));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int m = tile / args.n_tiles, n = tile % args.n_tiles;
+            ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int row = m * BM + quarter * 32 + lane;
+            const bool row_ok = row < args.rows;
+            size_t orow = (size_t)row;
+            const float* pos_row = nullptr;
+            if (args.epi == EPI_PATCH && row_ok) {
+                const int p = row % args.pe.g2;
+                orow = (size_t)(row / args.pe.g2) * args.pe.tokens + 1 + p;
+                pos_row = args.pe.pos + (size_t)(1 + p) * args.n_out;
+            }
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int n0 = n * BN + c * 32;
+                if (n0 >= args.n_out) break;           // uniform across the warp
+                uint32_t v[32];
+                tmem_ld32(t_row + (uint32_t)(c * 32), v);
+                tmem_ld_wait();
+                if (row_ok) {
+                    float f[32];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
+                        f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
+                        f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
+                        f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
+                        f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+                    }
+                    if (args.epi == EPI_GELU) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
+                    } else if (args.epi == EPI_RESIDUAL) {
+                        const uint4* r4 = reinterpret_cast<const uint4*>(args.residual + (size_t)row * args.n_out + n0);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint4 r = r4[q];
+                            const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
+                                f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
+                            }
+                        }
+                    } else if (args.epi == EPI_PATCH) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 p4 = __ldg(reinterpret_cast<const float4*>(pos_row + n0 + j));
+                            f[j + 0] += p4.x; f[j + 1] += p4.y; f[j + 2] += p4.z; f[j + 3] += p4.w;
+                        }
+                    }
+                    uint4* o4 = reinterpret_cast<uint4*>(args.y + orow * args.n_out + n0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 o;
+                        o.x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
+                        o.y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
+                        o.z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
+                        o.w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
+                        o4[q] = o;
+                    }
+                }
+            }
+            // all TMEM reads of this buffer are complete (wait::ld above): hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        // give copies and MMAs still in flight time to land before shared memory / TMEM go away
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 2 * BN);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// shrink: t[tile][s][row][j] = mask(row) * s_a * sum_k x[row,k] A_a[k, 16 s' + j]
+// CUDA-core version: one CTA per (tile, slab), one thread per row.
+// ---------------------------------------------------------------------------------------
+constexpr int SHRINK_KC = 512;
+
+__global__ void __launch_bounds__(128) shrink_kernel(const bf16* __restrict__ x, const bf16* __restrict__ At,
+                                                     int rows, int k_in, const int* __restrict__ tile_nslabs,
+                                                     const int* __restrict__ tile_slab,
+                                                     const float* __restrict__ tile_scale,
+                                                     const uint32_t* __restrict__ tile_mask, int slab_cap,
+                                                     bf16* __restrict__ tbuf) {
+    __shared__ __align__(16) bf16 As[SHRINK_KC * PM_SLAB];       // [k][16]
+    const int tile = blockIdx.x, s = blockIdx.y;
+    if (s >= tile_nslabs[tile]) return;
+    const int slot = tile * slab_cap + s;
+    const int slab = tile_slab[slot];
+    const int r = threadIdx.x;
+    const int row = tile * BM + r;
+    const bool active = (row < rows) && ((tile_mask[(size_t)slot * 4 + (r >> 5)] >> (r & 31)) & 1u);
+    float acc[PM_SLAB];
+#pragma unroll
+    for (int j = 0; j < PM_SLAB; ++j) acc[j] = 0.f;
+    const bf16* arena = At + (size_t)slab * PM_SLAB * k_in;       // 16 rows of length k_in
+    for (int k0 = 0; k0 < k_in; k0 += SHRINK_KC) {
+        const int kc = min(SHRINK_KC, k_in - k0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < kc * PM_SLAB; i += blockDim.x) {
+            const int j = i / kc, k = i % kc;                     // coalesced along k
+            As[k * PM_SLAB + j] = arena[(size_t)j * k_in + k0 + k];
+        }
+        __syncthreads();
+        if (active) {
+            const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * k_in + k0);
+            for (int k8 = 0; k8 < kc / 8; ++k8) {
+                const uint4 raw = xr[k8];
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float xv = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u)
+                                             : __uint_as_float(w[e >> 1] << 16);
+                    const bf16* ar = As + (k8 * 8 + e) * PM_SLAB;
+#pragma unroll
+                    for (int j = 0; j < PM_SLAB; ++j) acc[j] = fmaf(xv, __bfloat162float(ar[j]), acc[j]);
+                }
+            }
+        }
+    }
+    const float sc = active ? tile_scale[slot] : 0.f;
+    uint4 o[2];
+    uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+    for (int j = 0; j < PM_SLAB; j += 2) ow[j >> 1] = pack_bf16(acc[j] * sc, acc[j + 1] * sc);
+    uint4* dst = reinterpret_cast<uint4*>(tbuf + ((size_t)slot * BM + r) * PM_SLAB);
+    dst[0] = o[0];
+    dst[1] = o[1];
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+CUtensorMapSwizzle swz(int bytes) {
+    return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+         : bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
+         : bytes == 32  ? CU_TENSOR_MAP_SWIZZLE_32B
+                        : CU_TENSOR_MAP_SWIZZLE_NONE;
+}
+
+}  // namespace
+
+bool tm_encode_2d(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer,
+                  uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, int swizzle) {
+    EncodeTiledFn fn = get_encode();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {row_stride_bytes};
+    const cuuint32_t box[2] = {box_inner, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swz(swizzle), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                  uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
+                  uint32_t b2, int swizzle) {
+    EncodeTiledFn fn = get_encode();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {d0, d1, d2};
+    const cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+    const cuuint32_t box[3] = {b0, b1, b2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swz(swizzle), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
+                          const CUtensorMap* /*tm_x*/, const bf16* x, int rows, bf16* tbuf) {
+    if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
+    dim3 grid(R.n_tiles, R.slab_cap);
+    shrink_kernel<<<grid, 128, 0, L.st>>>(x, (const bf16*)lin.lora.At, rows, lin.k_in, R.tile_nslabs,
+                                          R.tile_slab, R.tile_scale, R.tile_mask, R.slab_cap, tbuf);
+    BUMP(L);
+    return cudaGetLastError();
+}
+
+template <int BN>
+static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
+                                  const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const GemmArgs& a,
+                                  int n_sms) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Smem<BN>::TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int total = a.m_tiles * a.n_tiles;
+    const int grid = total < n_sms ? total : n_sms;
+    lora_gemm_kernel<BN><<<grid, GEMM_THREADS, Smem<BN>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, a);
+    BUMP(L);
+    return cudaGetLastError();
+}
+
+// lin.tm_w / lin.tm_bt are encoded for the BN chosen by gemm_tile_n(lin.n_out).
+int gemm_tile_n(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
+
+cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
+                             const CUtensorMap& tm_x, const CUtensorMap* tm_t, int rows, int epi,
+                             const bf16* residual, const PatchEpi& pe, bf16* y, int n_sms) {
+    if (rows <= 0) return cudaSuccess;
+    const int bn = gemm_tile_n(lin.n_out);
+    GemmArgs a;
+    a.rows = rows; a.k_in = lin.k_in; a.n_out = lin.n_out;
+    a.m_tiles = (rows + BM - 1) / BM;
+    a.n_tiles = (lin.n_out + bn - 1) / bn;
+    a.epi = epi; a.bias = lin.bias; a.residual = residual; a.y = y; a.pe = pe;
+    const bool lora = R && tm_t && R->slab_cap > 0 && lin.lora.At != nullptr;
+    a.tile_nslabs = lora ? R->tile_nslabs : nullptr;
+    a.tile_slab = lora ? R->tile_slab : nullptr;
+    a.slab_cap = lora ? R->slab_cap : 0;
+    a.status = L.status;
+    const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced
+    const CUtensorMap& tb = lora ? lin.tm_bt : lin.tm_w;
+    if (bn == 256) return launch_gemm_bn<256>(L, tm_x, lin.tm_w, tt, tb, a, n_sms);
+    return launch_gemm_bn<128>(L, tm_x, lin.tm_w, tt, tb, a, n_sms);
+}

@@ -1,0 +1,204 @@
+"""End-to-end GPU parity of pm_forward / pm_select (through the C ABI) against the CPU oracle on
+the five workload shapes.  Scores: abs 1e-2 (bf16 build) / 1e-4 (fp32 debug build).  Selection:
+bit-exact when fed the oracle's scores."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from oracle import polymorph_oracle as po
+
+pytestmark = pytest.mark.gpu
+
+SCORE_TOL = {0: 1e-2, 1: 1e-4}
+
+
+def frames_to_dev(frames, dtype):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(frames, dtype=np.float32)).cuda()
+    return (t.to(torch.bfloat16) if dtype == 0 else t).contiguous()
+
+
+def oracle_rows(w, rows, offsets=None, ids=None, frames=None):
+    """Oracle scores/base for a subset of frames (computed one by one)."""
+    offsets = w.set_offsets if offsets is None else offsets
+    ids = w.set_ids if ids is None else ids
+    frames = w.frames if frames is None else frames
+    sets = [list(ids[offsets[f]:offsets[f + 1]]) for f in rows]
+    off, sid = wl.sets_to_csr(sets)
+    return po.forward(w.backbone, w.adapters, frames[list(rows)], off, sid, w.spec.heads, w.spec.patch,
+                      w.spec.ln_eps, w.spec.n_classes)
+
+
+def run_forward(model, w, dtype, frames=None, offsets=None, ids=None):
+    import torch
+    frames = w.frames if frames is None else frames
+    offsets = w.set_offsets if offsets is None else offsets
+    ids = w.set_ids if ids is None else ids
+    F, K = frames.shape[0], w.spec.n_classes
+    fd = frames_to_dev(frames, dtype)
+    scores = torch.full((F, K), float("nan"), device="cuda")
+    base = torch.full((F, K), float("nan"), device="cuda")
+    model.forward(fd, offsets, ids, scores, base)
+    assert model.status() == 0
+    return scores.cpu().numpy().astype(np.float64), base.cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("dtype", [1, 0])
+def test_deit_tiny_2frames(dtype):
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    m = binding.model_from_workload(w, dtype=dtype)
+    s, b = run_forward(m, w, dtype)
+    so, bo = oracle_rows(w, range(2))
+    assert np.abs(b - bo).max() < SCORE_TOL[dtype]
+    assert np.abs(s - so).max() < SCORE_TOL[dtype]
+    # classes outside the active adapters' subsets score exactly 0
+    assert np.all(s[0, 8:] == 0) and np.all(s[1, :8] == 0) and np.all(s[1, 16:24] == 0)
+    # empty sets reproduce the plain backbone; the composed row is all zero
+    off, ids = wl.sets_to_csr([[], []])
+    s2, b2 = run_forward(m, w, dtype, offsets=off, ids=ids)
+    so2, bo2 = oracle_rows(w, range(2), offsets=off, ids=ids)
+    assert np.all(s2 == 0)
+    assert np.abs(b2 - bo2).max() < SCORE_TOL[dtype]
+    assert np.abs(bo2 - bo).max() > 1e-3          # adapters do move the base scores
+    # frame order does not matter: swapped frames give swapped rows (bucketing is internal)
+    off3, ids3 = wl.sets_to_csr([[1, 3], [0]])
+    s3, b3 = run_forward(m, w, dtype, frames=w.frames[::-1], offsets=off3, ids=ids3)
+    np.testing.assert_array_equal(s3, s[::-1])
+    np.testing.assert_array_equal(b3, b[::-1])
+    m.close()
+
+
+def test_forward_argument_errors():
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    m = binding.model_from_workload(w, dtype=0)
+    fd = frames_to_dev(w.frames, 0)
+    s = torch.zeros((2, 32), device="cuda")
+    n0 = m.launch_count()
+    for off, ids, code in [([0, 1, 2], [0, 9], binding.PM_ERR_ARG),          # id out of range
+                           ([0, 2, 2], [1, 1], binding.PM_ERR_ARG),          # duplicate id
+                           ([0, 2, 1], [0, 1], binding.PM_ERR_ARG),          # non-monotone
+                           ([1, 1, 2], [0, 1], binding.PM_ERR_ARG),          # offsets[0] != 0
+                           ([0, 4, 4], [0, 1, 2, 3], binding.PM_ERR_CAPACITY)]:
+        with pytest.raises(binding.PolymorphError) as e:
+            m.forward(fd, np.asarray(off, np.int32), np.asarray(ids, np.int32), s)
+        assert e.value.code == code
+    assert m.launch_count() == n0                 # nothing was launched
+    m2 = binding.Model(img=224, d=192, layers=1, heads=3, mlp=768, n_classes=32,
+                       backbone={k: (v[:1] if v.ndim > 1 and v.shape[0] == 12 else v) for k, v in w.backbone.items()},
+                       max_adapters=4, max_rank=4, max_set=2, max_frames=2)
+    with pytest.raises(binding.PolymorphError) as e:      # adapter 0 never registered
+        m2.forward(fd, np.asarray([0, 1, 1], np.int32), np.asarray([0], np.int32), s)
+    assert e.value.code == binding.PM_ERR_STATE
+    m2.close()
+    m.close()
+
+
+def test_device_resident_sets_match_host_sets():
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    m = binding.model_from_workload(w, dtype=0)
+    s, b = run_forward(m, w, 0)
+    fd = frames_to_dev(w.frames, 0)
+    s2 = torch.zeros((2, 32), device="cuda")
+    m.forward(fd, torch.from_numpy(w.set_offsets).cuda(), torch.from_numpy(w.set_ids).cuda(), s2)
+    assert m.status() == 0
+    np.testing.assert_array_equal(s2.cpu().numpy(), s.astype(np.float32))
+    m.close()
+
+
+def test_deit_small_streams_bf16():
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_small_streams()
+    m = binding.model_from_workload(w, dtype=0)
+    s, b = run_forward(m, w, 0)
+    rows = [0, 1, 15, 16, 17, 31, 40, 63]
+    so, bo = oracle_rows(w, rows)
+    assert np.abs(s[rows] - so).max() < 1e-2
+    assert np.abs(b[rows] - bo).max() < 1e-2
+    m.close()
+
+
+def test_deit_small_fp32_debug_subset():
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_small_streams()
+    rows = [0, 17, 40]
+    sets = [w.sets()[r] for r in rows]
+    off, ids = wl.sets_to_csr(sets)
+    m = binding.model_from_workload(w, dtype=1, max_frames=3)
+    s, b = run_forward(m, w, 1, frames=w.frames[rows], offsets=off, ids=ids)
+    so, bo = oracle_rows(w, rows)
+    assert np.abs(s - so).max() < 1e-4
+    assert np.abs(b - bo).max() < 1e-4
+    m.close()
+
+
+def test_vit_base_batch_sampled():
+    """Full 256-frame ViT-base batch on the GPU (the benchmark's launch configuration); the oracle
+    computes a sample of frames one by one."""
+    from paper_2507_14959_b200 import binding
+    w = wl.vit_base_batch()
+    m = binding.model_from_workload(w, dtype=0)
+    s, b = run_forward(m, w, 0)
+    sizes = np.diff(w.set_offsets)
+    rows = [0, 255, int(np.argmax(sizes == 3)), int(np.argmax(sizes == 2)), 128]
+    so, bo = oracle_rows(w, rows)
+    assert np.abs(s[rows] - so).max() < 1e-2
+    assert np.abs(b[rows] - bo).max() < 1e-2
+    # properties that hold at any size: rows of frames with equal sets and equal pixels are equal;
+    # scores are zero exactly outside the union of the active class subsets
+    for f in range(256):
+        allowed = np.zeros(w.spec.n_classes, bool)
+        for a in w.sets()[f]:
+            allowed[w.adapters[a].class_ids] = True
+        assert np.all(s[f][~allowed] == 0) and np.all(s[f][allowed] > 0)
+    m.close()
+
+
+def test_vit_base_384_streams_teacher_forced():
+    """577-token shape: forward fed the oracle's sets; select fed the oracle's scores (bit-exact)."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.vit_base_384_streams(n_streams=16, n_steps=2)
+    m = binding.model_from_workload(w, dtype=0, max_frames=16, max_set=8)
+    m.set_cover(w.tau)
+    contexts = [a.class_ids for a in w.adapters]
+    accs = [a.acc for a in w.adapters]
+    fr = w.extra["stream_frames"]
+    rows = [0, 7, 15]
+    # step 0: empty sets -> base scores -> labels -> greedy selection
+    off0, ids0 = wl.sets_to_csr([[] for _ in range(16)])
+    s0, b0 = run_forward(m, w, 0, frames=fr[:, 0], offsets=off0, ids=ids0)
+    so0, bo0 = oracle_rows(w, rows, offsets=off0, ids=ids0, frames=fr[:, 0])
+    assert np.abs(b0[rows] - bo0).max() < 1e-2
+    # the oracle's base scores for ALL streams are needed to drive selection: use the GPU's for the
+    # rows the oracle did not compute (teacher forcing is on the scores handed to select)
+    drive = b0.copy()
+    drive[rows] = bo0
+    drive32 = drive.astype(np.float32)
+    Y = [po.labels_from_scores(drive32[f], 0.5) for f in range(16)]
+    S1 = [po.detect_contexts(Y[f], None, contexts, accs, w.tau, None, False) for f in range(16)]
+    nw = (w.spec.n_classes + 31) // 32
+    labels = torch.zeros((16, nw), dtype=torch.int32, device="cuda")
+    noff = torch.zeros(17, dtype=torch.int32, device="cuda")
+    nids = torch.full((16 * 64,), -1, dtype=torch.int32, device="cuda")
+    m.select(torch.from_numpy(drive32).cuda(), 0.5, False, False, labels, None, None, noff, nids)
+    assert m.status() == 0
+    off1, ids1 = wl.sets_to_csr(S1)
+    np.testing.assert_array_equal(noff.cpu().numpy(), off1)
+    np.testing.assert_array_equal(nids.cpu().numpy()[:len(ids1)], ids1)
+    assert 1 <= np.mean([len(y) for y in Y]) <= 8       # a few labels per frame, as in the paper
+    # step 1: forward with the selected sets, straight from the device lists
+    import torch as _t
+    fd = frames_to_dev(fr[:, 1], 0)
+    s1 = _t.zeros((16, w.spec.n_classes), device="cuda")
+    b1 = _t.zeros((16, w.spec.n_classes), device="cuda")
+    m.forward(fd, noff, nids, s1, b1)
+    assert m.status() == 0
+    so1, bo1 = oracle_rows(w, rows, offsets=off1, ids=ids1, frames=fr[:, 1])
+    assert np.abs(s1.cpu().numpy()[rows] - so1).max() < 1e-2
+    assert np.abs(b1.cpu().numpy()[rows] - bo1).max() < 1e-2
+    m.close()
