@@ -150,6 +150,15 @@ const char* pm_last_error(pm_handle h);
 /* Number of kernels the library has launched on this handle since creation. */
 long long pm_launch_count(pm_handle h);
 
+/* Device timing of the library's own kernels, by class, with CUDA events recorded on the launching
+ * stream around each launch site: class 0 fused base+LoRA GEMM (patch embed included), 1 LoRA
+ * shrink, 2 attention, 3 LayerNorm, 4 everything else (patch gather, CLS rows, heads, select).
+ * pm_profile_enable(h, 1) clears and starts recording, (h, 0) stops.  pm_profile_read synchronises
+ * the stream, returns total milliseconds and launch-site counts per class (arrays of 5) since the
+ * last read, and clears them. */
+int pm_profile_enable(pm_handle h, int on);
+int pm_profile_read(pm_handle h, void* cuda_stream, double* ms_by_class, long long* launches_by_class);
+
 /* ---- single operators (the same kernels pm_forward uses), for unit tests and sweeps ----- */
 
 /* One base + multi-LoRA linear y = epilogue(x W + b + sum_a s_a (x A_a) B_a)   (Sec. 3.1).

@@ -21,7 +21,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
 
 EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_select",
-    "pm_status", "pm_last_error", "pm_launch_count", "pm_linear_create", "pm_linear_register",
+    "pm_status", "pm_last_error", "pm_launch_count", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention",
 ]
@@ -81,6 +81,8 @@ def load():
     lib.pm_last_error.restype = C.c_char_p
     lib.pm_launch_count.argtypes = [vp]
     lib.pm_launch_count.restype = C.c_longlong
+    lib.pm_profile_enable.argtypes = [vp, ip]
+    lib.pm_profile_read.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.pm_linear_create.argtypes = [ip, ip, _FP, _FP, ip, ip, ip, ip, ip, ip, ip, C.POINTER(vp)]
     lib.pm_linear_register.argtypes = [vp, ip, ip, C.c_float, _FP, _FP]
     lib.pm_linear_forward.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
@@ -179,6 +181,18 @@ class Model:
 
     def status(self, stream=None):
         return self.lib.pm_status(self.handle, _stream_ptr(stream))
+
+    KERNEL_CLASSES = ("gemm", "shrink", "attention", "layernorm", "other")
+
+    def profile_enable(self, on):
+        self._check(self.lib.pm_profile_enable(self.handle, int(on)), "pm_profile_enable")
+
+    def profile_read(self, stream=None):
+        """{class: (total_ms, launch_sites)} since the last read; synchronises the stream."""
+        ms = (C.c_double * 5)()
+        n = (C.c_longlong * 5)()
+        self._check(self.lib.pm_profile_read(self.handle, _stream_ptr(stream), ms, n), "pm_profile_read")
+        return {k: (ms[i], int(n[i])) for i, k in enumerate(self.KERNEL_CLASSES)}
 
     def launch_count(self):
         return int(self.lib.pm_launch_count(self.handle))

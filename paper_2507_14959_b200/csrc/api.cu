@@ -317,6 +317,7 @@ struct pm_handle_s {
     DevBuf first, provider, mask_scratch;
     bool cover_ready = false;
     long long launches = 0;
+    Profiler prof;
     std::string err;
 };
 
@@ -382,7 +383,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     std::string& err = h->err;
     const pm_config& c = h->cfg;
     const int T_ = h->tokens, d = c.d, rows = n_frames * T_;
-    Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>();
+    Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
     const RouteDev& R = h->router.dev;
     constexpr bool TC = sizeof(T) == 2;
     if (TC) { int rc = encode_activation_maps(h, rows); if (rc) return rc; }
@@ -627,6 +628,7 @@ int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, i
     if (has_prev && (!prev_labels || !prev_offsets || !prev_ids)) { err = "has_prev needs prev_labels, prev_offsets and prev_ids"; return PM_ERR_ARG; }
     if (n_frames > h->cfg.max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
     Launch L; L.st = (cudaStream_t)cuda_stream; L.launches = &h->launches; L.status = h->status.as<int>();
+    L.prof = &h->prof;
     CK(launch_select(L, scores, n_frames, h->cfg.n_classes, h->cfg.max_adapters, score_thr, context_copy,
                      has_prev, prev_labels, prev_offsets, prev_ids, h->first.as<int>(),
                      h->provider.as<uint64_t>(), h->mask_scratch.as<uint64_t>(), next_offsets, next_ids,
@@ -651,6 +653,28 @@ int pm_status(pm_handle h, void* cuda_stream) {
 }
 
 const char* pm_last_error(pm_handle h) { return h ? h->err.c_str() : "NULL handle"; }
+
+int pm_profile_enable(pm_handle h, int on) {
+    if (!h) return PM_ERR_ARG;
+    h->prof.on = on != 0;
+    if (on) h->prof.used = 0;
+    return PM_OK;
+}
+
+int pm_profile_read(pm_handle h, void* cuda_stream, double* ms_by_class, long long* launches_by_class) {
+    if (!h || !ms_by_class || !launches_by_class) return PM_ERR_ARG;
+    std::string& err = h->err;
+    CK(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    for (int c = 0; c < KC_COUNT; ++c) { ms_by_class[c] = 0.0; launches_by_class[c] = 0; }
+    for (size_t i = 0; i < h->prof.used; ++i) {
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, h->prof.ev[2 * i], h->prof.ev[2 * i + 1]));
+        ms_by_class[h->prof.cls[i]] += ms;
+        launches_by_class[h->prof.cls[i]] += 1;
+    }
+    h->prof.used = 0;
+    return PM_OK;
+}
 long long pm_launch_count(pm_handle h) { return h ? h->launches : 0; }
 
 // ---- single operators -------------------------------------------------------------------

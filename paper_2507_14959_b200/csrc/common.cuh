@@ -67,10 +67,40 @@ struct PatchEpi {               // EPI_PATCH: GEMM row i = patch (i % g2) of slo
 // launch prototypes (definitions in kernels_simple.cu / gemm_tcgen05.cu / attention.cu)
 // every function enqueues on `st`, bumps *launches per kernel and returns a cudaError_t
 // ---------------------------------------------------------------------------------------
+// Optional per-kernel-class device timing (CUDA events on the launching stream).
+enum { KC_GEMM = 0, KC_SHRINK = 1, KC_ATTENTION = 2, KC_LAYERNORM = 3, KC_OTHER = 4, KC_COUNT = 5 };
+struct Profiler {
+    bool on = false;
+    std::vector<cudaEvent_t> ev;     // pairs: 2*i start, 2*i+1 stop
+    std::vector<int> cls;            // class of pair i
+    size_t used = 0;                 // pairs in use
+    ~Profiler() { for (cudaEvent_t e : ev) cudaEventDestroy(e); }
+};
+
 struct Launch {
     cudaStream_t st = 0;
     long long* launches = nullptr;
     int* status = nullptr;      // device status word
+    Profiler* prof = nullptr;
+};
+
+struct ProfScope {              // brackets the launches made while it is alive
+    Profiler* p = nullptr;
+    cudaStream_t st = 0;
+    size_t idx = 0;
+    ProfScope(const Launch& L, int kclass) {
+        if (!L.prof || !L.prof->on) return;
+        p = L.prof; st = L.st;
+        if (p->used * 2 >= p->ev.size()) {
+            cudaEvent_t a, b;
+            if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { p = nullptr; return; }
+            p->ev.push_back(a); p->ev.push_back(b); p->cls.push_back(kclass);
+        }
+        idx = p->used++;
+        p->cls[idx] = kclass;
+        cudaEventRecord(p->ev[2 * idx], st);
+    }
+    ~ProfScope() { if (p) cudaEventRecord(p->ev[2 * idx + 1], st); }
 };
 
 template <typename T>

@@ -509,6 +509,7 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
                           const CUtensorMap* /*tm_x*/, const bf16* x, int rows, bf16* tbuf) {
     if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
+    ProfScope ps(L, KC_SHRINK);
     dim3 grid(R.n_tiles, R.slab_cap);
     shrink_kernel<<<grid, 128, 0, L.st>>>(x, (const bf16*)lin.lora.At, rows, lin.k_in, R.tile_nslabs,
                                           R.tile_slab, R.tile_scale, R.tile_mask, R.slab_cap, tbuf);
@@ -529,6 +530,7 @@ static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, cons
     }
     const int total = a.m_tiles * a.n_tiles;
     const int grid = total < n_sms ? total : n_sms;
+    ProfScope ps(L, KC_GEMM);
     lora_gemm_kernel<BN><<<grid, GEMM_THREADS, Smem<BN>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, a);
     BUMP(L);
     return cudaGetLastError();

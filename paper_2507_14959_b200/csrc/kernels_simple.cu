@@ -133,6 +133,7 @@ template <typename T>
 cudaError_t launch_layernorm(const Launch& L, const T* x, const float* g, const float* b, T* y,
                              int rows, int d, float eps) {
     if (rows <= 0) return cudaSuccess;
+    ProfScope ps(L, KC_LAYERNORM);
     layernorm_kernel<T><<<(rows + 7) / 8, 256, 0, L.st>>>(x, g, b, y, rows, d, eps);
     BUMP(L);
     return cudaGetLastError();
@@ -178,6 +179,7 @@ cudaError_t launch_im2col(const Launch& L, const T* frames, const int* perm, T* 
     const size_t total = (size_t)n_frames * g * g * (3 * patch * patch / Vec16<T>::N);
     const int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     if (blocks == 0) return cudaSuccess;
+    ProfScope ps(L, KC_OTHER);
     im2col_kernel<T><<<blocks, 256, 0, L.st>>>(frames, perm, out, n_frames, img, patch);
     BUMP(L);
     return cudaGetLastError();
@@ -197,6 +199,7 @@ __global__ void cls_rows_kernel(const float* __restrict__ cls, const float* __re
 template <typename T>
 cudaError_t launch_cls_rows(const Launch& L, const float* cls, const float* pos, T* x, int n_frames,
                             int tokens, int d) {
+    ProfScope ps(L, KC_OTHER);
     cls_rows_kernel<T><<<(n_frames * d + 255) / 256, 256, 0, L.st>>>(cls, pos, x, n_frames, tokens, d);
     BUMP(L);
     return cudaGetLastError();
@@ -278,6 +281,7 @@ cudaError_t launch_naive_linear(const Launch& L, const LinearDev& lin, const Rou
                                 int tokens_per_frame, float* t32, int epi, const T* residual,
                                 const PatchEpi& pe, T* y) {
     if (rows <= 0) return cudaSuccess;
+    ProfScope ps(L, KC_GEMM);
     const int RS = slabs_max * PM_SLAB;
     const bool lora = (t32 != nullptr) && lin.lora.At != nullptr && R.max_set > 0;
     if (lora) {
@@ -355,6 +359,7 @@ template <typename T>
 cudaError_t launch_attention_simple(const Launch& L, const T* qkv, T* out, int n_frames, int tokens,
                                     int heads) {
     if (n_frames <= 0) return cudaSuccess;
+    ProfScope ps(L, KC_ATTENTION);
     dim3 grid((tokens + 7) / 8, n_frames * heads);
     attention_simple_kernel<T><<<grid, 256, 8 * tokens * sizeof(float), L.st>>>(qkv, out, tokens, heads);
     BUMP(L);
@@ -435,6 +440,7 @@ cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, 
                          const T* hcat, const float* hbias, const int* hcls, const int* hoff,
                          const RouteDev& R, float* scores_out, float* base_out) {
     if (n_frames <= 0) return cudaSuccess;
+    ProfScope ps(L, KC_OTHER);
     final_ln_kernel<T><<<(n_frames + 7) / 8, 256, 0, L.st>>>(x, lnf_g, lnf_b, z, n_frames, tokens, d, eps);
     BUMP(L);
     if (base_out) {
@@ -569,6 +575,7 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
                           uint32_t* prev_labels, const int* prev_off, const int* prev_ids,
                           const int* first, const uint64_t* provider, uint64_t* mask_scratch,
                           int* next_off, int* next_ids, int ids_capacity) {
+    ProfScope ps(L, KC_OTHER);
     select_kernel<<<1, 1024, 0, L.st>>>(scores, n_frames, n_classes, n_adapters, thr, context_copy,
                                         has_prev, prev_labels, prev_off, prev_ids, first, provider,
                                         mask_scratch, next_off, next_ids, ids_capacity, L.status);
