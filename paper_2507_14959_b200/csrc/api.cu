@@ -87,6 +87,10 @@ struct LinearObj {
             const int bn = gemm_tile_n(n_out);
             bool ok = tm_encode_2d(&dev.tm_w, wt.p, k_in, n_out, (uint64_t)k_in * 2, 64, bn, 128);
             if (ok && dev.lora.At) {
+                ok = tm_encode_2d(&dev.tm_at, at.p, k_in, (uint64_t)max_adapters * slabs_max * PM_SLAB,
+                                  (uint64_t)k_in * 2, 64, PM_SLAB, 128);
+            }
+            if (ok && dev.lora.At) {
                 ok = tm_encode_2d(&dev.tm_bt, bt.p, PM_SLAB, (uint64_t)max_adapters * slabs_max * n_out,
                                   PM_SLAB * 2, PM_SLAB, bn, 32);
             }

@@ -394,61 +394,177 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 }
 
 // ---------------------------------------------------------------------------------------
-// shrink: t[tile][s][row][j] = mask(row) * s_a * sum_k x[row,k] A_a[k, 16 s' + j]
-// CUDA-core version: one CTA per (tile, slab), one thread per row.
+// shrink on the tensor cores: t[tile][s][row][j] = mask(row) * s_a * sum_k x[row,k] A_a[k, 16 s' + j]
+//
+// One CTA per 128-row tile.  The tile's LoRA slabs are taken `sg` at a time: for each group the
+// x tile streams through shared memory once (TMA, 128B swizzle) next to the group's A^T slabs
+// (16 rows of the arena per slab, stacked), one UMMA of N = 16 * slabs per 16 K-columns
+// accumulates into TMEM, and the epilogue warps scale, mask, round to bf16 and store each slab
+// as a [128 x 16] block -- the layout the fused GEMM fetches as a 32B-swizzled operand.
 // ---------------------------------------------------------------------------------------
-constexpr int SHRINK_KC = 512;
+struct ShrinkArgs {
+    int rows, k_in, slab_cap, sg;
+    uint32_t tmem_cols;
+    const int* tile_nslabs;
+    const int* tile_slab;
+    const float* tile_scale;
+    const uint32_t* tile_mask;
+    bf16* tbuf;
+    int* status;
+};
 
-__global__ void __launch_bounds__(128) shrink_kernel(const bf16* __restrict__ x, const bf16* __restrict__ At,
-                                                     int rows, int k_in, const int* __restrict__ tile_nslabs,
-                                                     const int* __restrict__ tile_slab,
-                                                     const float* __restrict__ tile_scale,
-                                                     const uint32_t* __restrict__ tile_mask, int slab_cap,
-                                                     bf16* __restrict__ tbuf) {
-    __shared__ __align__(16) bf16 As[SHRINK_KC * PM_SLAB];       // [k][16]
-    const int tile = blockIdx.x, s = blockIdx.y;
-    if (s >= tile_nslabs[tile]) return;
-    const int slot = tile * slab_cap + s;
-    const int slab = tile_slab[slot];
-    const int r = threadIdx.x;
-    const int row = tile * BM + r;
-    const bool active = (row < rows) && ((tile_mask[(size_t)slot * 4 + (r >> 5)] >> (r & 31)) & 1u);
-    float acc[PM_SLAB];
-#pragma unroll
-    for (int j = 0; j < PM_SLAB; ++j) acc[j] = 0.f;
-    const bf16* arena = At + (size_t)slab * PM_SLAB * k_in;       // 16 rows of length k_in
-    for (int k0 = 0; k0 < k_in; k0 += SHRINK_KC) {
-        const int kc = min(SHRINK_KC, k_in - k0);
-        __syncthreads();
-        for (int i = threadIdx.x; i < kc * PM_SLAB; i += blockDim.x) {
-            const int j = i / kc, k = i % kc;                     // coalesced along k
-            As[k * PM_SLAB + j] = arena[(size_t)j * k_in + k0 + k];
-        }
-        __syncthreads();
-        if (active) {
-            const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * k_in + k0);
-            for (int k8 = 0; k8 < kc / 8; ++k8) {
-                const uint4 raw = xr[k8];
-                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float xv = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u)
-                                             : __uint_as_float(w[e >> 1] << 16);
-                    const bf16* ar = As + (k8 * 8 + e) * PM_SLAB;
-#pragma unroll
-                    for (int j = 0; j < PM_SLAB; ++j) acc[j] = fmaf(xv, __bfloat162float(ar[j]), acc[j]);
+constexpr int SHRINK_STAGES = 3;
+constexpr int SHRINK_X_BYTES = BM * BK * 2;          // 16 KB
+constexpr int SHRINK_A_SLAB_BYTES = PM_SLAB * BK * 2; // 2 KB: 16 arena rows x 64 K-columns
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_at,
+                 const ShrinkArgs args) {
+    const int tile = blockIdx.x;
+    const int ns = args.tile_nslabs[tile];
+    if (ns == 0) return;                                   // uniform: nothing allocated yet
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const int stage_bytes = SHRINK_X_BYTES + args.sg * SHRINK_A_SLAB_BYTES;
+    const int bar_off = SHRINK_STAGES * stage_bytes;
+    const uint32_t bars = base + bar_off;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (SHRINK_STAGES + s); };
+    const uint32_t tfull_bar = bars + 8u * (2 * SHRINK_STAGES);
+    const uint32_t tempty_bar = bars + 8u * (2 * SHRINK_STAGES + 1);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + bar_off + 8 * (2 * SHRINK_STAGES + 2));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + bar_off + 8 * (2 * SHRINK_STAGES + 2) + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = args.k_in / BK;
+    const int n_groups = (ns + args.sg - 1) / args.sg;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SHRINK_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(tfull_bar, 1);
+        mbar_init(tempty_bar, 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), args.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int cnt = min(args.sg, ns - g * args.sg);
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    mbar_expect_tx(full_bar(stage), SHRINK_X_BYTES + cnt * SHRINK_A_SLAB_BYTES);
+                    const uint32_t sa = base + stage * stage_bytes;
+                    tma_load_2d(sa, &tm_x, kb * BK, tile * BM, full_bar(stage));
+                    for (int i = 0; i < cnt; ++i) {
+                        const int slab = args.tile_slab[tile * args.slab_cap + g * args.sg + i];
+                        tma_load_2d(sa + SHRINK_X_BYTES + i * SHRINK_A_SLAB_BYTES, &tm_at, kb * BK,
+                                    slab * PM_SLAB, full_bar(stage));
+                    }
+                    if (++stage == SHRINK_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
-    }
-    const float sc = active ? tile_scale[slot] : 0.f;
-    uint4 o[2];
-    uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int cnt = min(args.sg, ns - g * args.sg);
+                const uint32_t idesc = instr_desc(cnt * PM_SLAB);
+                ok = mbar_wait(tempty_bar, acc_phase ^ 1u, abort_flag, args.status);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t accumulate = 0;
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * stage_bytes;
+                    const uint32_t sb = sa + SHRINK_X_BYTES;
 #pragma unroll
-    for (int j = 0; j < PM_SLAB; j += 2) ow[j >> 1] = pack_bf16(acc[j] * sc, acc[j + 1] * sc);
-    uint4* dst = reinterpret_cast<uint4*>(tbuf + ((size_t)slot * BM + r) * PM_SLAB);
-    dst[0] = o[0];
-    dst[1] = o[1];
+                    for (int k = 0; k < BK / 16; ++k) {
+                        umma_bf16(tmem_base, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
+                                  accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit(empty_bar(stage));
+                    if (++stage == SHRINK_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(tfull_bar);
+                acc_phase ^= 1u;
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            const int cnt = min(args.sg, ns - g * args.sg);
+            ok = mbar_wait(tfull_bar, acc_phase, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            for (int i = 0; i < cnt; ++i) {
+                const int slot = tile * args.slab_cap + g * args.sg + i;
+                uint32_t v[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(i * PM_SLAB), v);
+                tmem_ld_wait();
+                const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
+                const float sc = on ? args.tile_scale[slot] : 0.f;
+                uint4 o[2];
+                uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+                for (int j = 0; j < PM_SLAB; j += 2)
+                    ow[j >> 1] = pack_bf16(__uint_as_float(v[j]) * sc, __uint_as_float(v[j + 1]) * sc);
+                uint4* dst = reinterpret_cast<uint4*>(args.tbuf + ((size_t)slot * BM + r) * PM_SLAB);
+                dst[0] = o[0];
+                dst[1] = o[1];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar);
+            acc_phase ^= 1u;
+        }
+    }
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, args.tmem_cols);
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -507,12 +623,25 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 }
 
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* /*tm_x*/, const bf16* x, int rows, bf16* tbuf) {
+                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf) {
     if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
+    ShrinkArgs a;
+    a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap;
+    a.sg = R.slab_cap < 16 ? R.slab_cap : 16;
+    uint32_t cols = 32;
+    while ((int)cols < a.sg * PM_SLAB) cols <<= 1;
+    a.tmem_cols = cols;
+    a.tile_nslabs = R.tile_nslabs; a.tile_slab = R.tile_slab; a.tile_scale = R.tile_scale;
+    a.tile_mask = R.tile_mask; a.tbuf = tbuf; a.status = L.status;
+    const int smem = SHRINK_STAGES * (SHRINK_X_BYTES + a.sg * SHRINK_A_SLAB_BYTES) + 256 + 1024;
+    static int smem_set = 0;
+    if (smem > smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(shrink_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        smem_set = smem;
+    }
     ProfScope ps(L, KC_SHRINK);
-    dim3 grid(R.n_tiles, R.slab_cap);
-    shrink_kernel<<<grid, 128, 0, L.st>>>(x, (const bf16*)lin.lora.At, rows, lin.k_in, R.tile_nslabs,
-                                          R.tile_slab, R.tile_scale, R.tile_mask, R.slab_cap, tbuf);
+    shrink_tc_kernel<<<R.n_tiles, GEMM_THREADS, smem, L.st>>>(*tm_x, lin.tm_at, a);
     BUMP(L);
     return cudaGetLastError();
 }
