@@ -307,6 +307,7 @@ struct pm_handle_s {
     // activations
     DevBuf X, U, QKV, ATT, H, PATCH, Z, t32, tbuf, status;
     CUtensorMap tm_patch, tm_u, tm_att, tm_h, tm_t;
+    CUtensorMap tm_y_qkv, tm_y_x, tm_y_h;      // outputs, for the TMA-store epilogue
     int tm_rows = -1;
     Router router;
     // adapters
@@ -375,7 +376,10 @@ int encode_activation_maps(pm_handle_s* h, int rows) {
     bool ok = tm_encode_2d(&h->tm_patch, h->PATCH.p, h->patch_dim, prow, (uint64_t)h->patch_dim * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_u, h->U.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_att, h->ATT.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
-           && tm_encode_2d(&h->tm_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 64, PM_TILE_M, 128);
+           && tm_encode_2d(&h->tm_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 64, PM_TILE_M, 128)
+           && tm_encode_2d(&h->tm_y_qkv, h->QKV.p, 3 * d, rows, (uint64_t)3 * d * 2, 32, 32, 64)
+           && tm_encode_2d(&h->tm_y_x, h->X.p, d, rows, (uint64_t)d * 2, 32, 32, 64)
+           && tm_encode_2d(&h->tm_y_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 32, 32, 64);
     if (!ok) { h->err = "cuTensorMapEncodeTiled failed (activations)"; return PM_ERR_CUDA; }
     h->tm_rows = rows;
     return PM_OK;
@@ -404,7 +408,10 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
                 cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>());
                 if (e != cudaSuccess) return e;
             }
-            return launch_lora_gemm(L, lo.dev, use_lora ? &R : nullptr, *tmx, &h->tm_t, nrows, epi,
+            const CUtensorMap* tmy = (void*)y == h->QKV.p ? &h->tm_y_qkv
+                                   : (void*)y == h->H.p ? &h->tm_y_h
+                                   : (void*)y == h->X.p ? &h->tm_y_x : nullptr;
+            return launch_lora_gemm(L, lo.dev, use_lora ? &R : nullptr, *tmx, &h->tm_t, tmy, nrows, epi,
                                     (const bf16*)residual, pep, (bf16*)y, h->n_sms);
         } else {
             return launch_naive_linear<T>(L, lo.dev, R, h->meta, h->slabs_max, x, nrows, tokens_pf,
@@ -763,9 +770,13 @@ int pm_linear_forward(pm_linear l, const void* x, int n_frames, const int32_t* s
         if (!tm_encode_2d(&tm_x, x, l->k_in, rows, (uint64_t)l->k_in * 2, 64, PM_TILE_M, 128)) {
             err = "cuTensorMapEncodeTiled failed (x); x must be 16-byte aligned"; return PM_ERR_CUDA;
         }
+        CUtensorMap tm_y;
+        if (!tm_encode_2d(&tm_y, y, l->n_out, rows, (uint64_t)l->n_out * 2, 32, 32, 64)) {
+            err = "cuTensorMapEncodeTiled failed (y); y must be 16-byte aligned"; return PM_ERR_CUDA;
+        }
         const bool lora = R.max_set > 0 && l->lin.dev.lora.At != nullptr;
         if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>()));
-        CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, rows, l->epilogue,
+        CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, &tm_y, rows, l->epilogue,
                             (const bf16*)residual, none, (bf16*)y, l->n_sms));
     } else {
         CK(launch_naive_linear<float>(L, l->lin.dev, R, l->meta, l->slabs_max, (const float*)x, rows, l->tokens,

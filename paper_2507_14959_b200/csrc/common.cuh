@@ -126,9 +126,12 @@ cudaError_t launch_naive_linear(const Launch& L, const LinearDev& lin, const Rou
 // tensor-core path (bf16): shrink into the slab buffer, then the fused GEMM
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
                           const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf);
+// tm_y: [rows, n_out] output map with a (32 x 32) box and 64B swizzle for the TMA-store epilogue, or
+// null to store straight from registers (always the case for EPI_PATCH, whose rows are remapped)
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
-                             const CUtensorMap& tm_x, const CUtensorMap* tm_t, int rows, int epi,
-                             const bf16* residual, const PatchEpi& pe, bf16* y, int n_sms);
+                             const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
+                             int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
+                             int n_sms);
 template <typename T>
 cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, int d, float eps,
                          const float* lnf_g, const float* lnf_b, float* z,

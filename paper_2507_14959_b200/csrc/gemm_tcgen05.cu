@@ -159,8 +159,13 @@ struct GemmArgs {
     const int* tile_nslabs;
     const int* tile_slab;
     int slab_cap;
+    int tma_store;             // 1: the epilogue stores through shared memory + TMA (tm_y valid)
     int* status;
 };
+
+constexpr int EPI_WARPS = 4;
+constexpr int STAGING_BYTES_PER_WARP = 2 * 32 * 64;     // two [32 rows x 32 bf16] buffers
+constexpr int PLAN_BYTES = 12288;
 
 template <int BN>
 struct Smem {
@@ -169,15 +174,30 @@ struct Smem {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int T_SLAB_BYTES = BM * PM_SLAB * 2;      // 4096
     static constexpr int B_SLAB_BYTES = BN * PM_SLAB * 2;
-    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int STAGING_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int PLAN_OFFSET = STAGING_OFFSET + EPI_WARPS * STAGING_BYTES_PER_WARP;
+    static constexpr int BAR_OFFSET = PLAN_OFFSET + PLAN_BYTES;
     static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;      // barriers + alignment slack
 };
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
 
 template <int BN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                  const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
-                 const GemmArgs args) {
+                 const __grid_constant__ CUtensorMap tm_y, const GemmArgs args) {
     using S = Smem<BN>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -191,14 +211,37 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     auto tempty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 2 + s); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + S::BAR_OFFSET + 8 * (2 * STAGES + 4));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::BAR_OFFSET + 8 * (2 * STAGES + 4) + 8);
+    int* plan = reinterpret_cast<int*>(smem + S::PLAN_OFFSET);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = args.m_tiles * args.n_tiles;
     const int num_kb = args.k_in / BK;
 
+    // The LoRA plan of this CTA's tiles (slab count + arena slab ids) is copied to shared memory
+    // once, so that the producer and the MMA issuer never wait on a global load between tiles.
+    const int plan_stride = 1 + args.slab_cap;
+    const int plan_tiles = args.tile_nslabs ? PLAN_BYTES / (4 * plan_stride) : 0;
+    if (args.tile_nslabs) {
+        for (int i = threadIdx.x / 8; i < plan_tiles; i += GEMM_THREADS / 8) {
+            const int tile = blockIdx.x + i * gridDim.x;
+            if (tile >= total_tiles) break;
+            const int m = tile / args.n_tiles;
+            const int ns = args.tile_nslabs[m];
+            if ((threadIdx.x & 7) == 0) plan[i * plan_stride] = ns;
+            for (int q = threadIdx.x & 7; q < ns; q += 8) plan[i * plan_stride + 1 + q] = args.tile_slab[m * args.slab_cap + q];
+        }
+    }
+    auto tile_ns = [&](int it, int m) -> int {
+        if (!args.tile_nslabs) return 0;
+        return it < plan_tiles ? plan[it * plan_stride] : args.tile_nslabs[m];
+    };
+    auto tile_slab_id = [&](int it, int m, int q) -> int {
+        return it < plan_tiles ? plan[it * plan_stride + 1 + q] : args.tile_slab[m * args.slab_cap + q];
+    };
+
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -218,7 +261,8 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            int it = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
                 const int m = tile / args.n_tiles, n = tile % args.n_tiles;
                 for (int kb = 0; kb < num_kb && ok; ++kb) {
                     ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
@@ -229,7 +273,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     tma_load_2d(sa + S::A_BYTES, &tm_w, kb * BK, n * BN, full_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                const int ns = args.tile_nslabs ? args.tile_nslabs[m] : 0;
+                const int ns = tile_ns(it, m);
                 for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
                     const int cnt = min(SLABS_PER_STAGE, ns - g0);
                     ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
@@ -238,7 +282,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     const uint32_t sa = base + stage * S::STAGE_BYTES;
                     for (int i = 0; i < cnt; ++i) {
                         const int slot = m * args.slab_cap + g0 + i;
-                        const int slab = args.tile_slab[slot];
+                        const int slab = tile_slab_id(it, m, g0 + i);
                         tma_load_2d(sa + i * S::T_SLAB_BYTES, &tm_t, 0, slot * BM, full_bar(stage));
                         tma_load_2d(sa + S::A_BYTES + i * S::B_SLAB_BYTES, &tm_bt, 0,
                                     slab * args.n_out + n * BN, full_bar(stage));
@@ -256,8 +300,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            int it = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
                 const int m = tile / args.n_tiles;
+                const int ns = tile_ns(it, m);
                 ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, args.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -278,7 +324,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     umma_commit(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                const int ns = args.tile_nslabs ? args.tile_nslabs[m] : 0;
                 for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
                     const int cnt = min(SLABS_PER_STAGE, ns - g0);
                     ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
@@ -301,8 +346,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+        const uint32_t staging = base + S::STAGING_OFFSET + (uint32_t)(warp - 2) * STAGING_BYTES_PER_WARP;
         int acc = 0;
         uint32_t acc_phase = 0;
+        uint32_t chunk_no = 0;                        // running chunk counter: picks the staging buffer
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int m = tile / args.n_tiles, n = tile % args.n_tiles;
@@ -320,27 +367,33 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                 pos_row = args.pe.pos + (size_t)(1 + p) * args.n_out;
             }
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+            const int n_chunks = min(BN / 32, (args.n_out - n * BN) / 32);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < n_chunks; ++c) {
                 const int n0 = n * BN + c * 32;
-                if (n0 >= args.n_out) break;           // uniform across the warp
                 uint32_t v[32];
                 tmem_ld32(t_row + (uint32_t)(c * 32), v);
                 tmem_ld_wait();
-                if (row_ok) {
-                    float f[32];
+                if (c == n_chunks - 1) {
+                    // every TMEM read of this accumulator is done: hand the buffer back early
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(acc));
+                }
+                float f[32];
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
-                        f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
-                        f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
-                        f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
-                        f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
-                    }
-                    if (args.epi == EPI_GELU) {
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
+                    f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
+                    f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
+                    f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
+                    f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+                }
+                if (args.epi == EPI_GELU) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
-                    } else if (args.epi == EPI_RESIDUAL) {
+                    for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
+                } else if (args.epi == EPI_RESIDUAL) {
+                    if (row_ok) {
                         const uint4* r4 = reinterpret_cast<const uint4*>(args.residual + (size_t)row * args.n_out + n0);
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
@@ -352,31 +405,49 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                                 f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
                             }
                         }
-                    } else if (args.epi == EPI_PATCH) {
+                    }
+                } else if (args.epi == EPI_PATCH) {
+                    if (row_ok) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             const float4 p4 = __ldg(reinterpret_cast<const float4*>(pos_row + n0 + j));
                             f[j + 0] += p4.x; f[j + 1] += p4.y; f[j + 2] += p4.z; f[j + 3] += p4.w;
                         }
                     }
+                }
+                uint4 o[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    o[q].x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
+                    o[q].y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
+                    o[q].z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
+                    o[q].w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
+                }
+                if (args.tma_store) {
+                    // [32 rows x 64 B] block, 16-byte chunks XOR-swizzled by (row >> 1) & 3 (64B
+                    // swizzle), then one TMA store; rows past the end are clipped by the tensor map
+                    const uint32_t buf = staging + (chunk_no & 1u) * (32 * 64);
+                    if (lane == 0) bulk_wait_read1();        // the store that last used this buffer has read it
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        st_shared_v4(buf + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4), o[q]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tm_y, buf, n0, m * BM + quarter * 32);
+                        bulk_commit();
+                    }
+                    ++chunk_no;
+                } else if (row_ok) {
                     uint4* o4 = reinterpret_cast<uint4*>(args.y + orow * args.n_out + n0);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 o;
-                        o.x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
-                        o.y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
-                        o.z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
-                        o.w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
-                        o4[q] = o;
-                    }
+                    for (int q = 0; q < 4; ++q) o4[q] = o[q];
                 }
             }
-            // all TMEM reads of this buffer are complete (wait::ld above): hand it back
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        if (args.tma_store && lane == 0) bulk_wait_all();
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -648,8 +719,8 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
 
 template <int BN>
 static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
-                                  const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const GemmArgs& a,
-                                  int n_sms) {
+                                  const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
+                                  const GemmArgs& a, int n_sms) {
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -660,7 +731,7 @@ static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, cons
     const int total = a.m_tiles * a.n_tiles;
     const int grid = total < n_sms ? total : n_sms;
     ProfScope ps(L, KC_GEMM);
-    lora_gemm_kernel<BN><<<grid, GEMM_THREADS, Smem<BN>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, a);
+    lora_gemm_kernel<BN><<<grid, GEMM_THREADS, Smem<BN>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, tm_y, a);
     BUMP(L);
     return cudaGetLastError();
 }
@@ -669,8 +740,9 @@ static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, cons
 int gemm_tile_n(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
 
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
-                             const CUtensorMap& tm_x, const CUtensorMap* tm_t, int rows, int epi,
-                             const bf16* residual, const PatchEpi& pe, bf16* y, int n_sms) {
+                             const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
+                             int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
+                             int n_sms) {
     if (rows <= 0) return cudaSuccess;
     const int bn = gemm_tile_n(lin.n_out);
     GemmArgs a;
@@ -683,8 +755,10 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
     a.tile_slab = lora ? R->tile_slab : nullptr;
     a.slab_cap = lora ? R->slab_cap : 0;
     a.status = L.status;
+    a.tma_store = (tm_y != nullptr && epi != EPI_PATCH) ? 1 : 0;
     const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced
     const CUtensorMap& tb = lora ? lin.tm_bt : lin.tm_w;
-    if (bn == 256) return launch_gemm_bn<256>(L, tm_x, lin.tm_w, tt, tb, a, n_sms);
-    return launch_gemm_bn<128>(L, tm_x, lin.tm_w, tt, tb, a, n_sms);
+    const CUtensorMap& ty = a.tma_store ? *tm_y : tm_x;
+    if (bn == 256) return launch_gemm_bn<256>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
+    return launch_gemm_bn<128>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
 }
