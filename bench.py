@@ -184,7 +184,7 @@ def main():
 
     import torch
     import workloads as wl
-    from paper_2507_14959_b200 import binding
+    from paper_2507_14959_b200 import binding, shard
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -266,10 +266,7 @@ def main():
     barrier()
     ms_e2e = f0.elapsed_time(f1)
 
-    t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = shard.max_over_ranks([ms, ms_e2e], device="cuda")
 
     if rank == 0:
         peaks = measured_peaks()
