@@ -141,6 +141,49 @@ int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, i
               const int32_t* prev_offsets, const int32_t* prev_ids,
               int32_t* next_offsets, int32_t* next_ids, int ids_capacity, void* cuda_stream);
 
+/* Selection for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a deployment variant of pm_select, same Algorithm 2 result.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a control loop with a
+ * no-allocation rule after start-up, a plug-in that lives inside another framework's memory pool,
+ * a process whose device memory has been handed out in full beforehand.  Such a caller cannot
+ * build a pm_handle (pm_create / pm_set_cover allocate), so this call takes everything as plain
+ * buffers and keeps its one piece of scratch -- the per-frame adapter bit masks between the two
+ * phases of the kernel -- in a fixed array inside the library image:
+ * PM_SELECT_STATIC_MAX_FRAMES x PM_SELECT_STATIC_MAX_ADAPTERS / 8 bytes = 128 KiB (plus a 256-byte
+ * status block), resident on every GPU that loads the library until the process exits.
+ * The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *   scores, prev_labels, prev_offsets, prev_ids, next_offsets, next_ids, ids_capacity,
+ *   score_thr, context_copy, has_prev: exactly as in pm_select (all buffers dev)
+ *   n_classes, n_adapters   sizes of the label space and of the adapter id range
+ *   first      dev int32 [n_classes]: for each class the first adapter, in Algorithm 2's visiting
+ *              order (fewest listed classes first, then lowest id), that lists it with accuracy
+ *              >= tau; -1 if none
+ *   provider   dev uint64 [n_classes, ceil(n_adapters/64)]: bit a of row k set iff adapter a lists
+ *              class k with accuracy >= tau (the tables pm_set_cover builds inside a handle)
+ *   status_out dev int32 or NULL: cleared by the call, then PM_ERR_CAPACITY is stored if the id list
+ *              did not fit in ids_capacity (the lists are truncated).  With NULL the condition is
+ *              not reported.
+ * Errors: PM_ERR_ARG (NULL / non-positive sizes), PM_ERR_CAPACITY (n_frames >
+ * PM_SELECT_STATIC_MAX_FRAMES or n_adapters > PM_SELECT_STATIC_MAX_ADAPTERS; nothing is launched),
+ * PM_ERR_CUDA.
+ * Set-up: the first call on each device looks up the device address of the array (with that
+ * device current -- make the stream's device current before calling).  Make that first call
+ * before starting any stream capture.
+ * Sharing: all calls on a device use the same array and it keeps the previous call's contents.
+ * Nothing in it needs to start at zero (every word a call reads it has written first), but two
+ * calls whose kernels may overlap on the GPU -- different streams, no ordering -- race on it:
+ * serialise them. */
+#define PM_SELECT_STATIC_MAX_FRAMES 4096
+#define PM_SELECT_STATIC_MAX_ADAPTERS 256
+int pm_select_static(const float* scores, int n_frames, int n_classes, int n_adapters,
+                     float score_thr, int context_copy, int has_prev, uint32_t* prev_labels,
+                     const int32_t* prev_offsets, const int32_t* prev_ids,
+                     const int32_t* first, const uint64_t* provider,
+                     int32_t* next_offsets, int32_t* next_ids, int ids_capacity,
+                     int32_t* status_out, void* cuda_stream);
+
 /* Synchronises the stream and returns the device status word (PM_OK or the first recorded
  * error), then clears it. */
 int pm_status(pm_handle h, void* cuda_stream);

@@ -21,7 +21,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
 
 EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_select",
-    "pm_status", "pm_last_error", "pm_launch_count", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
+    "pm_select_static", "pm_status", "pm_last_error", "pm_launch_count", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention",
 ]
@@ -76,6 +76,7 @@ def load():
     lib.pm_destroy.restype = None
     lib.pm_forward.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
     lib.pm_select.argtypes = [vp, vp, ip, C.c_float, ip, ip, vp, vp, vp, vp, vp, ip, vp]
+    lib.pm_select_static.argtypes = [vp, ip, ip, ip, C.c_float, ip, ip, vp, vp, vp, vp, vp, vp, vp, ip, vp, vp]
     lib.pm_status.argtypes = [vp, vp]
     lib.pm_last_error.argtypes = [vp]
     lib.pm_last_error.restype = C.c_char_p
@@ -266,6 +267,19 @@ def attention(qkv, out, n_frames, tokens, heads, dtype, stream=None):
     rc = load().pm_attention(_ptr(qkv), _ptr(out), n_frames, tokens, heads, dtype, _stream_ptr(stream))
     if rc != PM_OK:
         raise PolymorphError(rc, "pm_attention")
+
+
+def select_static(scores, n_adapters, score_thr, context_copy, has_prev, prev_labels, prev_offsets, prev_ids,
+                  first, provider, next_offsets, next_ids, status_out=None, stream=None):
+    """pm_select_static: Algorithm 2 with caller-provided cover tables and no device allocation."""
+    n, k = int(scores.shape[0]), int(scores.shape[1])
+    cap = 0 if next_ids is None else int(next_ids.numel())
+    rc = load().pm_select_static(_ptr(scores), n, k, int(n_adapters), score_thr, int(context_copy), int(has_prev),
+                                 _ptr(prev_labels), _ptr(prev_offsets), _ptr(prev_ids), _ptr(first),
+                                 _ptr(provider), _ptr(next_offsets), _ptr(next_ids), cap, _ptr(status_out),
+                                 _stream_ptr(stream))
+    if rc != PM_OK:
+        raise PolymorphError(rc, "pm_select_static")
 
 
 def model_from_workload(w, *, dtype=0, max_frames=None, max_set=None):

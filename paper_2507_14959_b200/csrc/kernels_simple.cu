@@ -582,3 +582,65 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
     BUMP(L);
     return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------------------
+// pm_select_static: Algorithm 2 selection for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------
+// select_kernel needs one scratch word list per frame (the chosen adapter bit masks, written in its
+// first phase and read back after the prefix sum).  pm_select takes that scratch from the handle,
+// which allocates it; this variant keeps it in the library image instead, so a caller that is
+// forbidden to call cudaMalloc (a real-time loop with a no-allocation rule, a plugin running
+// inside another framework's memory pool, a process whose device memory is fully pre-assigned)
+// can still run the selection.  Every GPU that loads the library carries the array until exit.
+#define PM_SELECT_STATIC_WORDS (PM_SELECT_STATIC_MAX_FRAMES * (PM_SELECT_STATIC_MAX_ADAPTERS / 64))
+
+static __device__ __align__(256) unsigned long long pm_select_static_masks[PM_SELECT_STATIC_WORDS];
+static __device__ __align__(256) int pm_select_static_status[64];   // word 0: status when the caller passes none
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+struct StaticScratch { uint64_t* masks; int* status; };
+StaticScratch g_static_scratch[STATIC_MAX_DEVICES];       // device addresses, per device ordinal
+bool g_static_ready[STATIC_MAX_DEVICES];
+}  // namespace
+
+extern "C" int pm_select_static(const float* scores, int n_frames, int n_classes, int n_adapters,
+                                float score_thr, int context_copy, int has_prev, uint32_t* prev_labels,
+                                const int32_t* prev_offsets, const int32_t* prev_ids,
+                                const int32_t* first, const uint64_t* provider,
+                                int32_t* next_offsets, int32_t* next_ids, int ids_capacity,
+                                int32_t* status_out, void* cuda_stream) {
+    if (n_frames < 0 || n_classes <= 0 || n_adapters <= 0 || !scores || !first || !provider ||
+        !next_offsets || ids_capacity < 0 || (!next_ids && ids_capacity > 0))
+        return PM_ERR_ARG;
+    if (has_prev && (!prev_labels || !prev_offsets || !prev_ids)) return PM_ERR_ARG;
+    if (n_frames > PM_SELECT_STATIC_MAX_FRAMES || n_adapters > PM_SELECT_STATIC_MAX_ADAPTERS)
+        return PM_ERR_CAPACITY;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return PM_ERR_CUDA;
+    if (!g_static_ready[dev]) {
+        // The array's name is only a host-side stand-in here: ask the runtime for the device address
+        // of this device's copy (the current device is the one the stream belongs to).
+        void *m = nullptr, *s = nullptr;
+        if (cudaGetSymbolAddress(&m, pm_select_static_masks) != cudaSuccess ||
+            cudaGetSymbolAddress(&s, pm_select_static_status) != cudaSuccess || !m || !s) {
+            cudaGetLastError();
+            return PM_ERR_CUDA;
+        }
+        g_static_scratch[dev].masks = static_cast<uint64_t*>(m);
+        g_static_scratch[dev].status = static_cast<int*>(s);
+        g_static_ready[dev] = true;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int* status = status_out ? status_out : g_static_scratch[dev].status;
+    // the status word is the only thing that must start at zero; the mask words are all rewritten
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return PM_ERR_CUDA;
+    Launch L;
+    L.st = st;
+    L.status = status;
+    if (launch_select(L, scores, n_frames, n_classes, n_adapters, score_thr, context_copy, has_prev,
+                      prev_labels, prev_offsets, prev_ids, first, provider, g_static_scratch[dev].masks,
+                      next_offsets, next_ids, ids_capacity) != cudaSuccess)
+        return PM_ERR_CUDA;
+    return PM_OK;
+}
