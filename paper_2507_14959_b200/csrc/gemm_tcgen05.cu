@@ -9,7 +9,8 @@
 // GEMM and fetched by TMA like any other operand.  Operands are staged by TMA into 128B- (base)
 // and 32B- (LoRA slab) swizzled shared memory; a single thread issues tcgen05.mma; accumulators
 // live in TMEM (two buffers, so the epilogue of one tile overlaps the main loop of the next).
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue.
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..9 = epilogue (two
+// warps per TMEM lane quarter, each taking half of the tile's columns).
 // Every mbarrier wait is bounded: on expiry the CTA raises an abort flag, records
 // PM_ERR_TIMEOUT in the status word, drains and returns.
 #include "common.cuh"
@@ -21,7 +22,7 @@ namespace {
 constexpr int BM = PM_TILE_M;
 constexpr int BK = 64;
 constexpr int STAGES = 4;
-constexpr int GEMM_THREADS = 192;
+constexpr int SHRINK_THREADS = 192;
 constexpr int SLABS_PER_STAGE = 4;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;     // ~2 s
 
@@ -141,8 +142,24 @@ __device__ __forceinline__ uint32_t instr_desc(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
+// Exact-erf GELU x * Phi(x) through the rational approximation of Abramowitz & Stegun 7.1.28,
+//   erfc(z) = (1 + a1 z + ... + a6 z^6)^-16 + eps, |eps| <= 3e-7   (z >= 0),
+// with 2^(1/16) folded into the coefficients so that the reciprocal is erfc(z)/2 = Phi(-|x|):
+//   gelu(x) = max(x, 0) - |x| * Phi(-|x|).
+// 12 FP32 operations and one reciprocal per element; absolute error below 1e-6 for finite x.
 __device__ __forceinline__ float gelu_erf(float v) {
-    return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f));
+    const float z = fabsf(v) * 0.70710678118654752440f;
+    float p = 4.4970397e-05f;
+    p = fmaf(p, z, 2.8881188e-04f);
+    p = fmaf(p, z, 1.5874455e-04f);
+    p = fmaf(p, z, 9.6809685e-03f);
+    p = fmaf(p, z, 4.4153997e-02f);
+    p = fmaf(p, z, 7.3645402e-02f);
+    p = fmaf(p, z, 1.0442738f);
+    p *= p; p *= p; p *= p; p *= p;
+    float h;                                      // p = +inf (|x| > ~25) gives 0
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(h) : "f"(p));
+    return fmaf(-fabsf(v), h, fmaxf(v, 0.f));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -163,11 +180,11 @@ struct GemmArgs {
     int* status;
 };
 
-constexpr int EPI_WARPS = 4;
 constexpr int STAGING_BYTES_PER_WARP = 2 * 32 * 64;     // two [32 rows x 32 bf16] buffers
-constexpr int PLAN_BYTES = 12288;
+constexpr int PLAN_BYTES = 2048;
 
-template <int BN>
+// EW = number of epilogue warps (4 or 8); the CTA has 2 + EW warps.
+template <int BN, int EW>
 struct Smem {
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
@@ -175,9 +192,9 @@ struct Smem {
     static constexpr int T_SLAB_BYTES = BM * PM_SLAB * 2;      // 4096
     static constexpr int B_SLAB_BYTES = BN * PM_SLAB * 2;
     static constexpr int STAGING_OFFSET = STAGES * STAGE_BYTES;
-    static constexpr int PLAN_OFFSET = STAGING_OFFSET + EPI_WARPS * STAGING_BYTES_PER_WARP;
+    static constexpr int PLAN_OFFSET = STAGING_OFFSET + EW * STAGING_BYTES_PER_WARP;
     static constexpr int BAR_OFFSET = PLAN_OFFSET + PLAN_BYTES;
-    static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;      // barriers + alignment slack
+    static constexpr int TOTAL = BAR_OFFSET + 256;             // + barriers (base must be 1024-aligned)
 };
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
@@ -193,16 +210,22 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
                  : "memory");
 }
 
-template <int BN>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+template <int BN, int EPI, int EW>
+__global__ void __launch_bounds__(64 + 32 * EW, 1)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                  const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
                  const __grid_constant__ CUtensorMap tm_y, const GemmArgs args) {
-    using S = Smem<BN>;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t* smem = smem_raw + (base - raw);
+    using S = Smem<BN, EW>;
+    constexpr int NTHREADS = 64 + 32 * EW;
+    constexpr int HALVES = EW / 4;                // epilogue warps per TMEM lane quarter
+    constexpr int CPW = BN / 32 / HALVES;         // 32-column chunks per epilogue warp
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if (base & 1023u) {                       // swizzled operands need a 1024-byte aligned window
+        if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
+        return;
+    }
+    uint8_t* smem = smem_raw;
     const uint32_t bars = base + S::BAR_OFFSET;
     // barrier words: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
     auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -222,7 +245,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     const int plan_stride = 1 + args.slab_cap;
     const int plan_tiles = args.tile_nslabs ? PLAN_BYTES / (4 * plan_stride) : 0;
     if (args.tile_nslabs) {
-        for (int i = threadIdx.x / 8; i < plan_tiles; i += GEMM_THREADS / 8) {
+        for (int i = threadIdx.x / 8; i < plan_tiles; i += NTHREADS / 8) {
             const int tile = blockIdx.x + i * gridDim.x;
             if (tile >= total_tiles) break;
             const int m = tile / args.n_tiles;
@@ -241,7 +264,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EW); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -344,8 +367,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2..)
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+        const int half = (warp - 2) >> 2;             // which share of the tile's 32-column chunks
         const uint32_t staging = base + S::STAGING_OFFSET + (uint32_t)(warp - 2) * STAGING_BYTES_PER_WARP;
         int acc = 0;
         uint32_t acc_phase = 0;
@@ -353,28 +377,50 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int m = tile / args.n_tiles, n = tile % args.n_tiles;
+            const int row = m * BM + quarter * 32 + lane;
+            const bool row_ok = row < args.rows;
+            const int n_chunks = min(BN / 32, (args.n_out - n * BN) / 32);      // even: n_out % 64 == 0
+            const int my_chunks = n_chunks / HALVES;
+            const int c0 = half * my_chunks;
+            // The residual rows of this warp's chunks are fetched before the accumulator is ready, so
+            // their latency hides behind the main loop.  (In-place use, y == residual, is safe: the
+            // same thread reads an element here and is the only one to overwrite it below.)
+            uint4 rr[EPI == EPI_RESIDUAL ? CPW : 1][4];
+            if constexpr (EPI == EPI_RESIDUAL) {
+#pragma unroll
+                for (int cc = 0; cc < CPW; ++cc) {
+                    if (cc < my_chunks && row_ok) {
+                        const uint4* r4 = reinterpret_cast<const uint4*>(
+                            args.residual + (size_t)row * args.n_out + n * BN + (c0 + cc) * 32);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) rr[cc][q] = r4[q];
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) rr[cc][q] = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
             ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, args.status);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int row = m * BM + quarter * 32 + lane;
-            const bool row_ok = row < args.rows;
             size_t orow = (size_t)row;
             const float* pos_row = nullptr;
-            if (args.epi == EPI_PATCH && row_ok) {
+            if (EPI == EPI_PATCH && row_ok) {
                 const int p = row % args.pe.g2;
                 orow = (size_t)(row / args.pe.g2) * args.pe.tokens + 1 + p;
                 pos_row = args.pe.pos + (size_t)(1 + p) * args.n_out;
             }
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-            const int n_chunks = min(BN / 32, (args.n_out - n * BN) / 32);
-#pragma unroll 1
-            for (int c = 0; c < n_chunks; ++c) {
+#pragma unroll
+            for (int cc = 0; cc < CPW; ++cc) {
+                if (cc >= my_chunks) break;
+                const int c = c0 + cc;
                 const int n0 = n * BN + c * 32;
                 uint32_t v[32];
                 tmem_ld32(t_row + (uint32_t)(c * 32), v);
                 tmem_ld_wait();
-                if (c == n_chunks - 1) {
+                if (cc == my_chunks - 1) {
                     // every TMEM read of this accumulator is done: hand the buffer back early
                     tc_fence_before();
                     __syncwarp();
@@ -389,24 +435,20 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
                     f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
                 }
-                if (args.epi == EPI_GELU) {
+                if constexpr (EPI == EPI_GELU) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
-                } else if (args.epi == EPI_RESIDUAL) {
-                    if (row_ok) {
-                        const uint4* r4 = reinterpret_cast<const uint4*>(args.residual + (size_t)row * args.n_out + n0);
+                } else if constexpr (EPI == EPI_RESIDUAL) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const uint4 r = r4[q];
-                            const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t w[4] = {rr[cc][q].x, rr[cc][q].y, rr[cc][q].z, rr[cc][q].w};
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
-                                f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
-                            }
+                        for (int e = 0; e < 4; ++e) {
+                            f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
+                            f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
                         }
                     }
-                } else if (args.epi == EPI_PATCH) {
+                } else if constexpr (EPI == EPI_PATCH) {
                     if (row_ok) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
@@ -499,7 +541,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
         : "memory");
 }
 
-__global__ void __launch_bounds__(GEMM_THREADS)
+__global__ void __launch_bounds__(SHRINK_THREADS)
 shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_at,
                  const ShrinkArgs args) {
     const int tile = blockIdx.x;
@@ -712,28 +754,46 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
         smem_set = smem;
     }
     ProfScope ps(L, KC_SHRINK);
-    shrink_tc_kernel<<<R.n_tiles, GEMM_THREADS, smem, L.st>>>(*tm_x, lin.tm_at, a);
+    shrink_tc_kernel<<<R.n_tiles, SHRINK_THREADS, smem, L.st>>>(*tm_x, lin.tm_at, a);
     BUMP(L);
     return cudaGetLastError();
 }
 
-template <int BN>
+#ifndef PM_GEMM_EPI_WARPS
+#define PM_GEMM_EPI_WARPS 8
+#endif
+constexpr int GEMM_EPI_WARPS = PM_GEMM_EPI_WARPS;      // 4 or 8
+
+template <int BN, int EPI>
 static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
                                   const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                   const GemmArgs& a, int n_sms) {
+    constexpr int EW = GEMM_EPI_WARPS;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Smem<BN>::TOTAL);
+        cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN, EPI, EW>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, EW>::TOTAL);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     const int total = a.m_tiles * a.n_tiles;
     const int grid = total < n_sms ? total : n_sms;
     ProfScope ps(L, KC_GEMM);
-    lora_gemm_kernel<BN><<<grid, GEMM_THREADS, Smem<BN>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, tm_y, a);
+    lora_gemm_kernel<BN, EPI, EW><<<grid, 64 + 32 * EW, Smem<BN, EW>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, tm_y, a);
     BUMP(L);
     return cudaGetLastError();
+}
+
+template <int BN>
+static cudaError_t launch_gemm_epi(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
+                                   const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
+                                   const GemmArgs& a, int n_sms) {
+    switch (a.epi) {
+        case EPI_GELU: return launch_gemm_bn<BN, EPI_GELU>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        case EPI_RESIDUAL: return launch_gemm_bn<BN, EPI_RESIDUAL>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        case EPI_PATCH: return launch_gemm_bn<BN, EPI_PATCH>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        default: return launch_gemm_bn<BN, EPI_NONE>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+    }
 }
 
 // lin.tm_w / lin.tm_bt are encoded for the BN chosen by gemm_tile_n(lin.n_out).
@@ -759,6 +819,6 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
     const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced
     const CUtensorMap& tb = lora ? lin.tm_bt : lin.tm_w;
     const CUtensorMap& ty = a.tma_store ? *tm_y : tm_x;
-    if (bn == 256) return launch_gemm_bn<256>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
-    return launch_gemm_bn<128>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
+    if (bn == 256) return launch_gemm_epi<256>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
+    return launch_gemm_epi<128>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
 }

@@ -132,6 +132,28 @@ def test_lora_linear(dtype, case):
     lin.close()
 
 
+def test_gelu_epilogue_accuracy():
+    """The GELU epilogue against the exact-erf definition: y = gelu(4 x) through an identity-like
+    weight, x sweeping [-3, 3] (so the argument spans [-12, 12]); the bf16 result must be within one
+    bf16 step of the exact value."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    n, rows = 64, 197 * 3
+    w = 4.0 * np.eye(n, dtype=np.float32)
+    x = wl.round_bf16(np.linspace(-3.0, 3.0, rows * n, dtype=np.float32).reshape(rows, n))
+    lin = binding.Linear(w, np.zeros(n, np.float32), max_adapters=1, max_rank=16, max_set=1, max_frames=3,
+                         tokens=197, epilogue=1, dtype=0)
+    xd = to_dev(x, 0)
+    yd = torch.full((rows, n), float("nan"), device="cuda", dtype=torch.bfloat16)
+    lin.forward(xd, 3, np.zeros(4, np.int32), np.zeros(0, np.int32), yd)
+    assert lin.status() == 0
+    want = po.gelu(4.0 * x.astype(np.float64))
+    got = to_np(yd)
+    step = np.maximum(np.abs(want), 2.0 ** -20) * 2.0 ** -8          # one bf16 step at |want|
+    assert np.all(np.abs(got - want) <= step + 2e-6)
+    lin.close()
+
+
 def test_linear_argument_errors():
     import torch
     from paper_2507_14959_b200 import binding
