@@ -308,6 +308,7 @@ struct pm_handle_s {
     DevBuf X, U, QKV, ATT, H, PATCH, Z, t32, tbuf, status;
     CUtensorMap tm_patch, tm_u, tm_att, tm_h, tm_t;
     CUtensorMap tm_y_qkv, tm_y_x, tm_y_h;      // outputs, for the TMA-store epilogue
+    CUtensorMap tm_att_q, tm_att_kv;           // attention operands over QKV
     int tm_rows = -1;
     Router router;
     // adapters
@@ -379,7 +380,9 @@ int encode_activation_maps(pm_handle_s* h, int rows) {
            && tm_encode_2d(&h->tm_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_y_qkv, h->QKV.p, 3 * d, rows, (uint64_t)3 * d * 2, 32, 32, 64)
            && tm_encode_2d(&h->tm_y_x, h->X.p, d, rows, (uint64_t)d * 2, 32, 32, 64)
-           && tm_encode_2d(&h->tm_y_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 32, 32, 64);
+           && tm_encode_2d(&h->tm_y_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 32, 32, 64)
+           && attention_encode_maps(h->QKV.as<bf16>(), rows / h->tokens, h->tokens, h->cfg.heads, &h->tm_att_q,
+                                    &h->tm_att_kv);
     if (!ok) { h->err = "cuTensorMapEncodeTiled failed (activations)"; return PM_ERR_CUDA; }
     h->tm_rows = rows;
     return PM_OK;
@@ -425,7 +428,12 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     for (int l = 0; l < c.layers; ++l) {
         CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
         CK(linear(h->lin[l * 4 + 0], U, &h->tm_u, rows, T_, true, EPI_NONE, nullptr, none, QKV));
-        if constexpr (TC) CK(launch_attention_mma(L, (const bf16*)QKV, (bf16*)ATT, n_frames, T_, c.heads));
+        if constexpr (TC) {
+            if (attention_tc_supported(T_))
+                CK(launch_attention_tc(L, h->tm_att_q, h->tm_att_kv, (bf16*)ATT, n_frames, T_, c.heads));
+            else
+                CK(launch_attention_mma(L, (const bf16*)QKV, (bf16*)ATT, n_frames, T_, c.heads));
+        }
         else CK(launch_attention_simple<T>(L, QKV, ATT, n_frames, T_, c.heads));
         CK(linear(h->lin[l * 4 + 1], ATT, &h->tm_att, rows, T_, true, EPI_RESIDUAL, X, none, X));
         CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
@@ -811,8 +819,25 @@ int pm_attention(const void* qkv, void* out, int n_frames, int tokens, int heads
     if (!qkv || !out || n_frames < 0 || tokens <= 0 || heads <= 0 || (dtype != 0 && dtype != 1))
         return PM_ERR_ARG;
     Launch L; L.st = (cudaStream_t)cuda_stream;
-    cudaError_t e = dtype == 0 ? launch_attention_mma(L, (const bf16*)qkv, (bf16*)out, n_frames, tokens, heads)
-                               : launch_attention_simple<float>(L, (const float*)qkv, (float*)out, n_frames, tokens, heads);
+    if (n_frames == 0) return PM_OK;
+    cudaError_t e;
+    if (dtype == 1) {
+        e = launch_attention_simple<float>(L, (const float*)qkv, (float*)out, n_frames, tokens, heads);
+    } else if (attention_tc_supported(tokens)) {
+        // the operator has no handle, hence no status word of its own: a bounded wait that expires is
+        // reported through the return code of a later call on the same device
+        static int* status_word = nullptr;
+        if (!status_word) {
+            if (cudaMalloc(&status_word, sizeof(int)) != cudaSuccess) return PM_ERR_OOM;
+            if (cudaMemset(status_word, 0, sizeof(int)) != cudaSuccess) return PM_ERR_CUDA;
+        }
+        L.status = status_word;
+        CUtensorMap tm_q, tm_kv;
+        if (!attention_encode_maps((const bf16*)qkv, n_frames, tokens, heads, &tm_q, &tm_kv)) return PM_ERR_CUDA;
+        e = launch_attention_tc(L, tm_q, tm_kv, (bf16*)out, n_frames, tokens, heads);
+    } else {
+        e = launch_attention_mma(L, (const bf16*)qkv, (bf16*)out, n_frames, tokens, heads);
+    }
     return e == cudaSuccess ? PM_OK : PM_ERR_CUDA;
 }
 

@@ -1,5 +1,9 @@
 // Attention of the bf16 build: softmax(q k^T / 8) v per (frame, head), head dim 64.
 //
+// Two kernels.  attention_tc_kernel (below, used up to 624 tokens) runs both contractions on the
+// tcgen05 tensor cores with the scores in tensor memory; attention_mma_kernel is the register-level
+// version kept for longer sequences:
+//
 // One CTA owns one (frame, head) (or a slice of its query rows when there are more than 256):
 // K and V of the head are staged once in shared memory (16-byte chunks XOR-swizzled by row so
 // that ldmatrix is conflict-free), each warp owns 16 query rows and walks the keys in blocks of
@@ -7,6 +11,7 @@
 // (mma.sync m16n8k16, bf16 in, fp32 accumulate).  Key blocks are trimmed to the 8-key tile, so
 // 197 tokens cost 200 key columns, not 256.
 #include "common.cuh"
+#include "tcgen05_ptx.cuh"
 
 #define BUMP(L) do { if ((L).launches) ++*(L).launches; } while (0)
 
@@ -168,8 +173,297 @@ __global__ void __launch_bounds__(512) attention_mma_kernel(const bf16* __restri
         if (r_hi < tokens) *reinterpret_cast<uint32_t*>(obase + (size_t)r_hi * d + c) = pack2(o[i][2] * inv_hi, o[i][3] * inv_hi);
     }
 }
+// ---------------------------------------------------------------------------------------
+// tcgen05 attention.  One CTA per (frame, head); K and V of the head are brought in once by TMA
+// (128B swizzle), the query rows are taken 128 at a time:
+//     S = Q K^T            UMMA 128 x nb x 16, four K steps, fp32 scores in tensor memory
+//     P = exp2(c (S - m))  four warps, one score row per thread (tcgen05.ld), written back over S
+//                          as packed bf16 (tcgen05.st), row sums kept in registers
+//     O = P V              UMMA 128 x 64 x 16 with the A operand read from tensor memory and V as
+//                          an MN-major shared-memory operand, one K step per 16 keys
+//     out = O / rowsum     tcgen05.ld, bf16, straight to global memory
+// Keys come in blocks of up to 208 (13 x 16).  With one block (up to 208 tokens) the row maximum
+// comes from the same scores.  With several blocks the scores are formed twice: a first sweep
+// yields each row's maximum over all keys, the second forms P against that final maximum and
+// accumulates O over the blocks, so no rescaling of O is ever needed.
+// The issuing thread and the softmax warps alternate through two mbarriers (scores / O ready,
+// rows done); two CTAs per SM overlap one head's softmax with another's loads and MMAs.
+// ---------------------------------------------------------------------------------------
+constexpr int AQ = 128;                    // query rows per tile
+constexpr int AKB = 208;                   // keys per score block
+constexpr int ATT_THREADS = 160;           // warp 0: TMEM owner, TMA + MMA issue; warps 1..4: softmax
+constexpr int AQ_BYTES = AQ * 128;
+constexpr int AKB_BYTES = AKB * 128;
+constexpr int ATT_MAX_BLOCKS = 3;
+
+struct AttnArgs {
+    int tokens, heads, tpad, n_blocks, n_qtiles;
+    uint32_t tmem_cols, o_col;
+    bf16* out;
+    int* status;
+};
+
+// maximum of the first `lim` of 32 score columns (all of them if lim >= 32)
+template <int N, bool MASK>
+__device__ __forceinline__ float chunk_max(const uint32_t* v, int lim, float m) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const float sj = __uint_as_float(v[j]);
+        m = fmaxf(m, (!MASK || j < lim) ? sj : -INFINITY);
+    }
+    return m;
+}
+// p_j = exp2(c s_j - mc) (0 beyond lim), packed to bf16 pairs; returns the sum of the p_j
+template <int N, bool MASK>
+__device__ __forceinline__ float chunk_probs(const uint32_t* v, int lim, float c, float mc, uint32_t* packed) {
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < N; j += 2) {
+        float p0 = exp2f(fmaf(__uint_as_float(v[j]), c, -mc));
+        float p1 = exp2f(fmaf(__uint_as_float(v[j + 1]), c, -mc));
+        if (MASK) { p0 = j < lim ? p0 : 0.f; p1 = j + 1 < lim ? p1 : 0.f; }
+        sum += p0 + p1;
+        packed[j >> 1] = pack2(p0, p1);
+    }
+    return sum;
+}
+
+__global__ void __launch_bounds__(ATT_THREADS)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
+                    const AttnArgs args) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if (base & 1023u) {                       // swizzled operands need a 1024-byte aligned window
+        if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
+        return;
+    }
+    const int f = blockIdx.x / args.heads, h = blockIdx.x % args.heads;
+    const int d = args.heads * HD;
+    const int T = args.tokens;
+    const int n_blocks = args.n_blocks;
+    const uint32_t q_s = base;
+    const uint32_t k_s = q_s + AQ_BYTES;
+    const uint32_t v_s = k_s + n_blocks * AKB_BYTES;
+    const uint32_t bars = v_s + n_blocks * AKB_BYTES;
+    const uint32_t kv_bar = bars, q_bar = bars + 8, s_bar = bars + 16, r_bar = bars + 24;
+    uint8_t* bar_ptr = smem_raw + (bars - base);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 40);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(kv_bar, 1); mbar_init(q_bar, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), args.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t o_tmem = tmem_base + args.o_col;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------ TMA + MMA issue
+            mbar_expect_tx(kv_bar, (uint32_t)(n_blocks * 2 * AKB_BYTES));
+            for (int b = 0; b < n_blocks; ++b) {
+                tma_load_2d(k_s + b * AKB_BYTES, &tm_kv, d + h * HD, f * T + b * AKB, kv_bar);
+                tma_load_2d(v_s + b * AKB_BYTES, &tm_kv, 2 * d + h * HD, f * T + b * AKB, kv_bar);
+            }
+            const uint32_t idesc_pv = instr_desc_b_mn(HD);
+            uint32_t step = 0;
+            bool ok = true;
+            for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
+                mbar_expect_tx(q_bar, AQ_BYTES);
+                tma_load_2d(q_s, &tm_q, h * HD, f * T + qt * AQ, q_bar);
+                if (qt == 0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
+                ok = ok && mbar_wait(q_bar, qt & 1, abort_flag, args.status);
+                if (!ok) break;
+                tc_fence_after();
+                for (int pass = (n_blocks > 1 ? 0 : 1); pass < 2 && ok; ++pass) {
+                    for (int b = 0; b < n_blocks && ok; ++b) {
+                        const int nb = min(AKB, args.tpad - b * AKB);
+                        const uint32_t idesc_s = instr_desc(nb);
+#pragma unroll
+                        for (int k = 0; k < HD / 16; ++k)
+                            umma_bf16(tmem_base, smem_desc(q_s + k * 32, 128),
+                                      smem_desc(k_s + b * AKB_BYTES + k * 32, 128), idesc_s, k > 0);
+                        umma_commit(s_bar);
+                        ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
+                        ++step;
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (pass == 1) {
+                            for (int kk = 0; kk < nb / 16; ++kk)
+                                umma_bf16_ts(o_tmem, tmem_base + (uint32_t)(kk * 8),
+                                             smem_desc(v_s + b * AKB_BYTES + kk * 2048, 128), idesc_pv,
+                                             (b > 0 || kk > 0) ? 1u : 0u);
+                            umma_commit(s_bar);
+                            ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
+                            ++step;
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                    }
+                }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------- softmax + output (warps 1..4)
+        const int quarter = warp & 3;                            // TMEM lanes 32*quarter .. +31
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const float c = 0.125f * 1.4426950408889634f;            // 1/sqrt(64) * log2(e)
+        uint32_t step = 0;
+        bool ok = true;
+        auto begin_step = [&]() {
+            ok = mbar_wait(s_bar, step & 1u, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (ok) tc_fence_after();
+            return ok;
+        };
+        auto end_step = [&]() {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(r_bar);
+            ++step;
+        };
+        // row maximum of one score block (columns at or beyond `valid` are ignored)
+        auto block_max = [&](int nb, int valid, float m) {
+            for (int c0 = 0; c0 < nb; c0 += 32) {
+                uint32_t v[32];
+                if (nb - c0 >= 32) {
+                    tmem_ld32(t_lane + (uint32_t)c0, v);
+                    tmem_ld_wait();
+                    m = (valid - c0 >= 32) ? chunk_max<32, false>(v, 32, m) : chunk_max<32, true>(v, valid - c0, m);
+                } else {
+                    tmem_ld16(t_lane + (uint32_t)c0, v);
+                    tmem_ld_wait();
+                    m = (valid - c0 >= 16) ? chunk_max<16, false>(v, 16, m) : chunk_max<16, true>(v, valid - c0, m);
+                }
+            }
+            return m;
+        };
+        for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
+            const int q_row = qt * AQ + quarter * 32 + lane;
+            const bool warp_active = qt * AQ + quarter * 32 < T;      // else: no row of this warp exists
+            float m = -INFINITY, l = 0.f;
+            if (n_blocks > 1) {
+                for (int b = 0; b < n_blocks; ++b) {
+                    if (!begin_step()) break;
+                    if (warp_active) m = block_max(min(AKB, args.tpad - b * AKB), T - b * AKB, m);
+                    end_step();
+                }
+                if (!ok) break;
+            }
+            for (int b = 0; b < n_blocks; ++b) {
+                const int nb = min(AKB, args.tpad - b * AKB), valid = T - b * AKB;
+                if (!begin_step()) break;
+                if (warp_active) {
+                    if (n_blocks == 1) m = block_max(nb, valid, m);
+                    const float mc = m * c;
+                    for (int c0 = 0; c0 < nb; c0 += 32) {
+                        uint32_t v[32], pk[16];
+                        if (nb - c0 >= 32) {
+                            tmem_ld32(t_lane + (uint32_t)c0, v);
+                            tmem_ld_wait();
+                            l += (valid - c0 >= 32) ? chunk_probs<32, false>(v, 32, c, mc, pk)
+                                                    : chunk_probs<32, true>(v, valid - c0, c, mc, pk);
+                            tmem_st16(t_lane + (uint32_t)(c0 >> 1), pk);
+                        } else {
+                            tmem_ld16(t_lane + (uint32_t)c0, v);
+                            tmem_ld_wait();
+                            l += (valid - c0 >= 16) ? chunk_probs<16, false>(v, 16, c, mc, pk)
+                                                    : chunk_probs<16, true>(v, valid - c0, c, mc, pk);
+                            tmem_st8(t_lane + (uint32_t)(c0 >> 1), pk);
+                        }
+                    }
+                    tmem_st_wait();
+                }
+                end_step();
+                // O (+)= P V_b is issued now; after the last block the finished rows are written out
+                if (!begin_step()) break;
+                if (b == n_blocks - 1 && warp_active) {
+                    const float inv = 1.f / l;
+                    bf16* orow = args.out + ((size_t)f * T + q_row) * d + h * HD;
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t v[32];
+                        tmem_ld32((t_lane + args.o_col) + (uint32_t)(half * 32), v);
+                        tmem_ld_wait();
+                        if (q_row < T) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                uint4 o;
+                                o.x = pack2(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
+                                o.y = pack2(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
+                                o.z = pack2(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
+                                o.w = pack2(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
+                                reinterpret_cast<uint4*>(orow + half * 32)[q] = o;
+                            }
+                        }
+                    }
+                }
+                end_step();
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);    // let copies / MMAs in flight land
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, args.tmem_cols);
+    }
+}
 
 }  // namespace
+
+bool attention_tc_supported(int tokens) { return (tokens + 15) / 16 * 16 <= ATT_MAX_BLOCKS * AKB; }
+
+bool attention_encode_maps(const bf16* qkv, int n_frames, int tokens, int heads, CUtensorMap* tm_q,
+                           CUtensorMap* tm_kv) {
+    const uint64_t w = (uint64_t)3 * heads * HD, rows = (uint64_t)n_frames * tokens;
+    return tm_encode_2d(tm_q, qkv, w, rows, w * 2, HD, AQ, 128) &&
+           tm_encode_2d(tm_kv, qkv, w, rows, w * 2, HD, AKB, 128);
+}
+
+cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const CUtensorMap& tm_kv,
+                                bf16* out, int n_frames, int tokens, int heads) {
+    if (n_frames <= 0) return cudaSuccess;
+    AttnArgs a;
+    a.tokens = tokens; a.heads = heads;
+    a.tpad = (tokens + 15) / 16 * 16;
+    a.n_blocks = (a.tpad + AKB - 1) / AKB;
+    a.n_qtiles = (tokens + AQ - 1) / AQ;
+    // one block: P (104 columns) replaces S (208) and O takes columns 128..191 of the same 256;
+    // several blocks: O must outlive the score blocks and sits in a second group of 256 columns
+    a.tmem_cols = a.n_blocks == 1 ? 256u : 512u;
+    a.o_col = a.n_blocks == 1 ? 128u : 256u;
+    a.out = out; a.status = L.status;
+    // at least 110 KB, so that no more than two CTAs (2 x 256 TMEM columns) share an SM
+    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
+    if (smem < 110 * 1024) smem = 110 * 1024;
+    static size_t smem_set = 0;
+    if (smem > smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        smem_set = smem;
+    }
+    ProfScope ps(L, KC_ATTENTION);
+    attention_tc_kernel<<<n_frames * heads, ATT_THREADS, smem, L.st>>>(tm_q, tm_kv, a);
+    BUMP(L);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_attention_mma(const Launch& L, const bf16* qkv, bf16* out, int n_frames, int tokens,
                                  int heads) {

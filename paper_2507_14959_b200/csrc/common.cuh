@@ -111,6 +111,12 @@ cudaError_t launch_attention_simple(const Launch& L, const T* qkv, T* out, int n
                                     int heads);
 cudaError_t launch_attention_mma(const Launch& L, const bf16* qkv, bf16* out, int n_frames,
                                  int tokens, int heads);
+// tcgen05 attention (bf16, up to 624 tokens): tensor maps over qkv [n_frames*tokens, 3*heads*64]
+bool attention_tc_supported(int tokens);
+bool attention_encode_maps(const bf16* qkv, int n_frames, int tokens, int heads, CUtensorMap* tm_q,
+                           CUtensorMap* tm_kv);
+cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const CUtensorMap& tm_kv,
+                                bf16* out, int n_frames, int tokens, int heads);
 template <typename T>
 cudaError_t launch_im2col(const Launch& L, const T* frames, const int* perm, T* out, int n_frames,
                           int img, int patch);
