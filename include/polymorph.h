@@ -150,8 +150,8 @@ int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, i
  * build a pm_handle (pm_create / pm_set_cover allocate), so this call takes everything as plain
  * buffers and keeps its one piece of scratch -- the per-frame adapter bit masks between the two
  * phases of the kernel -- in a fixed array inside the library image:
- * PM_SELECT_STATIC_MAX_FRAMES x PM_SELECT_STATIC_MAX_ADAPTERS / 8 bytes = 128 KiB (plus a 256-byte
- * status block), resident on every GPU that loads the library until the process exits.
+ * PM_SELECT_STATIC_MAX_FRAMES x PM_SELECT_STATIC_MAX_ADAPTERS / 8 bytes = 128 KiB (plus a counter
+ * word and a 256-byte status block), resident on every GPU that loads the library until the process exits.
  * The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *
  *   scores, prev_labels, prev_offsets, prev_ids, next_offsets, next_ids, ids_capacity,
@@ -172,9 +172,9 @@ int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, i
  * device current -- make the stream's device current before calling).  Make that first call
  * before starting any stream capture.
  * Sharing: all calls on a device use the same array and it keeps the previous call's contents.
- * Nothing in it needs to start at zero (every word a call reads it has written first), but two
- * calls whose kernels may overlap on the GPU -- different streams, no ordering -- race on it:
- * serialise them. */
+ * The call clears the two words that must start at zero (status, block counter) on the stream; every
+ * other word it reads it has written first.  Two calls whose kernels may overlap on the GPU --
+ * different streams, no ordering -- race on the array: serialise them. */
 #define PM_SELECT_STATIC_MAX_FRAMES 4096
 #define PM_SELECT_STATIC_MAX_ADAPTERS 256
 int pm_select_static(const float* scores, int n_frames, int n_classes, int n_adapters,

@@ -602,7 +602,9 @@ int pm_set_cover(pm_handle h, float tau) {
         }
     CK(h->first.alloc(first.size() * sizeof(int)));
     CK(h->provider.alloc(prov.size() * sizeof(uint64_t)));
-    CK(h->mask_scratch.alloc((size_t)h->cfg.max_frames * AW * sizeof(uint64_t)));
+    // per-frame adapter masks + the select kernel's block counter (zero between launches)
+    CK(h->mask_scratch.alloc(((size_t)h->cfg.max_frames * AW + 1) * sizeof(uint64_t)));
+    CK(cudaMemset(h->mask_scratch.p, 0, h->mask_scratch.bytes));
     CK(cudaMemcpy(h->first.p, first.data(), first.size() * sizeof(int), cudaMemcpyHostToDevice));
     CK(cudaMemcpy(h->provider.p, prov.data(), prov.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
     h->cover_ready = true;

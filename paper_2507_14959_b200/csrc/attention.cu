@@ -241,18 +241,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int d = args.heads * HD;
     const int T = args.tokens;
     const int n_blocks = args.n_blocks;
-    const uint32_t q_s = base;
-    const uint32_t k_s = q_s + AQ_BYTES;
+    const uint32_t q_s = base;                               // two query-tile buffers
+    const uint32_t k_s = q_s + 2 * AQ_BYTES;
     const uint32_t v_s = k_s + n_blocks * AKB_BYTES;
     const uint32_t bars = v_s + n_blocks * AKB_BYTES;
-    const uint32_t kv_bar = bars, q_bar = bars + 8, s_bar = bars + 16, r_bar = bars + 24;
+    const uint32_t kv_bar = bars, s_bar = bars + 8, r_bar = bars + 16, q_bar0 = bars + 24;   // q_bar0, q_bar0 + 8
     uint8_t* bar_ptr = smem_raw + (bars - base);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 32);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 40);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 40);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 48);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(kv_bar, 1); mbar_init(q_bar, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4);
+        mbar_init(kv_bar, 1); mbar_init(q_bar0, 1); mbar_init(q_bar0 + 8, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -278,20 +278,26 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const uint32_t idesc_pv = instr_desc_b_mn(HD);
             uint32_t step = 0;
             bool ok = true;
+            auto load_q = [&](int qt) {       // the buffer's previous tile (qt - 2) has been consumed
+                const uint32_t bar = q_bar0 + 8u * (qt & 1);
+                mbar_expect_tx(bar, AQ_BYTES);
+                tma_load_2d(q_s + (qt & 1) * AQ_BYTES, &tm_q, h * HD, f * T + qt * AQ, bar);
+            };
+            load_q(0);
             for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
-                mbar_expect_tx(q_bar, AQ_BYTES);
-                tma_load_2d(q_s, &tm_q, h * HD, f * T + qt * AQ, q_bar);
+                if (qt + 1 < args.n_qtiles) load_q(qt + 1);
                 if (qt == 0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
-                ok = ok && mbar_wait(q_bar, qt & 1, abort_flag, args.status);
+                ok = ok && mbar_wait(q_bar0 + 8u * (qt & 1), (qt >> 1) & 1, abort_flag, args.status);
                 if (!ok) break;
                 tc_fence_after();
+                const uint32_t q_cur = q_s + (qt & 1) * AQ_BYTES;
                 for (int pass = (n_blocks > 1 ? 0 : 1); pass < 2 && ok; ++pass) {
                     for (int b = 0; b < n_blocks && ok; ++b) {
                         const int nb = min(AKB, args.tpad - b * AKB);
                         const uint32_t idesc_s = instr_desc(nb);
 #pragma unroll
                         for (int k = 0; k < HD / 16; ++k)
-                            umma_bf16(tmem_base, smem_desc(q_s + k * 32, 128),
+                            umma_bf16(tmem_base, smem_desc(q_cur + k * 32, 128),
                                       smem_desc(k_s + b * AKB_BYTES + k * 32, 128), idesc_s, k > 0);
                         umma_commit(s_bar);
                         ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
@@ -451,7 +457,7 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
     a.o_col = a.n_blocks == 1 ? 128u : 256u;
     a.out = out; a.status = L.status;
     // at least 110 KB, so that no more than two CTAs (2 x 256 TMEM columns) share an SM
-    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
+    size_t smem = (size_t)2 * AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
     if (smem < 110 * 1024) smem = 110 * 1024;
     static size_t smem_set = 0;
     if (smem > smem_set) {

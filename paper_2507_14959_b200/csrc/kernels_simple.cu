@@ -396,17 +396,37 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ z, const T* _
 
 __device__ __forceinline__ float sigmoidf_acc(float v) { return 1.f / (1.f + expf(-v)); }
 
-// grid (ceil(K/8), F): warp = one class of one slot; base_out rows are in the caller's order
+// grid (ceil(K/8), ceil(F/32)): a warp keeps the weight row of one class in registers and walks 32
+// slots, so the weights are read once per 32 frames; base_out rows are in the caller's order
+constexpr int BASE_HEAD_FRAMES = 32;
 template <typename T>
 __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict__ z, const T* __restrict__ wt,
                                                         const float* __restrict__ bias,
                                                         const int* __restrict__ perm, int d, int n_classes,
-                                                        float* __restrict__ base_out) {
+                                                        int n_frames, float* __restrict__ base_out) {
     const int k = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int slot = blockIdx.y;
+    const int lane = threadIdx.x & 31;
     if (k >= n_classes) return;
-    const float v = dot_row<T>(z + (size_t)slot * d, wt + (size_t)k * d, d, threadIdx.x & 31) + bias[k];
-    if ((threadIdx.x & 31) == 0) base_out[(size_t)perm[slot] * n_classes + k] = sigmoidf_acc(v);
+    constexpr int MAXV = 32;                      // d <= 1024: at most 32 weights per lane
+    float w[MAXV];
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+        const int c = lane + 32 * i;
+        w[i] = c < d ? to_f(wt[(size_t)k * d + c]) : 0.f;
+    }
+    const float bk = bias[k];
+    const int s0 = blockIdx.y * BASE_HEAD_FRAMES, s1 = min(n_frames, s0 + BASE_HEAD_FRAMES);
+    for (int slot = s0; slot < s1; ++slot) {
+        const float* zr = z + (size_t)slot * d;
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < MAXV; ++i) {
+            const int c = lane + 32 * i;
+            if (c < d) acc = fmaf(zr[c], w[i], acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) base_out[(size_t)perm[slot] * n_classes + k] = sigmoidf_acc(acc + bk);
+    }
 }
 
 // grid (max_set, F): block = the p-th active adapter of one slot; its warps walk the adapter's
@@ -444,8 +464,8 @@ cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, 
     final_ln_kernel<T><<<(n_frames + 7) / 8, 256, 0, L.st>>>(x, lnf_g, lnf_b, z, n_frames, tokens, d, eps);
     BUMP(L);
     if (base_out) {
-        dim3 grid((n_classes + 7) / 8, n_frames);
-        base_head_kernel<T><<<grid, 256, 0, L.st>>>(z, base_wt, base_b, R.perm, d, n_classes, base_out);
+        dim3 grid((n_classes + 7) / 8, (n_frames + BASE_HEAD_FRAMES - 1) / BASE_HEAD_FRAMES);
+        base_head_kernel<T><<<grid, 256, 0, L.st>>>(z, base_wt, base_b, R.perm, d, n_classes, n_frames, base_out);
         BUMP(L);
     }
     cudaError_t e = cudaMemsetAsync(scores_out, 0, (size_t)n_frames * n_classes * sizeof(float), L.st);
@@ -462,12 +482,18 @@ template cudaError_t launch_heads<float>(const Launch&, const float*, int, int, 
 template cudaError_t launch_heads<bf16>(const Launch&, const bf16*, int, int, int, float, const float*, const float*, float*, const bf16*, const float*, int, const bf16*, const float*, const int*, const int*, const RouteDev&, float*, float*);
 
 // ---------------------------------------------------------------------------------------
-// Algorithm 2 on the device: one block, one warp per frame
+// Algorithm 2 on the device: one warp per frame, any number of blocks
 // ---------------------------------------------------------------------------------------
 // The greedy branch visits contexts by (size, id) and takes a context iff it provides a still
 // uncovered label; that set equals { first(l) : l in Y_t }, first(l) being the first provider of l
 // in visiting order, so it reduces to a table lookup and a bit-mask OR.
-__global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, int n_frames,
+// Phase 1 (all blocks): threshold -> label bit set -> keep / copy / greedy -> adapter bit mask and
+// its population count per frame.  Phase 2 (the block that finishes last, found with a counter in
+// the scratch area): prefix sum of the counts and emission of the sorted id lists.  `masks` holds
+// n_frames * ceil(n_adapters/64) words followed by one counter word that is zero between launches.
+constexpr int SELECT_THREADS = 256;
+
+__global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __restrict__ scores, int n_frames,
                                                       int n_classes, int n_adapters, float thr,
                                                       int context_copy, int has_prev,
                                                       uint32_t* __restrict__ prev_labels,
@@ -475,16 +501,19 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
                                                       const int* __restrict__ prev_ids,
                                                       const int* __restrict__ first,
                                                       const uint64_t* __restrict__ provider,
-                                                      uint64_t* __restrict__ masks,
-                                                      int* __restrict__ next_off,
+                                                      uint64_t* masks,
+                                                      int* next_off,
                                                       int* __restrict__ next_ids, int ids_capacity,
                                                       int* __restrict__ status) {
-    __shared__ int partial[1024];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    __shared__ int partial[SELECT_THREADS];
+    __shared__ int is_last;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = SELECT_THREADS >> 5;
     const int NW = (n_classes + 31) / 32;
     const int AW = (n_adapters + 63) / 64;     // <= 4 (checked on the host)
+    unsigned int* done = reinterpret_cast<unsigned int*>(masks + (size_t)n_frames * AW);
 
-    for (int f = warp; f < n_frames; f += nwarps) {
+    const int f = blockIdx.x * nwarps + warp;
+    if (f < n_frames) {
         uint64_t prev_mask[4] = {0, 0, 0, 0}, greedy[4] = {0, 0, 0, 0};
         if (has_prev) {
             for (int i = prev_off[f] + lane; i < prev_off[f + 1]; i += 32) {
@@ -498,21 +527,33 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
             }
         }
         bool same = true, covered = true;
-        for (int w = 0; w < NW; ++w) {
-            const int k = w * 32 + lane;
-            const bool on = (k < n_classes) && (scores[(size_t)f * n_classes + k] > thr);
-            const uint32_t word = __ballot_sync(0xFFFFFFFFu, on);
-            if (prev_labels) {
-                if (has_prev && prev_labels[(size_t)f * NW + w] != word) same = false;
-                __syncwarp();
-                if (lane == 0) prev_labels[(size_t)f * NW + w] = word;
+        for (int w0 = 0; w0 < NW; w0 += 8) {
+            float sc[8];
+            uint32_t old[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {               // eight independent loads in flight
+                const int k = (w0 + i) * 32 + lane;
+                sc[i] = (w0 + i < NW && k < n_classes) ? scores[(size_t)f * n_classes + k] : -INFINITY;
+                old[i] = (has_prev && prev_labels && w0 + i < NW && lane == 0) ? prev_labels[(size_t)f * NW + w0 + i] : 0u;
             }
-            if (on) {
-                bool cov = false;
-                for (int q = 0; q < AW; ++q) cov |= (provider[(size_t)k * AW + q] & prev_mask[q]) != 0;
-                if (!cov) covered = false;
-                const int a = first[k];
-                if (a >= 0) greedy[a >> 6] |= 1ull << (a & 63);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int w = w0 + i;
+                if (w >= NW) break;
+                const int k = w * 32 + lane;
+                const bool on = sc[i] > thr;
+                const uint32_t word = __ballot_sync(0xFFFFFFFFu, on);
+                if (prev_labels && lane == 0) {
+                    if (has_prev && old[i] != word) same = false;
+                    prev_labels[(size_t)f * NW + w] = word;
+                }
+                if (on) {
+                    bool cov = false;
+                    for (int q = 0; q < AW; ++q) cov |= (provider[(size_t)k * AW + q] & prev_mask[q]) != 0;
+                    if (!cov) covered = false;
+                    const int a = first[k];
+                    if (a >= 0) greedy[a >> 6] |= 1ull << (a & 63);
+                }
             }
         }
         covered = __all_sync(0xFFFFFFFFu, covered);
@@ -531,31 +572,39 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
         }
         if (lane == 0) next_off[f + 1] = cnt;
     }
+    // ---- the last block to arrive here does the scan and the emission
+    __threadfence();
     __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(done, 1u) == gridDim.x - 1) ? 1 : 0;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    volatile int* voff = next_off;
+    volatile uint64_t* vmasks = masks;
     // exclusive scan of the counts: each thread owns a contiguous chunk of frames
-    const int per = (n_frames + blockDim.x - 1) / blockDim.x;
+    const int per = (n_frames + SELECT_THREADS - 1) / SELECT_THREADS;
     const int lo = min(n_frames, (int)threadIdx.x * per), hi = min(n_frames, lo + per);
     int s = 0;
-    for (int f = lo; f < hi; ++f) s += next_off[f + 1];
+    for (int g = lo; g < hi; ++g) s += voff[g + 1];
     partial[threadIdx.x] = s;
     __syncthreads();
-    for (int o = 1; o < (int)blockDim.x; o <<= 1) {
+    for (int o = 1; o < SELECT_THREADS; o <<= 1) {
         const int v = (int)threadIdx.x >= o ? partial[threadIdx.x - o] : 0;
         __syncthreads();
         partial[threadIdx.x] += v;
         __syncthreads();
     }
     int run = partial[threadIdx.x] - s;        // exclusive prefix of this chunk
-    if (threadIdx.x == 0) next_off[0] = 0;
-    for (int f = lo; f < hi; ++f) {
-        run += next_off[f + 1];
-        next_off[f + 1] = run;
+    if (threadIdx.x == 0) { voff[0] = 0; *done = 0u; }
+    for (int g = lo; g < hi; ++g) {
+        run += voff[g + 1];
+        voff[g + 1] = run;
     }
     __syncthreads();
-    for (int f = warp; f < n_frames; f += nwarps) {
-        int pos = next_off[f];
+    for (int g = warp; g < n_frames; g += nwarps) {
+        int pos = voff[g];
         for (int q = 0; q < AW; ++q) {
-            const uint64_t m = masks[(size_t)f * AW + q];
+            const uint64_t m = vmasks[(size_t)g * AW + q];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 const uint32_t bits = (uint32_t)(m >> (32 * half));
@@ -576,7 +625,8 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
                           const int* first, const uint64_t* provider, uint64_t* mask_scratch,
                           int* next_off, int* next_ids, int ids_capacity) {
     ProfScope ps(L, KC_OTHER);
-    select_kernel<<<1, 1024, 0, L.st>>>(scores, n_frames, n_classes, n_adapters, thr, context_copy,
+    const int blocks = n_frames > 0 ? (n_frames + SELECT_THREADS / 32 - 1) / (SELECT_THREADS / 32) : 1;
+    select_kernel<<<blocks, SELECT_THREADS, 0, L.st>>>(scores, n_frames, n_classes, n_adapters, thr, context_copy,
                                         has_prev, prev_labels, prev_off, prev_ids, first, provider,
                                         mask_scratch, next_off, next_ids, ids_capacity, L.status);
     BUMP(L);
@@ -594,7 +644,7 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
 // can still run the selection.  Every GPU that loads the library carries the array until exit.
 #define PM_SELECT_STATIC_WORDS (PM_SELECT_STATIC_MAX_FRAMES * (PM_SELECT_STATIC_MAX_ADAPTERS / 64))
 
-static __device__ __align__(256) unsigned long long pm_select_static_masks[PM_SELECT_STATIC_WORDS];
+static __device__ __align__(256) unsigned long long pm_select_static_masks[PM_SELECT_STATIC_WORDS + 1];   // + block counter
 static __device__ __align__(256) int pm_select_static_status[64];   // word 0: status when the caller passes none
 
 namespace {
@@ -633,8 +683,12 @@ extern "C" int pm_select_static(const float* scores, int n_frames, int n_classes
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int* status = status_out ? status_out : g_static_scratch[dev].status;
-    // the status word is the only thing that must start at zero; the mask words are all rewritten
-    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return PM_ERR_CUDA;
+    // what must start at zero: the status word and the kernel's block counter (the word after the
+    // last mask word of this call); the mask words themselves are all rewritten before they are read
+    const size_t counter_at = (size_t)n_frames * ((n_adapters + 63) / 64);
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess ||
+        cudaMemsetAsync(g_static_scratch[dev].masks + counter_at, 0, sizeof(uint64_t), st) != cudaSuccess)
+        return PM_ERR_CUDA;
     Launch L;
     L.st = st;
     L.status = status;
