@@ -187,7 +187,8 @@ __global__ void __launch_bounds__(512) attention_mma_kernel(const bf16* __restri
 // yields each row's maximum over all keys, the second forms P against that final maximum and
 // accumulates O over the blocks, so no rescaling of O is ever needed.
 // The issuing thread and the softmax warps alternate through two mbarriers (scores / O ready,
-// rows done); two CTAs per SM overlap one head's softmax with another's loads and MMAs.
+// rows done); with one key block three CTAs fit an SM: two hold tensor memory and compute while the
+// third, whose loads were issued before it asked for tensor memory, waits for columns.
 // ---------------------------------------------------------------------------------------
 constexpr int AQ = 128;                    // query rows per tile
 constexpr int AKB = 208;                   // keys per score block
@@ -206,29 +207,70 @@ struct AttnArgs {
 // maximum of the first `lim` of 32 score columns (all of them if lim >= 32)
 template <int N, bool MASK>
 __device__ __forceinline__ float chunk_max(const uint32_t* v, int lim, float m) {
+    float t[4] = {m, -INFINITY, -INFINITY, -INFINITY};       // four independent chains
 #pragma unroll
     for (int j = 0; j < N; ++j) {
         const float sj = __uint_as_float(v[j]);
-        m = fmaxf(m, (!MASK || j < lim) ? sj : -INFINITY);
+        t[j & 3] = fmaxf(t[j & 3], (!MASK || j < lim) ? sj : -INFINITY);
     }
-    return m;
+    return fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3]));
+}
+__device__ __forceinline__ float ex2_approx(float x) {     // one MUFU instruction; flushes denormals
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 // p_j = exp2(c s_j - mc) (0 beyond lim), packed to bf16 pairs; returns the sum of the p_j
 template <int N, bool MASK>
 __device__ __forceinline__ float chunk_probs(const uint32_t* v, int lim, float c, float mc, uint32_t* packed) {
-    float sum = 0.f;
+    float sum[4] = {0.f, 0.f, 0.f, 0.f};                     // four independent chains
 #pragma unroll
     for (int j = 0; j < N; j += 2) {
-        float p0 = exp2f(fmaf(__uint_as_float(v[j]), c, -mc));
-        float p1 = exp2f(fmaf(__uint_as_float(v[j + 1]), c, -mc));
+        float p0 = ex2_approx(fmaf(__uint_as_float(v[j]), c, -mc));
+        float p1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), c, -mc));
         if (MASK) { p0 = j < lim ? p0 : 0.f; p1 = j + 1 < lim ? p1 : 0.f; }
-        sum += p0 + p1;
+        sum[(j >> 1) & 3] += p0 + p1;
         packed[j >> 1] = pack2(p0, p1);
     }
-    return sum;
+    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
-__global__ void __launch_bounds__(ATT_THREADS)
+// One sweep over a score block of nb columns (a multiple of 16), 16 columns at a time, with the
+// tensor-memory load of the next chunk in flight while the current one is processed.
+// PROBS = false: running row maximum (acc in, acc out).  PROBS = true: writes P (packed bf16) over
+// the scores and returns acc + the row sum of this block.  Columns at or beyond `valid` are ignored.
+template <bool PROBS>
+__device__ __forceinline__ float score_chunk(uint32_t t_lane, const uint32_t* v, int c0, int valid, float c,
+                                             float mc, float acc) {
+    const int lim = valid - c0;
+    if (PROBS) {
+        uint32_t pk[8];
+        acc += lim >= 16 ? chunk_probs<16, false>(v, 16, c, mc, pk) : chunk_probs<16, true>(v, lim, c, mc, pk);
+        tmem_st8(t_lane + (uint32_t)(c0 >> 1), pk);
+        return acc;
+    }
+    return lim >= 16 ? chunk_max<16, false>(v, 16, acc) : chunk_max<16, true>(v, lim, acc);
+}
+template <bool PROBS>
+__device__ __forceinline__ float score_block_sweep(uint32_t t_lane, int nb, int valid, float c, float mc, float acc) {
+    uint32_t va[16], vb[16];
+    tmem_ld16(t_lane, va);
+    tmem_ld_wait();
+#pragma unroll 1
+    for (int c0 = 0; c0 < nb; c0 += 32) {
+        if (c0 + 16 < nb) tmem_ld16(t_lane + (uint32_t)(c0 + 16), vb);
+        acc = score_chunk<PROBS>(t_lane, va, c0, valid, c, mc, acc);
+        tmem_ld_wait();
+        if (c0 + 16 < nb) {
+            if (c0 + 32 < nb) tmem_ld16(t_lane + (uint32_t)(c0 + 32), va);
+            acc = score_chunk<PROBS>(t_lane, vb, c0 + 16, valid, c, mc, acc);
+            tmem_ld_wait();
+        }
+    }
+    return acc;
+}
+
+__global__ void __launch_bounds__(ATT_THREADS, 3)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
                     const AttnArgs args) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -241,22 +283,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int d = args.heads * HD;
     const int T = args.tokens;
     const int n_blocks = args.n_blocks;
-    const uint32_t q_s = base;                               // two query-tile buffers
-    const uint32_t k_s = q_s + 2 * AQ_BYTES;
+    const uint32_t q_s = base;
+    const uint32_t k_s = q_s + AQ_BYTES;
     const uint32_t v_s = k_s + n_blocks * AKB_BYTES;
     const uint32_t bars = v_s + n_blocks * AKB_BYTES;
-    const uint32_t kv_bar = bars, s_bar = bars + 8, r_bar = bars + 16, q_bar0 = bars + 24;   // q_bar0, q_bar0 + 8
+    const uint32_t kv_bar = bars, s_bar = bars + 8, r_bar = bars + 16, q_bar = bars + 24;
     uint8_t* bar_ptr = smem_raw + (bars - base);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 40);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 48);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 40);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(kv_bar, 1); mbar_init(q_bar0, 1); mbar_init(q_bar0 + 8, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4);
+        mbar_init(kv_bar, 1); mbar_init(q_bar, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // All operand loads of the head go out before tensor memory is requested: with three CTAs
+        // resident per SM but tensor memory for two, the third one's loads land while it waits for
+        // its columns.
+        mbar_expect_tx(kv_bar, (uint32_t)(n_blocks * 2 * AKB_BYTES));
+        for (int b = 0; b < n_blocks; ++b) {
+            tma_load_2d(k_s + b * AKB_BYTES, &tm_kv, d + h * HD, f * T + b * AKB, kv_bar);
+            tma_load_2d(v_s + b * AKB_BYTES, &tm_kv, 2 * d + h * HD, f * T + b * AKB, kv_bar);
+        }
+        mbar_expect_tx(q_bar, AQ_BYTES);
+        tma_load_2d(q_s, &tm_q, h * HD, f * T, q_bar);
     }
+    __syncwarp();
     if (warp == 0) {
         tmem_alloc(smem_u32((const void*)tmem_slot), args.tmem_cols);
         tmem_relinquish();
@@ -270,34 +323,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (warp == 0) {
         if (lane == 0) {
             // ------------------------------------------------------ TMA + MMA issue
-            mbar_expect_tx(kv_bar, (uint32_t)(n_blocks * 2 * AKB_BYTES));
-            for (int b = 0; b < n_blocks; ++b) {
-                tma_load_2d(k_s + b * AKB_BYTES, &tm_kv, d + h * HD, f * T + b * AKB, kv_bar);
-                tma_load_2d(v_s + b * AKB_BYTES, &tm_kv, 2 * d + h * HD, f * T + b * AKB, kv_bar);
-            }
             const uint32_t idesc_pv = instr_desc_b_mn(HD);
             uint32_t step = 0;
             bool ok = true;
-            auto load_q = [&](int qt) {       // the buffer's previous tile (qt - 2) has been consumed
-                const uint32_t bar = q_bar0 + 8u * (qt & 1);
-                mbar_expect_tx(bar, AQ_BYTES);
-                tma_load_2d(q_s + (qt & 1) * AQ_BYTES, &tm_q, h * HD, f * T + qt * AQ, bar);
-            };
-            load_q(0);
             for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
-                if (qt + 1 < args.n_qtiles) load_q(qt + 1);
                 if (qt == 0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
-                ok = ok && mbar_wait(q_bar0 + 8u * (qt & 1), (qt >> 1) & 1, abort_flag, args.status);
+                ok = ok && mbar_wait(q_bar, qt & 1, abort_flag, args.status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t q_cur = q_s + (qt & 1) * AQ_BYTES;
                 for (int pass = (n_blocks > 1 ? 0 : 1); pass < 2 && ok; ++pass) {
                     for (int b = 0; b < n_blocks && ok; ++b) {
                         const int nb = min(AKB, args.tpad - b * AKB);
                         const uint32_t idesc_s = instr_desc(nb);
 #pragma unroll
                         for (int k = 0; k < HD / 16; ++k)
-                            umma_bf16(tmem_base, smem_desc(q_cur + k * 32, 128),
+                            umma_bf16(tmem_base, smem_desc(q_s + k * 32, 128),
                                       smem_desc(k_s + b * AKB_BYTES + k * 32, 128), idesc_s, k > 0);
                         umma_commit(s_bar);
                         ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
@@ -305,6 +345,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (!ok) break;
                         tc_fence_after();
                         if (pass == 1) {
+                            if (b == n_blocks - 1 && qt + 1 < args.n_qtiles) {
+                                // the last scores of this tile exist, so its query rows are no longer
+                                // needed: fetch the next tile's behind the P V products
+                                mbar_expect_tx(q_bar, AQ_BYTES);
+                                tma_load_2d(q_s, &tm_q, h * HD, f * T + (qt + 1) * AQ, q_bar);
+                            }
                             for (int kk = 0; kk < nb / 16; ++kk)
                                 umma_bf16_ts(o_tmem, tmem_base + (uint32_t)(kk * 8),
                                              smem_desc(v_s + b * AKB_BYTES + kk * 2048, 128), idesc_pv,
@@ -338,22 +384,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (lane == 0) mbar_arrive(r_bar);
             ++step;
         };
-        // row maximum of one score block (columns at or beyond `valid` are ignored)
-        auto block_max = [&](int nb, int valid, float m) {
-            for (int c0 = 0; c0 < nb; c0 += 32) {
-                uint32_t v[32];
-                if (nb - c0 >= 32) {
-                    tmem_ld32(t_lane + (uint32_t)c0, v);
-                    tmem_ld_wait();
-                    m = (valid - c0 >= 32) ? chunk_max<32, false>(v, 32, m) : chunk_max<32, true>(v, valid - c0, m);
-                } else {
-                    tmem_ld16(t_lane + (uint32_t)c0, v);
-                    tmem_ld_wait();
-                    m = (valid - c0 >= 16) ? chunk_max<16, false>(v, 16, m) : chunk_max<16, true>(v, valid - c0, m);
-                }
-            }
-            return m;
-        };
         for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
             const int q_row = qt * AQ + quarter * 32 + lane;
             const bool warp_active = qt * AQ + quarter * 32 < T;      // else: no row of this warp exists
@@ -361,7 +391,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (n_blocks > 1) {
                 for (int b = 0; b < n_blocks; ++b) {
                     if (!begin_step()) break;
-                    if (warp_active) m = block_max(min(AKB, args.tpad - b * AKB), T - b * AKB, m);
+                    if (warp_active)
+                        m = score_block_sweep<false>(t_lane, min(AKB, args.tpad - b * AKB), T - b * AKB, 0.f, 0.f, m);
                     end_step();
                 }
                 if (!ok) break;
@@ -370,24 +401,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const int nb = min(AKB, args.tpad - b * AKB), valid = T - b * AKB;
                 if (!begin_step()) break;
                 if (warp_active) {
-                    if (n_blocks == 1) m = block_max(nb, valid, m);
-                    const float mc = m * c;
-                    for (int c0 = 0; c0 < nb; c0 += 32) {
-                        uint32_t v[32], pk[16];
-                        if (nb - c0 >= 32) {
-                            tmem_ld32(t_lane + (uint32_t)c0, v);
-                            tmem_ld_wait();
-                            l += (valid - c0 >= 32) ? chunk_probs<32, false>(v, 32, c, mc, pk)
-                                                    : chunk_probs<32, true>(v, valid - c0, c, mc, pk);
-                            tmem_st16(t_lane + (uint32_t)(c0 >> 1), pk);
-                        } else {
-                            tmem_ld16(t_lane + (uint32_t)c0, v);
-                            tmem_ld_wait();
-                            l += (valid - c0 >= 16) ? chunk_probs<16, false>(v, 16, c, mc, pk)
-                                                    : chunk_probs<16, true>(v, valid - c0, c, mc, pk);
-                            tmem_st8(t_lane + (uint32_t)(c0 >> 1), pk);
-                        }
-                    }
+                    if (n_blocks == 1) m = score_block_sweep<false>(t_lane, nb, valid, 0.f, 0.f, m);
+                    l = score_block_sweep<true>(t_lane, nb, valid, c, m * c, l);
                     tmem_st_wait();
                 }
                 end_step();
@@ -456,9 +471,8 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
     a.tmem_cols = a.n_blocks == 1 ? 256u : 512u;
     a.o_col = a.n_blocks == 1 ? 128u : 256u;
     a.out = out; a.status = L.status;
-    // at least 110 KB, so that no more than two CTAs (2 x 256 TMEM columns) share an SM
-    size_t smem = (size_t)2 * AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
-    if (smem < 110 * 1024) smem = 110 * 1024;
+    // one block: 68 KB, three CTAs per SM (two computing, the third loading while it waits for TMEM)
+    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
     static size_t smem_set = 0;
     if (smem > smem_set) {
         cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
