@@ -408,7 +408,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
         if constexpr (TC) {
             const bool use_lora = lora && R.max_set > 0;
             if (use_lora) {
-                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>());
+                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>(), h->n_sms);
                 if (e != cudaSuccess) return e;
             }
             const CUtensorMap* tmy = (void*)y == h->QKV.p ? &h->tm_y_qkv
@@ -785,7 +785,7 @@ int pm_linear_forward(pm_linear l, const void* x, int n_frames, const int32_t* s
             err = "cuTensorMapEncodeTiled failed (y); y must be 16-byte aligned"; return PM_ERR_CUDA;
         }
         const bool lora = R.max_set > 0 && l->lin.dev.lora.At != nullptr;
-        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>()));
+        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>(), l->n_sms));
         CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, &tm_y, rows, l->epilogue,
                             (const bf16*)residual, none, (bf16*)y, l->n_sms));
     } else {

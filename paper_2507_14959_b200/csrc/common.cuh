@@ -131,7 +131,7 @@ cudaError_t launch_naive_linear(const Launch& L, const LinearDev& lin, const Rou
                                 const PatchEpi& pe, T* y);
 // tensor-core path (bf16): shrink into the slab buffer, then the fused GEMM
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf);
+                          const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf, int n_sms);
 // tm_y: [rows, n_out] output map with a (32 x 32) box and 64B swizzle for the TMA-store epilogue, or
 // null to store straight from registers (always the case for EPI_PATCH, whose rows are remapped)
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,

@@ -380,15 +380,17 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 // ---------------------------------------------------------------------------------------
 // shrink on the tensor cores: t[tile][s][row][j] = mask(row) * s_a * sum_k x[row,k] A_a[k, 16 s' + j]
 //
-// One CTA per 128-row tile.  The tile's LoRA slabs are taken `sg` at a time: for each group the
-// x tile streams through shared memory once (TMA, 128B swizzle) next to the group's A^T slabs
-// (16 rows of the arena per slab, stacked), one UMMA of N = 16 * slabs per 16 K-columns
-// accumulates into TMEM, and the epilogue warps scale, mask, round to bf16 and store each slab
-// as a [128 x 16] block -- the layout the fused GEMM fetches as a 32B-swizzled operand.
+// Persistent: each CTA walks 128-row tiles (tile = blockIdx.x, += gridDim.x) and, inside a tile,
+// groups of up to `sg` LoRA slabs.  For each (tile, group) the x tile streams through shared
+// memory once (TMA, 128B swizzle) next to the group's A^T slabs (16 arena rows per slab, stacked),
+// one UMMA of N = 16 * slabs per 16 K-columns accumulates into one of two TMEM buffers, and the
+// epilogue warps scale, mask, round to bf16 and store each slab as a [128 x 16] block -- the
+// layout the fused GEMM fetches as a 32B-swizzled operand.  The TMA ring and the accumulator
+// buffers carry on across tiles, so loads of the next tile run under the arithmetic of this one.
 // ---------------------------------------------------------------------------------------
 struct ShrinkArgs {
-    int rows, k_in, slab_cap, sg;
-    uint32_t tmem_cols;
+    int rows, k_in, slab_cap, sg, n_tiles, stages;
+    uint32_t acc_cols;             // TMEM columns of one accumulator buffer (power of two >= 16 * sg)
     const int* tile_nslabs;
     const int* tile_slab;
     const float* tile_scale;
@@ -397,45 +399,42 @@ struct ShrinkArgs {
     int* status;
 };
 
-constexpr int SHRINK_STAGES = 3;
+constexpr int SHRINK_MAX_STAGES = 4;
 constexpr int SHRINK_X_BYTES = BM * BK * 2;          // 16 KB
 constexpr int SHRINK_A_SLAB_BYTES = PM_SLAB * BK * 2; // 2 KB: 16 arena rows x 64 K-columns
-
 
 __global__ void __launch_bounds__(SHRINK_THREADS)
 shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_at,
                  const ShrinkArgs args) {
-    const int tile = blockIdx.x;
-    const int ns = args.tile_nslabs[tile];
-    if (ns == 0) return;                                   // uniform: nothing allocated yet
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t* smem = smem_raw + (base - raw);
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t base = smem_u32(smem);
+    if (base & 1023u) {                       // swizzled operands need a 1024-byte aligned window
+        if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
+        return;
+    }
+    const int STG = args.stages;
     const int stage_bytes = SHRINK_X_BYTES + args.sg * SHRINK_A_SLAB_BYTES;
-    const int bar_off = SHRINK_STAGES * stage_bytes;
+    const int bar_off = STG * stage_bytes;
     const uint32_t bars = base + bar_off;
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (SHRINK_STAGES + s); };
-    const uint32_t tfull_bar = bars + 8u * (2 * SHRINK_STAGES);
-    const uint32_t tempty_bar = bars + 8u * (2 * SHRINK_STAGES + 1);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + bar_off + 8 * (2 * SHRINK_STAGES + 2));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + bar_off + 8 * (2 * SHRINK_STAGES + 2) + 8);
+    auto empty_bar = [&](int s) { return bars + 8u * (SHRINK_MAX_STAGES + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * SHRINK_MAX_STAGES + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * SHRINK_MAX_STAGES + 2 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + bar_off + 8 * (2 * SHRINK_MAX_STAGES + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + bar_off + 8 * (2 * SHRINK_MAX_STAGES + 4) + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = args.k_in / BK;
-    const int n_groups = (ns + args.sg - 1) / args.sg;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < SHRINK_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        mbar_init(tfull_bar, 1);
-        mbar_init(tempty_bar, 4);
+        for (int s = 0; s < STG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32((const void*)tmem_slot), args.tmem_cols);
+        tmem_alloc(smem_u32((const void*)tmem_slot), 2 * args.acc_cols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -445,88 +444,103 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 
     if (warp == 0) {
         if (lane == 0) {
+            // -------------------------------------------------------------- TMA producer
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int g = 0; g < n_groups && ok; ++g) {
-                const int cnt = min(args.sg, ns - g * args.sg);
-                for (int kb = 0; kb < num_kb && ok; ++kb) {
-                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
-                    if (!ok) break;
-                    mbar_expect_tx(full_bar(stage), SHRINK_X_BYTES + cnt * SHRINK_A_SLAB_BYTES);
-                    const uint32_t sa = base + stage * stage_bytes;
-                    tma_load_2d(sa, &tm_x, kb * BK, tile * BM, full_bar(stage));
-                    for (int i = 0; i < cnt; ++i) {
-                        const int slab = args.tile_slab[tile * args.slab_cap + g * args.sg + i];
-                        tma_load_2d(sa + SHRINK_X_BYTES + i * SHRINK_A_SLAB_BYTES, &tm_at, kb * BK,
-                                    slab * PM_SLAB, full_bar(stage));
+            for (int tile = blockIdx.x; tile < args.n_tiles && ok; tile += gridDim.x) {
+                const int ns = args.tile_nslabs[tile];
+                for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
+                    const int cnt = min(args.sg, ns - g0);
+                    for (int kb = 0; kb < num_kb && ok; ++kb) {
+                        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                        if (!ok) break;
+                        mbar_expect_tx(full_bar(stage), SHRINK_X_BYTES + cnt * SHRINK_A_SLAB_BYTES);
+                        const uint32_t sa = base + stage * stage_bytes;
+                        tma_load_2d(sa, &tm_x, kb * BK, tile * BM, full_bar(stage));
+                        for (int i = 0; i < cnt; ++i) {
+                            const int slab = args.tile_slab[tile * args.slab_cap + g0 + i];
+                            tma_load_2d(sa + SHRINK_X_BYTES + i * SHRINK_A_SLAB_BYTES, &tm_at, kb * BK,
+                                        slab * PM_SLAB, full_bar(stage));
+                        }
+                        if (++stage == STG) { stage = 0; phase ^= 1u; }
                     }
-                    if (++stage == SHRINK_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            int stage = 0;
+            // -------------------------------------------------------------- MMA issuer
+            int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int g = 0; g < n_groups && ok; ++g) {
-                const int cnt = min(args.sg, ns - g * args.sg);
-                const uint32_t idesc = instr_desc(cnt * PM_SLAB);
-                ok = mbar_wait(tempty_bar, acc_phase ^ 1u, abort_flag, args.status);
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t accumulate = 0;
-                for (int kb = 0; kb < num_kb && ok; ++kb) {
-                    ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+            for (int tile = blockIdx.x; tile < args.n_tiles && ok; tile += gridDim.x) {
+                const int ns = args.tile_nslabs[tile];
+                for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
+                    const int cnt = min(args.sg, ns - g0);
+                    const uint32_t idesc = instr_desc(cnt * PM_SLAB);
+                    ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, args.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = base + stage * stage_bytes;
-                    const uint32_t sb = sa + SHRINK_X_BYTES;
+                    const uint32_t d_tmem = tmem_base + (uint32_t)acc * args.acc_cols;
+                    uint32_t accumulate = 0;
+                    for (int kb = 0; kb < num_kb && ok; ++kb) {
+                        ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t sa = base + stage * stage_bytes;
+                        const uint32_t sb = sa + SHRINK_X_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k) {
-                        umma_bf16(tmem_base, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
-                                  accumulate);
-                        accumulate = 1;
+                        for (int k = 0; k < BK / 16; ++k) {
+                            umma_bf16(d_tmem, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
+                                      accumulate);
+                            accumulate = 1;
+                        }
+                        umma_commit(empty_bar(stage));
+                        if (++stage == STG) { stage = 0; phase ^= 1u; }
                     }
-                    umma_commit(empty_bar(stage));
-                    if (++stage == SHRINK_STAGES) { stage = 0; phase ^= 1u; }
+                    if (ok) umma_commit(tfull_bar(acc));
+                    if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
                 }
-                if (ok) umma_commit(tfull_bar);
-                acc_phase ^= 1u;
             }
         }
     } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;
         const int r = quarter * 32 + lane;
+        int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int g = 0; g < n_groups && ok; ++g) {
-            const int cnt = min(args.sg, ns - g * args.sg);
-            ok = mbar_wait(tfull_bar, acc_phase, abort_flag, args.status);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            for (int i = 0; i < cnt; ++i) {
-                const int slot = tile * args.slab_cap + g * args.sg + i;
-                uint32_t v[16];
-                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(i * PM_SLAB), v);
-                tmem_ld_wait();
-                const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
-                const float sc = on ? args.tile_scale[slot] : 0.f;
-                uint4 o[2];
-                uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+        for (int tile = blockIdx.x; tile < args.n_tiles && ok; tile += gridDim.x) {
+            const int ns = args.tile_nslabs[tile];
+            for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
+                const int cnt = min(args.sg, ns - g0);
+                ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, args.status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * args.acc_cols;
+                for (int i = 0; i < cnt; ++i) {
+                    const int slot = tile * args.slab_cap + g0 + i;
+                    uint32_t v[16];
+                    tmem_ld16(t_row + (uint32_t)(i * PM_SLAB), v);
+                    tmem_ld_wait();
+                    const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
+                    const float sc = on ? args.tile_scale[slot] : 0.f;
+                    uint4 o[2];
+                    uint32_t* ow = reinterpret_cast<uint32_t*>(o);
 #pragma unroll
-                for (int j = 0; j < PM_SLAB; j += 2)
-                    ow[j >> 1] = pack_bf16(__uint_as_float(v[j]) * sc, __uint_as_float(v[j + 1]) * sc);
-                uint4* dst = reinterpret_cast<uint4*>(args.tbuf + ((size_t)slot * BM + r) * PM_SLAB);
-                dst[0] = o[0];
-                dst[1] = o[1];
+                    for (int j = 0; j < PM_SLAB; j += 2)
+                        ow[j >> 1] = pack_bf16(__uint_as_float(v[j]) * sc, __uint_as_float(v[j + 1]) * sc);
+                    uint4* dst = reinterpret_cast<uint4*>(args.tbuf + ((size_t)slot * BM + r) * PM_SLAB);
+                    dst[0] = o[0];
+                    dst[1] = o[1];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar);
-            acc_phase ^= 1u;
         }
     }
     __syncwarp();
@@ -537,7 +551,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, args.tmem_cols);
+        tmem_dealloc(tmem_base, 2 * args.acc_cols);
     }
 }
 
@@ -597,25 +611,30 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 }
 
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf) {
+                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int n_sms) {
     if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
     ShrinkArgs a;
-    a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap;
+    a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap; a.n_tiles = R.n_tiles;
     a.sg = R.slab_cap < 16 ? R.slab_cap : 16;
     uint32_t cols = 32;
     while ((int)cols < a.sg * PM_SLAB) cols <<= 1;
-    a.tmem_cols = cols;
+    a.acc_cols = cols;                                   // two buffers: at most 2 x 256 columns
+    const int stage_bytes = SHRINK_X_BYTES + a.sg * SHRINK_A_SLAB_BYTES;
+    // four stages while two CTAs still fit an SM (and their 2 x 2 accumulators fit its TMEM)
+    a.stages = (4 * stage_bytes + 256 <= 112 * 1024) ? 4 : 3;
     a.tile_nslabs = R.tile_nslabs; a.tile_slab = R.tile_slab; a.tile_scale = R.tile_scale;
     a.tile_mask = R.tile_mask; a.tbuf = tbuf; a.status = L.status;
-    const int smem = SHRINK_STAGES * (SHRINK_X_BYTES + a.sg * SHRINK_A_SLAB_BYTES) + 256 + 1024;
+    const int smem = a.stages * stage_bytes + 256;
     static int smem_set = 0;
     if (smem > smem_set) {
         cudaError_t e = cudaFuncSetAttribute(shrink_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
+    const int per_sm = (2 * smem + 4096 <= 227 * 1024 && 4 * cols <= 512) ? 2 : 1;
+    const int grid = R.n_tiles < n_sms * per_sm ? R.n_tiles : n_sms * per_sm;
     ProfScope ps(L, KC_SHRINK);
-    shrink_tc_kernel<<<R.n_tiles, SHRINK_THREADS, smem, L.st>>>(*tm_x, lin.tm_at, a);
+    shrink_tc_kernel<<<grid, SHRINK_THREADS, smem, L.st>>>(*tm_x, lin.tm_at, a);
     BUMP(L);
     return cudaGetLastError();
 }
