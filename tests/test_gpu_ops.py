@@ -132,6 +132,37 @@ def test_lora_linear(dtype, case):
     lin.close()
 
 
+def test_lora_linear_full_size_sampled():
+    """One cell of the single-linear grid at full size (256 frames x 197 tokens, 768 -> 2304, 128
+    rank-16 adapters, 1-8 active per frame) in the launch configuration the sweep times; the oracle
+    computes sampled rows one by one (first and last row tiles, frame boundaries, the ragged tail)."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    cell = wl.linear_cell(768, 2304, 256, 16, clustered=False)
+    lin = binding.Linear(cell.w, cell.b, max_adapters=128, max_rank=16, max_set=8, max_frames=256,
+                         tokens=cell.tokens, epilogue=0, dtype=0)
+    for a in range(128):
+        lin.register(a, 16, cell.scale, cell.A[a], cell.B[a])
+    rows = 256 * cell.tokens
+    xd = to_dev(cell.x, 0)
+    yd = torch.full((rows, 2304), float("nan"), device="cuda", dtype=torch.bfloat16)
+    lin.forward(xd, 256, cell.set_offsets, cell.set_ids, yd)
+    assert lin.status() == 0
+    assert not torch.isnan(yd.float()).any()
+    g = wl.rng_for("full_size_rows")
+    sample = sorted(set([0, 127, 128, 196, 197, 198, rows - 1, rows - 65, rows - 128, rows - 129]
+                        + [int(r) for r in g.integers(0, rows, 54)]))
+    got = to_np(yd[sample])
+    w64, b64 = cell.w.astype(np.float64), cell.b.astype(np.float64)
+    for i, r in enumerate(sample):
+        f = r // cell.tokens
+        act = [(cell.scale, cell.A[a].astype(np.float64), cell.B[a].astype(np.float64))
+               for a in sorted(cell.set_ids[cell.set_offsets[f]:cell.set_offsets[f + 1]])]
+        want = po.lora_linear(cell.x[r:r + 1].astype(np.float64), w64, b64, act)[0]
+        np.testing.assert_allclose(got[i], want, **TOL[0])
+    lin.close()
+
+
 def test_gelu_epilogue_accuracy():
     """The GELU epilogue against the exact-erf definition: y = gelu(4 x) through an identity-like
     weight, x sweeping [-3, 3] (so the argument spans [-12, 12]); the bf16 result must be within one
