@@ -96,6 +96,14 @@ struct LinearObj {
             }
             if (!ok) { err = "cuTensorMapEncodeTiled failed (static operands)"; return PM_ERR_CUDA; }
             dev.has_tm = true;
+            if (n_out % 256 == 0) {
+                ok = tm_encode_2d(&dev.tm_w_half, wt.p, k_in, n_out, (uint64_t)k_in * 2, 64, 128, 128);
+                if (ok && dev.lora.At)
+                    ok = tm_encode_2d(&dev.tm_bt_half, bt.p, PM_SLAB, (uint64_t)max_adapters * slabs_max * n_out,
+                                      PM_SLAB * 2, PM_SLAB, 128, 32);
+                if (!ok) { err = "cuTensorMapEncodeTiled failed (half-tile operands)"; return PM_ERR_CUDA; }
+                dev.has_tm_half = true;
+            }
         }
         return PM_OK;
     }
@@ -146,9 +154,9 @@ struct Router {
     int init(int max_frames_, int max_set_, int max_adapters_, int slabs_max_, int tokens_, std::string& err) {
         max_frames = max_frames_; max_set = max_set_; max_adapters = max_adapters_;
         slabs_max = slabs_max_; tokens = tokens_;
-        const int frames_per_tile = (PM_TILE_M - 1) / tokens + 2;
-        slab_cap = std::min(frames_per_tile * max_set, max_adapters) * slabs_max;
-        max_tiles = (int)(((size_t)max_frames * tokens + PM_TILE_M - 1) / PM_TILE_M);
+        const int frames_per_pair = (2 * PM_TILE_M - 1) / tokens + 2;      // frames a 256-row pair can touch
+        slab_cap = std::min(frames_per_pair * max_set, max_adapters) * slabs_max;
+        max_tiles = (int)(((size_t)max_frames * tokens + 2 * PM_TILE_M - 1) / (2 * PM_TILE_M)) * 2;   // even
         auto take = [&](size_t& off, size_t bytes) { off = blob_bytes; blob_bytes += (bytes + 255) & ~(size_t)255; };
         take(off_perm, sizeof(int) * max_frames);
         take(off_soff, sizeof(int) * (max_frames + 1));
@@ -218,10 +226,11 @@ struct Router {
             h_soff[i + 1] = h_soff[i] + (int)st_.size();
         }
         const long long rows = (long long)n_frames * tokens;
-        const int n_tiles = (int)((rows + PM_TILE_M - 1) / PM_TILE_M);
-        for (int t = 0; t < n_tiles; ++t) {
-            const long long r0 = (long long)t * PM_TILE_M, r1 = std::min(rows, r0 + PM_TILE_M);
-            std::map<int, std::array<uint32_t, 4>> slabs;      // arena slab -> row mask, ascending
+        const int n_pairs = (int)((rows + 2 * PM_TILE_M - 1) / (2 * PM_TILE_M));
+        const int n_tiles = 2 * n_pairs;
+        for (int p = 0; p < n_pairs; ++p) {
+            const long long r0 = (long long)p * 2 * PM_TILE_M, r1 = std::min(rows, r0 + 2 * PM_TILE_M);
+            std::map<int, std::array<uint32_t, 8>> slabs;      // arena slab -> 256-bit row mask, ascending
             for (int slot = (int)(r0 / tokens); slot <= (int)((r1 - 1) / tokens); ++slot) {
                 const long long a0 = std::max(r0, (long long)slot * tokens);
                 const long long a1 = std::min(r1, (long long)(slot + 1) * tokens);
@@ -234,13 +243,16 @@ struct Router {
                 }
             }
             if ((int)slabs.size() > slab_cap) { err = "tile needs more LoRA slabs than the plan capacity"; return PM_ERR_CAPACITY; }
-            h_tn[t] = (int)slabs.size();
-            int i = 0;
-            for (auto& kv : slabs) {
-                const size_t at = (size_t)t * slab_cap + i++;
-                h_ts[at] = kv.first;
-                h_tsc[at] = scales[kv.first / slabs_max];
-                for (int q = 0; q < 4; ++q) h_tm[at * 4 + q] = kv.second[q];
+            for (int half = 0; half < 2; ++half) {
+                const int t = 2 * p + half;
+                h_tn[t] = (int)slabs.size();
+                int i = 0;
+                for (auto& kv : slabs) {
+                    const size_t at = (size_t)t * slab_cap + i++;
+                    h_ts[at] = kv.first;
+                    h_tsc[at] = scales[kv.first / slabs_max];
+                    for (int q = 0; q < 4; ++q) h_tm[at * 4 + q] = kv.second[half * 4 + q];
+                }
             }
         }
         CK(cudaMemcpyAsync(blob.p, stage, blob_bytes, cudaMemcpyHostToDevice, st));

@@ -35,6 +35,9 @@ struct LinearDev {
     // tensor maps of the static operands (bf16 build only)
     CUtensorMap tm_w, tm_at, tm_bt;
     bool has_tm = false;
+    // n_out a multiple of 256: boxes of 128 output columns for the CTA-pair GEMM
+    CUtensorMap tm_w_half, tm_bt_half;
+    bool has_tm_half = false;
 };
 
 // Per-batch routing of frames to adapters, in SLOT order (slot = position after bucketing
@@ -44,7 +47,9 @@ struct RouteDev {
     int* perm = nullptr;        // [F] slot -> caller's frame index
     int* slot_off = nullptr;    // [F+1] CSR over slots
     int* slot_ids = nullptr;    // [nnz] ascending adapter ids per slot
-    // tile plan (rows 128*t .. 128*t+127): the union of the LoRA slabs its rows need
+    // tile plan (rows 128*t .. 128*t+127).  Tiles 2p and 2p+1 carry the SAME slab list, the union of
+    // what the 256 rows of the pair need (the CTA-pair GEMM applies one slab to both halves); a
+    // tile's mask is zero for a slab none of its rows uses.  n_tiles is even.
     int* tile_nslabs = nullptr;     // [n_tiles]
     int* tile_slab = nullptr;       // [n_tiles, slab_cap] arena slab index a*slabs_max + s
     float* tile_scale = nullptr;    // [n_tiles, slab_cap] s_a

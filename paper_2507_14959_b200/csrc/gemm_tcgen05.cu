@@ -13,6 +13,8 @@
 // warps per TMEM lane quarter, each taking half of the tile's columns).
 // Every mbarrier wait is bounded: on expiry the CTA raises an abort flag, records
 // PM_ERR_TIMEOUT in the status word, drains and returns.
+// When n_out is a multiple of 256 the CTA-pair variant (lora_gemm_pair_kernel, cta_group::2, 256 x 256
+// tiles) is used; the single-CTA kernel serves the narrower shapes.
 #include "common.cuh"
 #include "tcgen05_ptx.cuh"
 
@@ -81,6 +83,130 @@ struct Smem {
     static constexpr int TOTAL = BAR_OFFSET + 256;             // + barriers (base must be 1024-aligned)
 };
 
+// Epilogue of one 128 x BN accumulator by one epilogue warp: its share of the tile's 32-column
+// chunks goes TMEM -> registers -> bias / GELU / residual / patch placement -> bf16 -> shared
+// memory -> TMA store (or straight to global memory).  Returns false once the CTA is aborting.
+// PAIR: the accumulator-free barrier lives in the even CTA of a pair (tempty_addr is a cluster address).
+template <int BN, int EPI, int HALVES, bool PAIR>
+__device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtensorMap& tm_y, uint32_t staging,
+                                              uint32_t& chunk_no, uint32_t tmem_base, int acc, uint32_t acc_phase,
+                                              uint32_t tfull_addr, uint32_t tempty_addr, volatile int* abort_flag,
+                                              int m, int n, int quarter, int half, int lane) {
+    constexpr int CPW = BN / 32 / HALVES;         // 32-column chunks per epilogue warp
+    const int row = m * BM + quarter * 32 + lane;     // m: 128-row tile index
+    const bool row_ok = row < args.rows;
+    const int n_chunks = min(BN / 32, (args.n_out - n * BN) / 32);      // even: n_out % 64 == 0
+    const int my_chunks = n_chunks / HALVES;
+    const int c0 = half * my_chunks;
+    // The residual rows of this warp's chunks are fetched before the accumulator is ready, so
+    // their latency hides behind the main loop.  (In-place use, y == residual, is safe: the
+    // same thread reads an element here and is the only one to overwrite it below.)
+    uint4 rr[EPI == EPI_RESIDUAL ? CPW : 1][4];
+    if constexpr (EPI == EPI_RESIDUAL) {
+#pragma unroll
+        for (int cc = 0; cc < CPW; ++cc) {
+            if (cc < my_chunks && row_ok) {
+                const uint4* r4 = reinterpret_cast<const uint4*>(
+                    args.residual + (size_t)row * args.n_out + n * BN + (c0 + cc) * 32);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) rr[cc][q] = r4[q];
+            } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) rr[cc][q] = make_uint4(0, 0, 0, 0);
+            }
+        }
+    }
+    bool ok = PAIR ? mbar_wait_cluster(tfull_addr, acc_phase, abort_flag, args.status)
+                   : mbar_wait(tfull_addr, acc_phase, abort_flag, args.status);
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    if (!ok) return false;
+    tc_fence_after();
+    size_t orow = (size_t)row;
+    const float* pos_row = nullptr;
+    if (EPI == EPI_PATCH && row_ok) {
+        const int p = row % args.pe.g2;
+        orow = (size_t)(row / args.pe.g2) * args.pe.tokens + 1 + p;
+        pos_row = args.pe.pos + (size_t)(1 + p) * args.n_out;
+    }
+    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll
+    for (int cc = 0; cc < CPW; ++cc) {
+        if (cc >= my_chunks) break;
+        const int c = c0 + cc;
+        const int n0 = n * BN + c * 32;
+        uint32_t v[32];
+        tmem_ld32(t_row + (uint32_t)(c * 32), v);
+        tmem_ld_wait();
+        if (cc == my_chunks - 1) {
+            // every TMEM read of this accumulator is done: hand the buffer back early
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { if (PAIR) mbar_arrive_cluster(tempty_addr); else mbar_arrive(tempty_addr); }
+        }
+        float f[32];
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+            const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
+            f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
+            f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
+            f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
+            f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+        }
+        if constexpr (EPI == EPI_GELU) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
+        } else if constexpr (EPI == EPI_RESIDUAL) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t w[4] = {rr[cc][q].x, rr[cc][q].y, rr[cc][q].z, rr[cc][q].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
+                    f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
+                }
+            }
+        } else if constexpr (EPI == EPI_PATCH) {
+            if (row_ok) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 p4 = __ldg(reinterpret_cast<const float4*>(pos_row + n0 + j));
+                    f[j + 0] += p4.x; f[j + 1] += p4.y; f[j + 2] += p4.z; f[j + 3] += p4.w;
+                }
+            }
+        }
+        uint4 o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            o[q].x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
+            o[q].y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
+            o[q].z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
+            o[q].w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
+        }
+        if (args.tma_store) {
+            // [32 rows x 64 B] block, 16-byte chunks XOR-swizzled by (row >> 1) & 3 (64B
+            // swizzle), then one TMA store; rows past the end are clipped by the tensor map
+            const uint32_t buf = staging + (chunk_no & 1u) * (32 * 64);
+            if (lane == 0) bulk_wait_read1();        // the store that last used this buffer has read it
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                st_shared_v4(buf + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4), o[q]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(&tm_y, buf, n0, m * BM + quarter * 32);
+                bulk_commit();
+            }
+            ++chunk_no;
+        } else if (row_ok) {
+            uint4* o4 = reinterpret_cast<uint4*>(args.y + orow * args.n_out + n0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) o4[q] = o[q];
+        }
+    }
+    return true;
+}
+
 template <int BN, int EPI, int EW>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
@@ -89,7 +215,6 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     using S = Smem<BN, EW>;
     constexpr int NTHREADS = 64 + 32 * EW;
     constexpr int HALVES = EW / 4;                // epilogue warps per TMEM lane quarter
-    constexpr int CPW = BN / 32 / HALVES;         // 32-column chunks per epilogue warp
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     if (base & 1023u) {                       // swizzled operands need a 1024-byte aligned window
@@ -248,116 +373,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int m = tile / args.n_tiles, n = tile % args.n_tiles;
-            const int row = m * BM + quarter * 32 + lane;
-            const bool row_ok = row < args.rows;
-            const int n_chunks = min(BN / 32, (args.n_out - n * BN) / 32);      // even: n_out % 64 == 0
-            const int my_chunks = n_chunks / HALVES;
-            const int c0 = half * my_chunks;
-            // The residual rows of this warp's chunks are fetched before the accumulator is ready, so
-            // their latency hides behind the main loop.  (In-place use, y == residual, is safe: the
-            // same thread reads an element here and is the only one to overwrite it below.)
-            uint4 rr[EPI == EPI_RESIDUAL ? CPW : 1][4];
-            if constexpr (EPI == EPI_RESIDUAL) {
-#pragma unroll
-                for (int cc = 0; cc < CPW; ++cc) {
-                    if (cc < my_chunks && row_ok) {
-                        const uint4* r4 = reinterpret_cast<const uint4*>(
-                            args.residual + (size_t)row * args.n_out + n * BN + (c0 + cc) * 32);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) rr[cc][q] = r4[q];
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) rr[cc][q] = make_uint4(0, 0, 0, 0);
-                    }
-                }
-            }
-            ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, args.status);
-            ok = __all_sync(0xFFFFFFFFu, ok);
+            ok = epilogue_tile<BN, EPI, HALVES, false>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
+                                                       tfull_bar(acc), tempty_bar(acc), abort_flag, m, n, quarter,
+                                                       half, lane);
             if (!ok) break;
-            tc_fence_after();
-            size_t orow = (size_t)row;
-            const float* pos_row = nullptr;
-            if (EPI == EPI_PATCH && row_ok) {
-                const int p = row % args.pe.g2;
-                orow = (size_t)(row / args.pe.g2) * args.pe.tokens + 1 + p;
-                pos_row = args.pe.pos + (size_t)(1 + p) * args.n_out;
-            }
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-#pragma unroll
-            for (int cc = 0; cc < CPW; ++cc) {
-                if (cc >= my_chunks) break;
-                const int c = c0 + cc;
-                const int n0 = n * BN + c * 32;
-                uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)(c * 32), v);
-                tmem_ld_wait();
-                if (cc == my_chunks - 1) {
-                    // every TMEM read of this accumulator is done: hand the buffer back early
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar(acc));
-                }
-                float f[32];
-#pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
-                    f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
-                    f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
-                    f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
-                    f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
-                }
-                if constexpr (EPI == EPI_GELU) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
-                } else if constexpr (EPI == EPI_RESIDUAL) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t w[4] = {rr[cc][q].x, rr[cc][q].y, rr[cc][q].z, rr[cc][q].w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
-                            f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
-                        }
-                    }
-                } else if constexpr (EPI == EPI_PATCH) {
-                    if (row_ok) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            const float4 p4 = __ldg(reinterpret_cast<const float4*>(pos_row + n0 + j));
-                            f[j + 0] += p4.x; f[j + 1] += p4.y; f[j + 2] += p4.z; f[j + 3] += p4.w;
-                        }
-                    }
-                }
-                uint4 o[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    o[q].x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
-                    o[q].y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
-                    o[q].z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
-                    o[q].w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
-                }
-                if (args.tma_store) {
-                    // [32 rows x 64 B] block, 16-byte chunks XOR-swizzled by (row >> 1) & 3 (64B
-                    // swizzle), then one TMA store; rows past the end are clipped by the tensor map
-                    const uint32_t buf = staging + (chunk_no & 1u) * (32 * 64);
-                    if (lane == 0) bulk_wait_read1();        // the store that last used this buffer has read it
-                    __syncwarp();
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        st_shared_v4(buf + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4), o[q]);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tm_y, buf, n0, m * BM + quarter * 32);
-                        bulk_commit();
-                    }
-                    ++chunk_no;
-                } else if (row_ok) {
-                    uint4* o4 = reinterpret_cast<uint4*>(args.y + orow * args.n_out + n0);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) o4[q] = o[q];
-                }
-            }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         if (args.tma_store && lane == 0) bulk_wait_all();
@@ -374,6 +393,228 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 2 * BN);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs (n_out a multiple of 256).  Two CTAs of a cluster share one
+// 256 x 256 output tile: each stages its own 128 rows of x (and of the t slabs) and HALF of the
+// W^T tile (and of the B slabs), so every byte of W^T crosses the L2 -> SM fabric once per 256
+// rows instead of once per 128, and one tcgen05.mma.cta_group::2 (M = 256) issued by the even
+// CTA drives the tensor cores of both SMs, each accumulating its own 128 rows in its own TMEM.
+//   full[s]    (even CTA)   bytes of both CTAs' loads of stage s (the odd CTA's TMA signals it)
+//   empty[s]   (both CTAs)  the pair MMAs that read stage s are done (multicast commit)
+//   tfull[a]   (both CTAs)  accumulator a is complete (multicast commit)
+//   tempty[a]  (even CTA)   both CTAs' epilogue warps have drained accumulator a
+// Six 32 KB stages per CTA.  No TMA multicast is used.
+// ---------------------------------------------------------------------------------------
+constexpr int P_BN = 256;
+constexpr int P_EW = 8;
+constexpr int P_STAGES = 6;
+constexpr int P_A_BYTES = BM * BK * 2;                 // 16 KB: this CTA's 128 rows of x
+constexpr int P_B_BYTES = (P_BN / 2) * BK * 2;         // 16 KB: this CTA's half of the W^T tile
+constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES;
+constexpr int P_T_SLAB_BYTES = BM * PM_SLAB * 2;       // 4 KB
+constexpr int P_B_SLAB_BYTES = (P_BN / 2) * PM_SLAB * 2;   // 4 KB
+constexpr int P_STAGING_OFFSET = P_STAGES * P_STAGE_BYTES;
+constexpr int P_PLAN_OFFSET = P_STAGING_OFFSET + P_EW * STAGING_BYTES_PER_WARP;
+constexpr int P_BAR_OFFSET = P_PLAN_OFFSET + PLAN_BYTES;
+constexpr int P_SMEM_TOTAL = P_BAR_OFFSET + 256;
+constexpr int P_THREADS = 64 + 32 * P_EW;
+
+template <int EPI>
+__global__ void __launch_bounds__(P_THREADS, 1)
+lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                      const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
+                      const __grid_constant__ CUtensorMap tm_y, const GemmArgs args) {
+    constexpr int BN = P_BN;
+    constexpr int HALVES = P_EW / 4;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs, 1: its peer
+    uint8_t* smem = smem_raw;
+    const uint32_t bars = base + P_BAR_OFFSET;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (P_STAGES + s); };
+    auto tfull_bar = [&](int s) { return bars + 8u * (2 * P_STAGES + s); };
+    auto tempty_bar = [&](int s) { return bars + 8u * (2 * P_STAGES + 2 + s); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + P_BAR_OFFSET + 8 * (2 * P_STAGES + 4));
+    // the peer CTA's TMEM base: written only by the peer (any time before the cluster barrier below),
+    // never by this CTA, so there is no ordering to get wrong
+    volatile uint32_t* peer_slot = tmem_slot + 1;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + P_BAR_OFFSET + 8 * (2 * P_STAGES + 4) + 8);
+    int* plan = reinterpret_cast<int*>(smem + P_PLAN_OFFSET);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int total_tiles = args.m_tiles * args.n_tiles;      // m_tiles counts 256-row tiles here
+    const int num_kb = args.k_in / BK;
+
+    // LoRA plan of this CTA's tiles (both halves of a 256-row tile carry the same slab list)
+    const int plan_stride = 1 + args.slab_cap;
+    const int plan_tiles = args.tile_nslabs ? PLAN_BYTES / (4 * plan_stride) : 0;
+    if (args.tile_nslabs) {
+        for (int i = threadIdx.x / 8; i < plan_tiles; i += P_THREADS / 8) {
+            const int tile = pair_id + i * n_pairs;
+            if (tile >= total_tiles) break;
+            const int m = 2 * (tile / args.n_tiles) + (int)rank;
+            const int ns = args.tile_nslabs[m];
+            if ((threadIdx.x & 7) == 0) plan[i * plan_stride] = ns;
+            for (int q = threadIdx.x & 7; q < ns; q += 8) plan[i * plan_stride + 1 + q] = args.tile_slab[m * args.slab_cap + q];
+        }
+    }
+    auto tile_ns = [&](int it, int m) -> int {
+        if (!args.tile_nslabs) return 0;
+        return it < plan_tiles ? plan[it * plan_stride] : args.tile_nslabs[m];
+    };
+    auto tile_slab_id = [&](int it, int m, int q) -> int {
+        return it < plan_tiles ? plan[it * plan_stride + 1 + q] : args.tile_slab[m * args.slab_cap + q];
+    };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 2 * P_EW); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), 512);     // all of this SM's tensor memory
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // both CTAs must hold the same TMEM columns (the pair MMA uses one address for both); tell the peer
+    if (threadIdx.x == 0) st_cluster_u32(mapa_cluster(smem_u32((const void*)peer_slot), rank ^ 1u), tmem_base);
+    cluster_sync_all();          // barriers initialised and TMEM bases exchanged in both CTAs
+    const bool usable = ((base & 1023u) == 0) && (*peer_slot == tmem_base);
+    if (!usable && threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
+
+    if (!usable) {
+        // fall through to the teardown
+    } else if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++it) {
+                const int m2 = tile / args.n_tiles, n = tile % args.n_tiles;
+                const int m = 2 * m2 + (int)rank;                   // this CTA's 128-row tile
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait_cluster(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    const uint32_t fb = mapa_cluster(full_bar(stage), 0);
+                    if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * P_STAGE_BYTES);
+                    const uint32_t sa = base + stage * P_STAGE_BYTES;
+                    tma_load_2d_pair(sa, &tm_x, kb * BK, m * BM, fb);
+                    tma_load_2d_pair(sa + P_A_BYTES, &tm_w, kb * BK, n * BN + (int)rank * (BN / 2), fb);
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                const int ns = tile_ns(it, m);
+                for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
+                    const int cnt = min(SLABS_PER_STAGE, ns - g0);
+                    ok = mbar_wait_cluster(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    const uint32_t fb = mapa_cluster(full_bar(stage), 0);
+                    if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * cnt * (P_T_SLAB_BYTES + P_B_SLAB_BYTES));
+                    const uint32_t sa = base + stage * P_STAGE_BYTES;
+                    for (int i = 0; i < cnt; ++i) {
+                        const int slot = m * args.slab_cap + g0 + i;
+                        const int slab = tile_slab_id(it, m, g0 + i);
+                        tma_load_2d_pair(sa + i * P_T_SLAB_BYTES, &tm_t, 0, slot * BM, fb);
+                        tma_load_2d_pair(sa + P_A_BYTES + i * P_B_SLAB_BYTES, &tm_bt, 0,
+                                         slab * args.n_out + n * BN + (int)rank * (BN / 2), fb);
+                    }
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (even CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_pair(BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++it) {
+                const int m = 2 * (tile / args.n_tiles);
+                const int ns = tile_ns(it, m);
+                ok = mbar_wait_cluster(tempty_bar(acc), acc_phase ^ 1u, abort_flag, args.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                uint32_t accumulate = 0;
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * P_STAGE_BYTES;
+                    const uint32_t sb = sa + P_A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        umma_bf16_pair(d_tmem, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
+                                       accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit_pair(empty_bar(stage));
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
+                    const int cnt = min(SLABS_PER_STAGE, ns - g0);
+                    ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * P_STAGE_BYTES;
+                    const uint32_t sb = sa + P_A_BYTES;
+                    for (int i = 0; i < cnt; ++i) {
+                        umma_bf16_pair(d_tmem, smem_desc(sa + i * P_T_SLAB_BYTES, 32),
+                                       smem_desc(sb + i * P_B_SLAB_BYTES, 32), idesc, accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit_pair(empty_bar(stage));
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit_pair(tfull_bar(acc));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (both CTAs)
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const uint32_t staging = base + P_STAGING_OFFSET + (uint32_t)(warp - 2) * STAGING_BYTES_PER_WARP;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        uint32_t chunk_no = 0;
+        bool ok = true;
+        for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
+            const int m = 2 * (tile / args.n_tiles) + (int)rank, n = tile % args.n_tiles;
+            ok = epilogue_tile<BN, EPI, HALVES, true>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
+                                                      tfull_bar(acc), mapa_cluster(tempty_bar(acc), 0), abort_flag,
+                                                      m, n, quarter, half, lane);
+            if (!ok) break;
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (args.tma_store && lane == 0) bulk_wait_all();
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);    // let copies / MMAs in flight land
+    }
+    tc_fence_before();
+    cluster_sync_all();          // the peer no longer reads this CTA's shared memory or signals its barriers
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
@@ -615,7 +856,8 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
     ShrinkArgs a;
     a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap; a.n_tiles = R.n_tiles;
-    a.sg = R.slab_cap < 16 ? R.slab_cap : 16;
+    // groups of at most 8 slabs: two 128-column accumulators per CTA, so two CTAs share an SM's TMEM
+    a.sg = R.slab_cap < 8 ? R.slab_cap : 8;
     uint32_t cols = 32;
     while ((int)cols < a.sg * PM_SLAB) cols <<= 1;
     a.acc_cols = cols;                                   // two buffers: at most 2 x 256 columns
@@ -676,7 +918,48 @@ static cudaError_t launch_gemm_epi(const Launch& L, const CUtensorMap& tm_x, con
     }
 }
 
-// lin.tm_w / lin.tm_bt are encoded for the BN chosen by gemm_tile_n(lin.n_out).
+template <int EPI>
+static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
+                                    const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
+                                    const GemmArgs& a, int n_sms) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             P_SMEM_TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int total = a.m_tiles * a.n_tiles;
+    const int pairs = total < n_sms / 2 ? total : n_sms / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(P_THREADS);
+    cfg.dynamicSmemBytes = P_SMEM_TOTAL;
+    cfg.stream = L.st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ProfScope ps(L, KC_GEMM);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_pair_kernel<EPI>, tm_x, tm_w, tm_t, tm_bt, tm_y, a);
+    BUMP(L);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+static cudaError_t launch_gemm_pair_epi(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
+                                        const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
+                                        const GemmArgs& a, int n_sms) {
+    switch (a.epi) {
+        case EPI_GELU: return launch_gemm_pair<EPI_GELU>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        case EPI_RESIDUAL: return launch_gemm_pair<EPI_RESIDUAL>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        case EPI_PATCH: return launch_gemm_pair<EPI_PATCH>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        default: return launch_gemm_pair<EPI_NONE>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+    }
+}
+
+// lin.tm_w / lin.tm_bt are encoded for the BN chosen by gemm_tile_n(lin.n_out); lin.tm_w_half /
+// lin.tm_bt_half (n_out a multiple of 256) fetch 128 of a tile's 256 columns for the pair kernel.
 int gemm_tile_n(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
 
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
@@ -697,8 +980,13 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
     a.status = L.status;
     a.tma_store = (tm_y != nullptr && epi != EPI_PATCH) ? 1 : 0;
     const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced
-    const CUtensorMap& tb = lora ? lin.tm_bt : lin.tm_w;
     const CUtensorMap& ty = a.tma_store ? *tm_y : tm_x;
+    if (lin.has_tm_half && n_sms >= 2) {
+        a.m_tiles = (rows + 2 * BM - 1) / (2 * BM);       // 256-row tiles
+        a.n_tiles = lin.n_out / P_BN;
+        return launch_gemm_pair_epi(L, tm_x, lin.tm_w_half, tt, lora ? lin.tm_bt_half : lin.tm_w_half, ty, a, n_sms);
+    }
+    const CUtensorMap& tb = lora ? lin.tm_bt : lin.tm_w;
     if (bn == 256) return launch_gemm_epi<256>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
     return launch_gemm_epi<128>(L, tm_x, lin.tm_w, tt, tb, ty, a, n_sms);
 }
