@@ -314,6 +314,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = instr_desc(BN);
+            // Descriptors of stage 0; a stage adds STAGE_BYTES / 16 and a K step of 16 adds 2 to the
+            // address field.  Keeping the issuing thread's work per K block to a handful of
+            // instructions matters: the tensor pipe runs dry whenever this thread is late.
+            const uint64_t da0 = smem_desc(base, 128), db0 = smem_desc(base + S::A_BYTES, 128);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -332,12 +336,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = base + stage * S::STAGE_BYTES;
-                    const uint32_t sb = sa + S::A_BYTES;
+                    const uint64_t so = (uint64_t)(stage * (S::STAGE_BYTES >> 4));
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
-                        umma_bf16(d_tmem, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
-                                  accumulate);
+                        umma_bf16(d_tmem, da0 + so + 2 * k, db0 + so + 2 * k, idesc, accumulate);
                         accumulate = 1;
                     }
                     umma_commit(empty_bar(stage));
@@ -537,6 +539,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = instr_desc_pair(BN);
+            const uint64_t da0 = smem_desc(base, 128), db0 = smem_desc(base + P_A_BYTES, 128);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -555,12 +558,10 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, args.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = base + stage * P_STAGE_BYTES;
-                    const uint32_t sb = sa + P_A_BYTES;
+                    const uint64_t so = (uint64_t)(stage * (P_STAGE_BYTES >> 4));
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
-                        umma_bf16_pair(d_tmem, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
-                                       accumulate);
+                        umma_bf16_pair(d_tmem, da0 + so + 2 * k, db0 + so + 2 * k, idesc, accumulate);
                         accumulate = 1;
                     }
                     umma_commit_pair(empty_bar(stage));

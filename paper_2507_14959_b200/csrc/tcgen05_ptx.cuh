@@ -35,8 +35,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait.  Returns false once the CTA is aborting.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* status) {
+    if (mbar_try_wait(bar, parity)) return true;        // fast path: nothing else on it
     if (*abort_flag) return false;
-    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return false;
@@ -216,8 +216,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t
 // bounded wait on a local mbarrier whose arrivals come from both CTAs of the pair
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   int* status) {
-    if (*abort_flag) return false;
     if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
     const long long t0 = clock64();
     while (!mbar_try_wait_cluster(bar, parity)) {
         if (*abort_flag) return false;
