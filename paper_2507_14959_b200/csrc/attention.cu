@@ -324,6 +324,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (lane == 0) {
             // ------------------------------------------------------ TMA + MMA issue
             const uint32_t idesc_pv = instr_desc_b_mn(HD);
+            // descriptors built once; a K step adds 2 (32 B) for Q / K and 128 (2048 B) for V
+            const uint64_t dq0 = smem_desc(q_s, 128), dk0 = smem_desc(k_s, 128), dv0 = smem_desc(v_s, 128);
             uint32_t step = 0;
             bool ok = true;
             for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
@@ -336,9 +338,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         const int nb = min(AKB, args.tpad - b * AKB);
                         const uint32_t idesc_s = instr_desc(nb);
 #pragma unroll
+                        const uint64_t bo = (uint64_t)((b * AKB_BYTES) >> 4);
+#pragma unroll
                         for (int k = 0; k < HD / 16; ++k)
-                            umma_bf16(tmem_base, smem_desc(q_s + k * 32, 128),
-                                      smem_desc(k_s + b * AKB_BYTES + k * 32, 128), idesc_s, k > 0);
+                            umma_bf16(tmem_base, dq0 + 2 * k, dk0 + bo + 2 * k, idesc_s, k > 0);
                         umma_commit(s_bar);
                         ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
                         ++step;
@@ -352,8 +355,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                 tma_load_2d(q_s, &tm_q, h * HD, f * T + (qt + 1) * AQ, q_bar);
                             }
                             for (int kk = 0; kk < nb / 16; ++kk)
-                                umma_bf16_ts(o_tmem, tmem_base + (uint32_t)(kk * 8),
-                                             smem_desc(v_s + b * AKB_BYTES + kk * 2048, 128), idesc_pv,
+                                umma_bf16_ts(o_tmem, tmem_base + (uint32_t)(kk * 8), dv0 + bo + 128 * kk, idesc_pv,
                                              (b > 0 || kk > 0) ? 1u : 0u);
                             umma_commit(s_bar);
                             ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);

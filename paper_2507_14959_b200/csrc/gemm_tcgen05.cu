@@ -713,6 +713,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     } else if (warp == 1) {
         if (lane == 0) {
             // -------------------------------------------------------------- MMA issuer
+            const uint64_t da0 = smem_desc(base, 128), db0 = smem_desc(base + SHRINK_X_BYTES, 128);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -730,12 +731,10 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                         ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t sa = base + stage * stage_bytes;
-                        const uint32_t sb = sa + SHRINK_X_BYTES;
+                        const uint64_t so = (uint64_t)((stage * stage_bytes) >> 4);
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k) {
-                            umma_bf16(d_tmem, smem_desc(sa + k * 32, 128), smem_desc(sb + k * 32, 128), idesc,
-                                      accumulate);
+                            umma_bf16(d_tmem, da0 + so + 2 * k, db0 + so + 2 * k, idesc, accumulate);
                             accumulate = 1;
                         }
                         umma_commit(empty_bar(stage));
