@@ -64,16 +64,38 @@ size_t esize(int dtype) { return dtype == 0 ? 2 : 4; }
 // One linear with its LoRA arenas.
 struct LinearObj {
     LinearDev dev;
-    DevBuf wt, bias, at, bt;
+    DevBuf wt, bias, at, bt, lng, lnc1, lnc2;
     int slabs_max = 0, max_adapters = 0, dtype = 0;
+    std::vector<float> ln_gamma, ln_beta;      // non-empty: the LayerNorm in front of this linear is folded in
 
+    // ln_g / ln_b (host [k_in], bf16 build only): fold LN(x) = (x - mean) rstd gamma + beta into the linear:
+    //   W' = gamma o W (then rounded to bf16), g[n] = sum_k W'[k,n] over the ROUNDED values (what the
+    //   tensor cores multiply), b' = b + beta W.
     int init(int k_in, int n_out, const float* w, const float* b, int max_adapters_, int slabs_max_,
-             int dtype_, std::string& err) {
+             int dtype_, std::string& err, const float* ln_g = nullptr, const float* ln_b = nullptr) {
         dev.k_in = k_in; dev.n_out = n_out;
         slabs_max = slabs_max_; max_adapters = max_adapters_; dtype = dtype_;
-        if (dtype == 0) CK(upload_transposed<bf16>(wt, w, k_in, n_out));
-        else CK(upload_transposed<float>(wt, w, k_in, n_out));
-        CK(upload<float>(bias, b, n_out));
+        if (dtype == 0 && ln_g && ln_b) {
+            ln_gamma.assign(ln_g, ln_g + k_in); ln_beta.assign(ln_b, ln_b + k_in);
+            std::vector<float> wf((size_t)k_in * n_out), bf(n_out), gs(n_out);
+            std::vector<double> gsum(n_out, 0.0), bsum(n_out, 0.0);
+            for (int k = 0; k < k_in; ++k)
+                for (int n = 0; n < n_out; ++n) {
+                    const float v = __bfloat162float(__float2bfloat16_rn(ln_g[k] * w[(size_t)k * n_out + n]));
+                    wf[(size_t)k * n_out + n] = v;
+                    gsum[n] += v;
+                    bsum[n] += (double)ln_b[k] * w[(size_t)k * n_out + n];
+                }
+            for (int n = 0; n < n_out; ++n) { gs[n] = (float)gsum[n]; bf[n] = (float)(b[n] + bsum[n]); }
+            CK(upload_transposed<bf16>(wt, wf.data(), k_in, n_out));
+            CK(upload<float>(bias, bf.data(), n_out));
+            CK(upload<float>(lng, gs.data(), n_out));
+            dev.ln_g = lng.as<float>();
+        } else {
+            if (dtype == 0) CK(upload_transposed<bf16>(wt, w, k_in, n_out));
+            else CK(upload_transposed<float>(wt, w, k_in, n_out));
+            CK(upload<float>(bias, b, n_out));
+        }
         dev.Wt = wt.p; dev.bias = bias.as<float>();
         if (max_adapters > 0 && slabs_max > 0) {
             const size_t RS = (size_t)slabs_max * PM_SLAB;
@@ -82,6 +104,13 @@ struct LinearObj {
             CK(cudaMemset(at.p, 0, at.bytes));
             CK(cudaMemset(bt.p, 0, bt.bytes));
             dev.lora.At = at.p; dev.lora.Bt = bt.p;
+            if (dev.ln_g) {
+                CK(lnc1.alloc((size_t)max_adapters * RS * sizeof(float)));
+                CK(lnc2.alloc((size_t)max_adapters * RS * sizeof(float)));
+                CK(cudaMemset(lnc1.p, 0, lnc1.bytes));
+                CK(cudaMemset(lnc2.p, 0, lnc2.bytes));
+                dev.ln_c1 = lnc1.as<float>(); dev.ln_c2 = lnc2.as<float>();
+            }
         }
         if (dtype == 0) {
             const int bn = gemm_tile_n(n_out);
@@ -113,9 +142,18 @@ struct LinearObj {
         const int k_in = dev.k_in, n_out = dev.n_out;
         const size_t RS = (size_t)slabs_max * PM_SLAB;
         std::vector<T> ha(RS * k_in, host_cvt<T>(0.f)), hb(RS * n_out, host_cvt<T>(0.f));
+        std::vector<float> c1(RS, 0.f), c2(RS, 0.f);
         if (A && B) {
+            const bool fold = dev.ln_g != nullptr;
+            std::vector<double> s1(rank, 0.0), s2(rank, 0.0);
             for (int k = 0; k < k_in; ++k)
-                for (int j = 0; j < rank; ++j) ha[(size_t)j * k_in + k] = host_cvt<T>(A[(size_t)k * rank + j]);
+                for (int j = 0; j < rank; ++j) {
+                    const float a0 = A[(size_t)k * rank + j];
+                    const T av = host_cvt<T>(fold ? ln_gamma[k] * a0 : a0);
+                    ha[(size_t)j * k_in + k] = av;
+                    if (fold) { s1[j] += (double)(float)av; s2[j] += (double)ln_beta[k] * a0; }
+                }
+            for (int j = 0; j < rank && fold; ++j) { c1[j] = (float)s1[j]; c2[j] = (float)s2[j]; }
             for (int j = 0; j < rank; ++j)
                 for (int n = 0; n < n_out; ++n)
                     hb[((size_t)(j / PM_SLAB) * n_out + n) * PM_SLAB + (j % PM_SLAB)] =
@@ -123,6 +161,10 @@ struct LinearObj {
         }
         CK(cudaMemcpy(at.as<T>() + (size_t)a * RS * k_in, ha.data(), ha.size() * sizeof(T), cudaMemcpyHostToDevice));
         CK(cudaMemcpy(bt.as<T>() + (size_t)a * RS * n_out, hb.data(), hb.size() * sizeof(T), cudaMemcpyHostToDevice));
+        if (dev.ln_g) {
+            CK(cudaMemcpy(lnc1.as<float>() + (size_t)a * RS, c1.data(), RS * sizeof(float), cudaMemcpyHostToDevice));
+            CK(cudaMemcpy(lnc2.as<float>() + (size_t)a * RS, c2.data(), RS * sizeof(float), cudaMemcpyHostToDevice));
+        }
         return PM_OK;
     }
     int set_adapter(int a, int rank, const float* A, const float* B, std::string& err) {
@@ -317,8 +359,8 @@ struct pm_handle_s {
     std::vector<LinearObj> lin;              // [layers*4]
     DevBuf cls, pos, ln1_g, ln1_b, ln2_g, ln2_b, lnf_g, lnf_b, head_wt, head_b;
     // activations
-    DevBuf X, U, QKV, ATT, H, PATCH, Z, t32, tbuf, status;
-    CUtensorMap tm_patch, tm_u, tm_att, tm_h, tm_t;
+    DevBuf X, U, QKV, ATT, H, PATCH, Z, t32, tbuf, status, ln_stats;
+    CUtensorMap tm_patch, tm_u, tm_att, tm_h, tm_t, tm_x_in;
     CUtensorMap tm_y_qkv, tm_y_x, tm_y_h;      // outputs, for the TMA-store epilogue
     CUtensorMap tm_att_q, tm_att_kv;           // attention operands over QKV
     int tm_rows = -1;
@@ -388,6 +430,7 @@ int encode_activation_maps(pm_handle_s* h, int rows) {
     const int prow = rows / h->tokens * h->g2;
     bool ok = tm_encode_2d(&h->tm_patch, h->PATCH.p, h->patch_dim, prow, (uint64_t)h->patch_dim * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_u, h->U.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
+           && tm_encode_2d(&h->tm_x_in, h->X.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_att, h->ATT.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_y_qkv, h->QKV.p, 3 * d, rows, (uint64_t)3 * d * 2, 32, 32, 64)
@@ -415,19 +458,20 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     T* X = h->X.as<T>(); T* U = h->U.as<T>(); T* QKV = h->QKV.as<T>(); T* ATT = h->ATT.as<T>();
     T* Hb = h->H.as<T>(); T* P = h->PATCH.as<T>();
 
+    // st: per-row LayerNorm statistics of x when the linear has its LayerNorm folded in, else null
     auto linear = [&](LinearObj& lo, const T* x, const CUtensorMap* tmx, int nrows, int tokens_pf, bool lora,
-                      int epi, const T* residual, const PatchEpi& pep, T* y) -> cudaError_t {
+                      int epi, const T* residual, const PatchEpi& pep, T* y, const float2* st = nullptr) -> cudaError_t {
         if constexpr (TC) {
             const bool use_lora = lora && R.max_set > 0;
             if (use_lora) {
-                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>(), h->n_sms);
+                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>(), h->n_sms, st);
                 if (e != cudaSuccess) return e;
             }
             const CUtensorMap* tmy = (void*)y == h->QKV.p ? &h->tm_y_qkv
                                    : (void*)y == h->H.p ? &h->tm_y_h
                                    : (void*)y == h->X.p ? &h->tm_y_x : nullptr;
             return launch_lora_gemm(L, lo.dev, use_lora ? &R : nullptr, *tmx, &h->tm_t, tmy, nrows, epi,
-                                    (const bf16*)residual, pep, (bf16*)y, h->n_sms);
+                                    (const bf16*)residual, pep, (bf16*)y, h->n_sms, st);
         } else {
             return launch_naive_linear<T>(L, lo.dev, R, h->meta, h->slabs_max, x, nrows, tokens_pf,
                                           lora ? h->t32.as<float>() : nullptr, epi, residual, pep, y);
@@ -438,8 +482,14 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     CK(linear(h->patch, P, &h->tm_patch, n_frames * h->g2, h->g2, false, EPI_PATCH, nullptr, pe, X));
     CK(launch_cls_rows<T>(L, h->cls.as<float>(), h->pos.as<float>(), X, n_frames, T_, d));
     for (int l = 0; l < c.layers; ++l) {
-        CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
-        CK(linear(h->lin[l * 4 + 0], U, &h->tm_u, rows, T_, true, EPI_NONE, nullptr, none, QKV));
+        if constexpr (TC) {
+            // LayerNorm 1 is folded into the qkv weights: only the row statistics are computed
+            CK(launch_row_stats(L, (const bf16*)X, h->ln_stats.as<float2>(), rows, d, c.ln_eps));
+            CK(linear(h->lin[l * 4 + 0], X, &h->tm_x_in, rows, T_, true, EPI_NONE, nullptr, none, QKV, h->ln_stats.as<float2>()));
+        } else {
+            CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
+            CK(linear(h->lin[l * 4 + 0], U, &h->tm_u, rows, T_, true, EPI_NONE, nullptr, none, QKV));
+        }
         if constexpr (TC) {
             if (attention_tc_supported(T_))
                 CK(launch_attention_tc(L, h->tm_att_q, h->tm_att_kv, (bf16*)ATT, n_frames, T_, c.heads));
@@ -448,8 +498,13 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
         }
         else CK(launch_attention_simple<T>(L, QKV, ATT, n_frames, T_, c.heads));
         CK(linear(h->lin[l * 4 + 1], ATT, &h->tm_att, rows, T_, true, EPI_RESIDUAL, X, none, X));
-        CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
-        CK(linear(h->lin[l * 4 + 2], U, &h->tm_u, rows, T_, true, EPI_GELU, nullptr, none, Hb));
+        if constexpr (TC) {
+            CK(launch_row_stats(L, (const bf16*)X, h->ln_stats.as<float2>(), rows, d, c.ln_eps));
+            CK(linear(h->lin[l * 4 + 2], X, &h->tm_x_in, rows, T_, true, EPI_GELU, nullptr, none, Hb, h->ln_stats.as<float2>()));
+        } else {
+            CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
+            CK(linear(h->lin[l * 4 + 2], U, &h->tm_u, rows, T_, true, EPI_GELU, nullptr, none, Hb));
+        }
         CK(linear(h->lin[l * 4 + 3], Hb, &h->tm_h, rows, T_, true, EPI_RESIDUAL, X, none, X));
     }
     CK(launch_heads<T>(L, X, n_frames, T_, d, c.ln_eps, h->lnf_g.as<float>(), h->lnf_b.as<float>(),
@@ -474,7 +529,10 @@ int create_t(pm_handle_s* h, const pm_backbone* w) {
                               w->fc1_b + (size_t)l * m, w->fc2_b + (size_t)l * d};
         const int kin[4] = {d, d, d, m}, nout[4] = {3 * d, d, m, d};
         for (int p = 0; p < 4; ++p) {
-            rc = h->lin[l * 4 + p].init(kin[p], nout[p], ws[p], bs[p], c.max_adapters, h->slabs_max, c.dtype, err);
+            // qkv follows LayerNorm 1 and fc1 follows LayerNorm 2: folded into their weights (bf16 build)
+            const float* lg = p == 0 ? w->ln1_g + (size_t)l * d : p == 2 ? w->ln2_g + (size_t)l * d : nullptr;
+            const float* lb = p == 0 ? w->ln1_b + (size_t)l * d : p == 2 ? w->ln2_b + (size_t)l * d : nullptr;
+            rc = h->lin[l * 4 + p].init(kin[p], nout[p], ws[p], bs[p], c.max_adapters, h->slabs_max, c.dtype, err, lg, lb);
             if (rc) return rc;
         }
     }
@@ -492,6 +550,7 @@ int create_t(pm_handle_s* h, const pm_backbone* w) {
     CK(h->H.alloc(rows_pad * m * sizeof(T)));
     CK(h->PATCH.alloc(rows_pad * h->patch_dim * sizeof(T)));
     CK(h->Z.alloc((size_t)c.max_frames * d * sizeof(float)));
+    CK(h->ln_stats.alloc(rows_pad * sizeof(float2)));
     CK(cudaMemset(h->X.p, 0, h->X.bytes)); CK(cudaMemset(h->U.p, 0, h->U.bytes));
     CK(cudaMemset(h->QKV.p, 0, h->QKV.bytes)); CK(cudaMemset(h->ATT.p, 0, h->ATT.bytes));
     CK(cudaMemset(h->H.p, 0, h->H.bytes)); CK(cudaMemset(h->PATCH.p, 0, h->PATCH.bytes));
@@ -797,9 +856,9 @@ int pm_linear_forward(pm_linear l, const void* x, int n_frames, const int32_t* s
             err = "cuTensorMapEncodeTiled failed (y); y must be 16-byte aligned"; return PM_ERR_CUDA;
         }
         const bool lora = R.max_set > 0 && l->lin.dev.lora.At != nullptr;
-        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>(), l->n_sms));
+        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>(), l->n_sms, nullptr));
         CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, &tm_y, rows, l->epilogue,
-                            (const bf16*)residual, none, (bf16*)y, l->n_sms));
+                            (const bf16*)residual, none, (bf16*)y, l->n_sms, nullptr));
     } else {
         CK(launch_naive_linear<float>(L, l->lin.dev, R, l->meta, l->slabs_max, (const float*)x, rows, l->tokens,
                                       l->t32.as<float>(), l->epilogue, (const float*)residual, none, (float*)y));

@@ -38,6 +38,13 @@ struct LinearDev {
     // n_out a multiple of 256: boxes of 128 output columns for the CTA-pair GEMM
     CUtensorMap tm_w_half, tm_bt_half;
     bool has_tm_half = false;
+    // LayerNorm folded into this linear (its input is the raw residual stream x, not LN(x)):
+    //   LN(x) W + b = rstd (x W' - mu g) + b',  W' = gamma o W,  g[n] = sum_k W'[k,n],  b' = b + beta W
+    // Wt / bias above then hold W' / b'; the LoRA arena holds A' = gamma o A and, per arena rank j,
+    //   ln_c1[j] = sum_k A'[k,j],  ln_c2[j] = sum_k beta[k] A[k,j].
+    const float* ln_g = nullptr;       // [n_out], null = not folded
+    const float* ln_c1 = nullptr;      // [max_adapters * RS]
+    const float* ln_c2 = nullptr;
 };
 
 // Per-batch routing of frames to adapters, in SLOT order (slot = position after bucketing
@@ -135,14 +142,17 @@ cudaError_t launch_naive_linear(const Launch& L, const LinearDev& lin, const Rou
                                 int tokens_per_frame, float* t32, int epi, const T* residual,
                                 const PatchEpi& pe, T* y);
 // tensor-core path (bf16): shrink into the slab buffer, then the fused GEMM
+// ln_stats: per-row (mean, 1/sqrt(var + eps)) of x, required iff lin.ln_g != null
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf, int n_sms);
+                          const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf, int n_sms,
+                          const float2* ln_stats);
+cudaError_t launch_row_stats(const Launch& L, const bf16* x, float2* stats, int rows, int d, float eps);
 // tm_y: [rows, n_out] output map with a (32 x 32) box and 64B swizzle for the TMA-store epilogue, or
 // null to store straight from registers (always the case for EPI_PATCH, whose rows are remapped)
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
                              const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
                              int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
-                             int n_sms);
+                             int n_sms, const float2* ln_stats);
 template <typename T>
 cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, int d, float eps,
                          const float* lnf_g, const float* lnf_b, float* z,

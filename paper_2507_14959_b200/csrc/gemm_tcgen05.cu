@@ -64,6 +64,9 @@ struct GemmArgs {
     int slab_cap;
     int tma_store;             // 1: the epilogue stores through shared memory + TMA (tm_y valid)
     int* status;
+    // LayerNorm folded into the linear (LNF kernels): y = rstd (acc - mean g) + bias, per row / column
+    const float* ln_g;
+    const float2* ln_stats;
 };
 
 constexpr int STAGING_BYTES_PER_WARP = 2 * 32 * 64;     // two [32 rows x 32 bf16] buffers
@@ -87,7 +90,7 @@ struct Smem {
 // chunks goes TMEM -> registers -> bias / GELU / residual / patch placement -> bf16 -> shared
 // memory -> TMA store (or straight to global memory).  Returns false once the CTA is aborting.
 // PAIR: the accumulator-free barrier lives in the even CTA of a pair (tempty_addr is a cluster address).
-template <int BN, int EPI, int HALVES, bool PAIR>
+template <int BN, int EPI, int HALVES, bool PAIR, bool LNF>
 __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtensorMap& tm_y, uint32_t staging,
                                               uint32_t& chunk_no, uint32_t tmem_base, int acc, uint32_t acc_phase,
                                               uint32_t tfull_addr, uint32_t tempty_addr, volatile int* abort_flag,
@@ -129,6 +132,8 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
         pos_row = args.pe.pos + (size_t)(1 + p) * args.n_out;
     }
     const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+    float2 st = make_float2(0.f, 1.f);                 // (mean, rstd) of this thread's row
+    if (LNF && row_ok) st = args.ln_stats[row];
 #pragma unroll
     for (int cc = 0; cc < CPW; ++cc) {
         if (cc >= my_chunks) break;
@@ -147,10 +152,18 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
             const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
-            f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
-            f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
-            f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
-            f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+            if constexpr (LNF) {
+                const float4 g4 = __ldg(reinterpret_cast<const float4*>(args.ln_g + n0 + j));
+                f[j + 0] = fmaf(st.y, fmaf(-st.x, g4.x, __uint_as_float(v[j + 0])), b4.x);
+                f[j + 1] = fmaf(st.y, fmaf(-st.x, g4.y, __uint_as_float(v[j + 1])), b4.y);
+                f[j + 2] = fmaf(st.y, fmaf(-st.x, g4.z, __uint_as_float(v[j + 2])), b4.z);
+                f[j + 3] = fmaf(st.y, fmaf(-st.x, g4.w, __uint_as_float(v[j + 3])), b4.w);
+            } else {
+                f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
+                f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
+                f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
+                f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+            }
         }
         if constexpr (EPI == EPI_GELU) {
 #pragma unroll
@@ -207,7 +220,7 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
     return true;
 }
 
-template <int BN, int EPI, int EW>
+template <int BN, int EPI, int EW, bool LNF>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                  const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
@@ -375,7 +388,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int m = tile / args.n_tiles, n = tile % args.n_tiles;
-            ok = epilogue_tile<BN, EPI, HALVES, false>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
+            ok = epilogue_tile<BN, EPI, HALVES, false, LNF>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
                                                        tfull_bar(acc), tempty_bar(acc), abort_flag, m, n, quarter,
                                                        half, lane);
             if (!ok) break;
@@ -424,7 +437,7 @@ constexpr int P_BAR_OFFSET = P_PLAN_OFFSET + PLAN_BYTES;
 constexpr int P_SMEM_TOTAL = P_BAR_OFFSET + 256;
 constexpr int P_THREADS = 64 + 32 * P_EW;
 
-template <int EPI>
+template <int EPI, bool LNF>
 __global__ void __launch_bounds__(P_THREADS, 1)
 lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                       const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
@@ -597,7 +610,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         bool ok = true;
         for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
             const int m = 2 * (tile / args.n_tiles) + (int)rank, n = tile % args.n_tiles;
-            ok = epilogue_tile<BN, EPI, HALVES, true>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
+            ok = epilogue_tile<BN, EPI, HALVES, true, LNF>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
                                                       tfull_bar(acc), mapa_cluster(tempty_bar(acc), 0), abort_flag,
                                                       m, n, quarter, half, lane);
             if (!ok) break;
@@ -639,6 +652,12 @@ struct ShrinkArgs {
     const uint32_t* tile_mask;
     bf16* tbuf;
     int* status;
+    // LayerNorm folded into the adapters (x is the raw residual stream, the arena holds gamma o A):
+    //   t = s (rstd (x A' - mean c1) + c2);  stored divided by rstd, because the fused GEMM applies
+    //   rstd to its whole accumulator, base and LoRA part alike
+    const float2* ln_stats;     // null = not folded
+    const float* ln_c1;
+    const float* ln_c2;
 };
 
 constexpr int SHRINK_MAX_STAGES = 4;
@@ -761,6 +780,12 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * args.acc_cols;
+                float mean = 0.f, inv_rstd = 0.f;
+                if (args.ln_stats && tile * BM + r < args.rows) {
+                    const float2 st = args.ln_stats[tile * BM + r];
+                    mean = st.x;
+                    inv_rstd = 1.f / st.y;
+                }
                 for (int i = 0; i < cnt; ++i) {
                     const int slot = tile * args.slab_cap + g0 + i;
                     uint32_t v[16];
@@ -768,6 +793,14 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     tmem_ld_wait();
                     const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
                     const float sc = on ? args.tile_scale[slot] : 0.f;
+                    if (args.ln_stats) {
+                        const float* c1 = args.ln_c1 + (size_t)args.tile_slab[slot] * PM_SLAB;
+                        const float* c2 = args.ln_c2 + (size_t)args.tile_slab[slot] * PM_SLAB;
+#pragma unroll
+                        for (int j = 0; j < PM_SLAB; ++j)
+                            v[j] = __float_as_uint(fmaf(-mean, __ldg(c1 + j), __uint_as_float(v[j])) +
+                                                   inv_rstd * __ldg(c2 + j));
+                    }
                     uint4 o[2];
                     uint32_t* ow = reinterpret_cast<uint32_t*>(o);
 #pragma unroll
@@ -852,7 +885,8 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 }
 
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int n_sms) {
+                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int n_sms,
+                          const float2* ln_stats) {
     if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
     ShrinkArgs a;
     a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap; a.n_tiles = R.n_tiles;
@@ -866,6 +900,8 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     a.stages = (4 * stage_bytes + 256 <= 112 * 1024) ? 4 : 3;
     a.tile_nslabs = R.tile_nslabs; a.tile_slab = R.tile_slab; a.tile_scale = R.tile_scale;
     a.tile_mask = R.tile_mask; a.tbuf = tbuf; a.status = L.status;
+    if ((lin.ln_g != nullptr) != (ln_stats != nullptr)) return cudaErrorInvalidValue;
+    a.ln_stats = ln_stats; a.ln_c1 = lin.ln_c1; a.ln_c2 = lin.ln_c2;
     const int smem = a.stages * stage_bytes + 256;
     static int smem_set = 0;
     if (smem > smem_set) {
@@ -886,14 +922,14 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
 #endif
 constexpr int GEMM_EPI_WARPS = PM_GEMM_EPI_WARPS;      // 4 or 8
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool LNF = false>
 static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
                                   const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                   const GemmArgs& a, int n_sms) {
     constexpr int EW = GEMM_EPI_WARPS;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN, EPI, EW>,
+        cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN, EPI, EW, LNF>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, EW>::TOTAL);
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -901,7 +937,7 @@ static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, cons
     const int total = a.m_tiles * a.n_tiles;
     const int grid = total < n_sms ? total : n_sms;
     ProfScope ps(L, KC_GEMM);
-    lora_gemm_kernel<BN, EPI, EW><<<grid, 64 + 32 * EW, Smem<BN, EW>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, tm_y, a);
+    lora_gemm_kernel<BN, EPI, EW, LNF><<<grid, 64 + 32 * EW, Smem<BN, EW>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, tm_y, a);
     BUMP(L);
     return cudaGetLastError();
 }
@@ -910,6 +946,11 @@ template <int BN>
 static cudaError_t launch_gemm_epi(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
                                    const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                    const GemmArgs& a, int n_sms) {
+    if (a.ln_stats) {        // LayerNorm folded in: only the epilogues that follow a LayerNorm
+        if (a.epi == EPI_GELU) return launch_gemm_bn<BN, EPI_GELU, true>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        if (a.epi == EPI_NONE) return launch_gemm_bn<BN, EPI_NONE, true>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        return cudaErrorInvalidValue;
+    }
     switch (a.epi) {
         case EPI_GELU: return launch_gemm_bn<BN, EPI_GELU>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
         case EPI_RESIDUAL: return launch_gemm_bn<BN, EPI_RESIDUAL>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
@@ -918,13 +959,13 @@ static cudaError_t launch_gemm_epi(const Launch& L, const CUtensorMap& tm_x, con
     }
 }
 
-template <int EPI>
+template <int EPI, bool LNF = false>
 static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
                                     const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                     const GemmArgs& a, int n_sms) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<EPI, LNF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              P_SMEM_TOTAL);
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -942,7 +983,7 @@ static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, co
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ProfScope ps(L, KC_GEMM);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_pair_kernel<EPI>, tm_x, tm_w, tm_t, tm_bt, tm_y, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_pair_kernel<EPI, LNF>, tm_x, tm_w, tm_t, tm_bt, tm_y, a);
     BUMP(L);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -950,6 +991,11 @@ static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, co
 static cudaError_t launch_gemm_pair_epi(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
                                         const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                         const GemmArgs& a, int n_sms) {
+    if (a.ln_stats) {
+        if (a.epi == EPI_GELU) return launch_gemm_pair<EPI_GELU, true>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        if (a.epi == EPI_NONE) return launch_gemm_pair<EPI_NONE, true>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        return cudaErrorInvalidValue;
+    }
     switch (a.epi) {
         case EPI_GELU: return launch_gemm_pair<EPI_GELU>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
         case EPI_RESIDUAL: return launch_gemm_pair<EPI_RESIDUAL>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
@@ -965,8 +1011,9 @@ int gemm_tile_n(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
                              const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
                              int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
-                             int n_sms) {
+                             int n_sms, const float2* ln_stats) {
     if (rows <= 0) return cudaSuccess;
+    if ((lin.ln_g != nullptr) != (ln_stats != nullptr)) return cudaErrorInvalidValue;
     const int bn = gemm_tile_n(lin.n_out);
     GemmArgs a;
     a.rows = rows; a.k_in = lin.k_in; a.n_out = lin.n_out;
@@ -978,6 +1025,7 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
     a.tile_slab = lora ? R->tile_slab : nullptr;
     a.slab_cap = lora ? R->slab_cap : 0;
     a.status = L.status;
+    a.ln_g = lin.ln_g; a.ln_stats = ln_stats;
     a.tma_store = (tm_y != nullptr && epi != EPI_PATCH) ? 1 : 0;
     const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced
     const CUtensorMap& ty = a.tma_store ? *tm_y : tm_x;

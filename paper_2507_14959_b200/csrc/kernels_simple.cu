@@ -129,6 +129,48 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const T* __restrict__ x,
     ln_row<T, T>(x + (size_t)row * d, g, b, y + (size_t)row * d, d, eps, threadIdx.x & 31);
 }
 
+// Row statistics only (mean and 1/sqrt(var + eps), biased variance, two passes over the registers):
+// for the linears that have LayerNorm folded into their weights the normalised rows are never
+// written out; the GEMM and shrink epilogues apply the statistics instead.
+__global__ void __launch_bounds__(256) row_stats_kernel(const bf16* __restrict__ x, float2* __restrict__ stats,
+                                                        int rows, int d, float eps) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const int nch = d >> 3;
+    const bf16* xr = x + (size_t)row * d;
+    float v[32];
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = lane + 32 * i;
+        if (c < nch) {
+            load16<bf16>(xr + c * 8, v + i * 8);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sum += v[i * 8 + j];
+        }
+    }
+    const float mean = warp_sum(sum) / (float)d;
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (lane + 32 * i < nch) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { const float t = v[i * 8 + j] - mean; sq += t * t; }
+        }
+    }
+    const float rstd = rsqrtf(warp_sum(sq) / (float)d + eps);
+    if (lane == 0) stats[row] = make_float2(mean, rstd);
+}
+
+cudaError_t launch_row_stats(const Launch& L, const bf16* x, float2* stats, int rows, int d, float eps) {
+    if (rows <= 0) return cudaSuccess;
+    ProfScope ps(L, KC_LAYERNORM);
+    row_stats_kernel<<<(rows + 7) / 8, 256, 0, L.st>>>(x, stats, rows, d, eps);
+    BUMP(L);
+    return cudaGetLastError();
+}
+
 template <typename T>
 cudaError_t launch_layernorm(const Launch& L, const T* x, const float* g, const float* b, T* y,
                              int rows, int d, float eps) {
