@@ -54,7 +54,12 @@ def gemm_flops_per_step(w):
     active_rank = sum(w.adapters[a].rank for a in w.set_ids)          # sum over frames of sum_a r_a
     F = w.n_frames
     base = sum(2 * k * n for k, n in shapes) * T * F * L
-    lora = sum(2 * (k + n) for k, n in shapes) * T * active_rank * L
+    # blocks an adapter really touches (its A/B pairs that are not None), per projection
+    lora = 0
+    for a in w.set_ids:
+        ad = w.adapters[a]
+        for i, (k, n) in enumerate(shapes):
+            lora += 2 * (k + n) * T * ad.rank * sum(1 for l in range(L) if ad.A[l * 4 + i] is not None)
     patch = 2 * s.patch_dim * d * (T - 1) * F
     return base + lora + patch
 
@@ -244,6 +249,9 @@ def main():
     ap.add_argument("--impl", default="polymorph", choices=["polymorph", "reference"])
     ap.add_argument("--frames", type=int, default=256, help="frames per GPU per step")
     ap.add_argument("--cpu-sample", type=int, default=16, help="frames of the CPU-baseline sample (0 = skip)")
+    ap.add_argument("--lora-last", type=int, default=None,
+                    help="batch workload only: adapters touch the last N blocks only (the paper's cheap "
+                         "placement); default: all blocks, the headline configuration")
     ap.add_argument("--workload", default="batch", choices=["batch", "streams"],
                     help="batch: ViT-base 224x224, 256 frames (the headline); streams: ViT-base 384x384, 16 streams "
                          "in closed loop (forward -> Algorithm 2 -> next forward), one step = one frame per stream")
@@ -273,7 +281,7 @@ def main():
         run_streams(args, rank, world, dist)
         return
 
-    w = wl.vit_base_batch(n_frames=args.frames)
+    w = wl.vit_base_batch(n_frames=args.frames, lora_last=args.lora_last)
     m = binding.model_from_workload(w, dtype=0)
     m.set_cover(w.tau)
     F, K = w.n_frames, w.spec.n_classes
@@ -371,7 +379,8 @@ def main():
             "config": {"workload": "vit_base_batch: ViT-base 224x224 (197 tokens), %d frames/GPU/step, 32 rank-16 "
                                    "adapters over 800 classes, 1-3 active adapters per frame (60/30/10 %%), "
                                    "forward + Algorithm 2 select" % F,
-                       "frames_per_gpu": F, "l2": "activations (~0.9 GB/step) exceed the 126 MB L2; no flush"},
+                       "frames_per_gpu": F, "l2": "activations (~0.9 GB/step) exceed the 126 MB L2; no flush",
+                       "lora_blocks": "all 12" if args.lora_last is None else "last %d" % args.lora_last},
             "e2e": {"value": world * F * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(frames_host.numel() * 2),
                     "d2h_bytes_per_step": int(scores_host.numel() * 4 + base_host.numel() * 4)},

@@ -168,8 +168,17 @@ struct LinearObj {
         return PM_OK;
     }
     int set_adapter(int a, int rank, const float* A, const float* B, std::string& err) {
+        if ((int)adapted.size() < max_adapters) adapted.assign(max_adapters, 0);
+        adapted[a] = (A && B) ? 1 : 0;
+        n_adapted = 0;
+        for (char c : adapted) n_adapted += c;
         return dtype == 0 ? set_adapter_t<bf16>(a, rank, A, B, err) : set_adapter_t<float>(a, rank, A, B, err);
     }
+    // adapters that really touch this linear (a NULL A/B pair leaves it un-adapted); with none, the
+    // forward skips the shrink and the LoRA steps here altogether -- the paper's cheap variant, LoRA in
+    // the last blocks only (Sec. 3.1), then costs nothing in the other blocks
+    std::vector<char> adapted;
+    int n_adapted = 0;
 };
 
 // Per-batch routing: validation, bucketing, tile plan, upload.
@@ -462,7 +471,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     auto linear = [&](LinearObj& lo, const T* x, const CUtensorMap* tmx, int nrows, int tokens_pf, bool lora,
                       int epi, const T* residual, const PatchEpi& pep, T* y, const float2* st = nullptr) -> cudaError_t {
         if constexpr (TC) {
-            const bool use_lora = lora && R.max_set > 0;
+            const bool use_lora = lora && R.max_set > 0 && lo.n_adapted > 0;
             if (use_lora) {
                 cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>(), h->n_sms, st);
                 if (e != cudaSuccess) return e;

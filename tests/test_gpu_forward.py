@@ -69,6 +69,46 @@ def test_deit_tiny_2frames(dtype):
     m.close()
 
 
+@pytest.mark.parametrize("dtype", [1, 0])
+def test_paper_variant_query_value_last_blocks(dtype):
+    """The paper's own placement of the adapters (Sec. 3.1, Sec. 4): LoRA on the query and value
+    projections of the last 20 % of the blocks only (2 of 12), every other block shared.  Expressed
+    through the same API: NULL A/B pairs everywhere else, and zero key columns in B of the qkv linear."""
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    d = w.spec.d
+    ads = []
+    for a, ad in enumerate(w.adapters):
+        A = [None] * len(ad.A)
+        B = [None] * len(ad.B)
+        for l in (10, 11):
+            A[l * 4] = ad.A[l * 4]
+            b = ad.B[l * 4].copy()
+            b[:, d:2 * d] = 0.0                      # query and value only: no update of the keys
+            B[l * 4] = b
+        ads.append(wl.Adapter(rank=ad.rank, scale=ad.scale, A=A, B=B, class_ids=ad.class_ids,
+                              head_w=ad.head_w, head_b=ad.head_b, acc=ad.acc))
+    w2 = wl.Workload(w.name, w.spec, w.backbone, ads, w.frames, w.set_offsets, w.set_ids)
+    m = binding.model_from_workload(w2, dtype=dtype)
+    n0 = m.launch_count()
+    s, b = run_forward(m, w2, dtype)
+    launches = m.launch_count() - n0
+    so, bo = oracle_rows(w2, range(2))
+    assert np.abs(s - so).max() < SCORE_TOL[dtype]
+    assert np.abs(b - bo).max() < SCORE_TOL[dtype]
+    # the adapters do act (compare with the plain backbone), yet only two linears carry LoRA work
+    off, ids = wl.sets_to_csr([[], []])
+    _, bo_plain = oracle_rows(w2, range(2), offsets=off, ids=ids)
+    assert np.abs(bo - bo_plain).max() > 1e-4
+    if dtype == 0:
+        m_all = binding.model_from_workload(w, dtype=0)
+        n1 = m_all.launch_count()
+        run_forward(m_all, w, 0)
+        assert m_all.launch_count() - n1 == launches + 46     # 48 shrink launches against 2
+        m_all.close()
+    m.close()
+
+
 def test_forward_argument_errors():
     import torch
     from paper_2507_14959_b200 import binding

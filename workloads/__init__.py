@@ -249,14 +249,17 @@ def overlapping_groups(n_groups: int, per_group: int):
     return K, [np.asarray(sorted(g), dtype=np.int32) for g in groups]
 
 
-def vit_base_batch(n_frames=256, layers=12) -> Workload:
+def vit_base_batch(n_frames=256, layers=12, lora_last=None) -> Workload:
     """ViT-base production shape: 32 rank-16 adapters over 800 classes (32 groups of 25, 10 %
-    of classes shared by two groups); 60/30/10 % of frames have 1/2/3 active adapters."""
+    of classes shared by two groups); 60/30/10 % of frames have 1/2/3 active adapters.
+    lora_last = N restricts every adapter to the last N blocks (the paper's cheap placement,
+    Sec. 3.1); None adapts all blocks."""
     name = "vit_base_batch"
     spec = ModelSpec(img=224, d=768, heads=12, mlp=3072, n_classes=800, layers=layers)
     bb = make_backbone(name, spec)
     _, groups = overlapping_groups(32, 25)
-    ads = [make_adapter(name, spec, a, 16, groups[a]) for a in range(32)]
+    lora_layers = None if lora_last is None else range(layers - lora_last, layers)
+    ads = [make_adapter(name, spec, a, 16, groups[a], layers=lora_layers) for a in range(32)]
     g = rng_for(name, "sets")
     sets = [draw_set(g, 32) for _ in range(n_frames)]
     off, ids = sets_to_csr(sets)
