@@ -297,8 +297,8 @@ def main():
             torch.zeros(F * len(w.adapters), dtype=torch.int32, device="cuda")) for _ in range(2)]
     stream = torch.cuda.current_stream()
 
-    def step(i):
-        m.forward(frames_dev, w.set_offsets, w.set_ids, scores, base)
+    def step(i, frames=None):
+        m.forward(frames_dev if frames is None else frames, w.set_offsets, w.set_ids, scores, base)
         prev, nxt = sel[i % 2], sel[(i + 1) % 2]
         m.select(base, 0.5, False, i > 0, labels, prev[0], prev[1], nxt[0], nxt[1])
 
@@ -346,9 +346,24 @@ def main():
     assert m.status() == 0, "device status word set during the timed region"
 
     # ---- end to end: host frames in, host scores out, copies inside the timed region ------
+    # Every step copies its frames from pinned host memory and its scores back.  The input copy runs on
+    # a second stream into one of two device buffers, so step i+1's frames travel while step i computes.
+    copy_stream = torch.cuda.Stream()
+    in_bufs = [frames_dev, torch.empty_like(frames_dev)]
+    ready = [torch.cuda.Event(), torch.cuda.Event()]
+    free = [torch.cuda.Event(), torch.cuda.Event()]
+    for ev in free:
+        ev.record(stream)
+
     def e2e_step(i):
-        frames_dev.copy_(frames_host, non_blocking=True)
-        step(i)
+        b = i % 2
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(free[b])          # the step that last read this buffer is done
+            in_bufs[b].copy_(frames_host, non_blocking=True)
+            ready[b].record(copy_stream)
+        stream.wait_event(ready[b])
+        step(i, in_bufs[b])
+        free[b].record(stream)
         scores_host.copy_(scores, non_blocking=True)
         base_host.copy_(base, non_blocking=True)
 
