@@ -90,11 +90,15 @@ struct Smem {
 // chunks goes TMEM -> registers -> bias / GELU / residual / patch placement -> bf16 -> shared
 // memory -> TMA store (or straight to global memory).  Returns false once the CTA is aborting.
 // PAIR: the accumulator-free barrier lives in the even CTA of a pair (tempty_addr is a cluster address).
-template <int BN, int EPI, int HALVES, bool PAIR, bool LNF>
+// RES_SMEM: the residual rows come through shared memory (TMA into res_buf, four 2 KB chunks of this
+// warp, completion on res_bar) instead of per-thread global loads.
+template <int BN, int EPI, int HALVES, bool PAIR, bool LNF, bool RES_SMEM>
 __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtensorMap& tm_y, uint32_t staging,
                                               uint32_t& chunk_no, uint32_t tmem_base, int acc, uint32_t acc_phase,
                                               uint32_t tfull_addr, uint32_t tempty_addr, volatile int* abort_flag,
-                                              int m, int n, int quarter, int half, int lane) {
+                                              int m, int n, int quarter, int half, int lane,
+                                              const CUtensorMap* tm_res, uint32_t res_buf, uint32_t res_bar,
+                                              uint32_t res_phase) {
     constexpr int CPW = BN / 32 / HALVES;         // 32-column chunks per epilogue warp
     const int row = m * BM + quarter * 32 + lane;     // m: 128-row tile index
     const bool row_ok = row < args.rows;
@@ -104,8 +108,18 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
     // The residual rows of this warp's chunks are fetched before the accumulator is ready, so
     // their latency hides behind the main loop.  (In-place use, y == residual, is safe: the
     // same thread reads an element here and is the only one to overwrite it below.)
-    uint4 rr[EPI == EPI_RESIDUAL ? CPW : 1][4];
-    if constexpr (EPI == EPI_RESIDUAL) {
+    uint4 rr[(EPI == EPI_RESIDUAL && !RES_SMEM) ? CPW : 1][4];
+    if constexpr (EPI == EPI_RESIDUAL && RES_SMEM) {
+        // one thread asks TMA for this warp's chunks of the residual tile (rows past the end read as
+        // zero); the warp's reads of the previous tile's chunks are ordered before these writes
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+            mbar_expect_tx(res_bar, (uint32_t)(my_chunks * 32 * 64));
+            for (int cc = 0; cc < my_chunks; ++cc)
+                tma_load_2d(res_buf + cc * (32 * 64), tm_res, n * BN + (c0 + cc) * 32, m * BM + quarter * 32, res_bar);
+        }
+    } else if constexpr (EPI == EPI_RESIDUAL) {
 #pragma unroll
         for (int cc = 0; cc < CPW; ++cc) {
             if (cc < my_chunks && row_ok) {
@@ -169,9 +183,25 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
 #pragma unroll
             for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
         } else if constexpr (EPI == EPI_RESIDUAL) {
+            if constexpr (RES_SMEM) {
+                if (cc == 0) {
+                    ok = mbar_wait(res_bar, res_phase, abort_flag, args.status);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) return false;
+                }
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const uint32_t w[4] = {rr[cc][q].x, rr[cc][q].y, rr[cc][q].z, rr[cc][q].w};
+                uint4 r4v;
+                if constexpr (RES_SMEM) {
+                    // same 64B swizzle as the store staging: 16-byte chunk q of row `lane`
+                    const uint32_t a = res_buf + cc * (32 * 64) + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4);
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(r4v.x), "=r"(r4v.y), "=r"(r4v.z), "=r"(r4v.w) : "r"(a));
+                } else {
+                    r4v = rr[cc][q];
+                }
+                const uint32_t w[4] = {r4v.x, r4v.y, r4v.z, r4v.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
@@ -388,9 +418,9 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int m = tile / args.n_tiles, n = tile % args.n_tiles;
-            ok = epilogue_tile<BN, EPI, HALVES, false, LNF>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
-                                                       tfull_bar(acc), tempty_bar(acc), abort_flag, m, n, quarter,
-                                                       half, lane);
+            ok = epilogue_tile<BN, EPI, HALVES, false, LNF, false>(args, tm_y, staging, chunk_no, tmem_base, acc,
+                                                              acc_phase, tfull_bar(acc), tempty_bar(acc), abort_flag,
+                                                              m, n, quarter, half, lane, nullptr, 0u, 0u, 0u);
             if (!ok) break;
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
@@ -425,39 +455,53 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 // ---------------------------------------------------------------------------------------
 constexpr int P_BN = 256;
 constexpr int P_EW = 8;
-constexpr int P_STAGES = 6;
+// Ring depth and residual landing area by epilogue: the residual epilogue trades two of the six 32 KB
+// stages for a 64 KB area into which TMA fetches the tile's residual rows ahead of the accumulator.
+template <int EPI, bool RESS>
+struct PairCfg {
+    static constexpr bool RES = EPI == EPI_RESIDUAL && RESS;
+    static constexpr int STAGES = RES ? 4 : 6;
+    static constexpr int RES_BYTES_PER_WARP = RES ? 4 * 32 * 64 : 0;       // four [32 rows x 32 bf16] chunks
+};
 constexpr int P_A_BYTES = BM * BK * 2;                 // 16 KB: this CTA's 128 rows of x
 constexpr int P_B_BYTES = (P_BN / 2) * BK * 2;         // 16 KB: this CTA's half of the W^T tile
 constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES;
 constexpr int P_T_SLAB_BYTES = BM * PM_SLAB * 2;       // 4 KB
 constexpr int P_B_SLAB_BYTES = (P_BN / 2) * PM_SLAB * 2;   // 4 KB
-constexpr int P_STAGING_OFFSET = P_STAGES * P_STAGE_BYTES;
-constexpr int P_PLAN_OFFSET = P_STAGING_OFFSET + P_EW * STAGING_BYTES_PER_WARP;
+constexpr int P_MAX_STAGES = 6;
+constexpr int P_STAGING_OFFSET = P_MAX_STAGES * P_STAGE_BYTES;      // stages, then (residual kernels) the
+constexpr int P_PLAN_OFFSET = P_STAGING_OFFSET + P_EW * STAGING_BYTES_PER_WARP;   // residual area inside them
 constexpr int P_BAR_OFFSET = P_PLAN_OFFSET + PLAN_BYTES;
 constexpr int P_SMEM_TOTAL = P_BAR_OFFSET + 256;
 constexpr int P_THREADS = 64 + 32 * P_EW;
 
-template <int EPI, bool LNF>
+// RESS (residual epilogue only): residual through shared memory with a four-stage ring (short K, where
+// the epilogue is exposed) instead of per-thread loads with the full six stages (long K).
+template <int EPI, bool LNF, bool RESS>
 __global__ void __launch_bounds__(P_THREADS, 1)
 lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                       const __grid_constant__ CUtensorMap tm_t, const __grid_constant__ CUtensorMap tm_bt,
-                      const __grid_constant__ CUtensorMap tm_y, const GemmArgs args) {
+                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res,
+                      const GemmArgs args) {
     constexpr int BN = P_BN;
     constexpr int HALVES = P_EW / 4;
+    constexpr int P_STAGES = PairCfg<EPI, RESS>::STAGES;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t base = smem_u32(smem_raw);
     const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs, 1: its peer
     uint8_t* smem = smem_raw;
     const uint32_t bars = base + P_BAR_OFFSET;
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (P_STAGES + s); };
-    auto tfull_bar = [&](int s) { return bars + 8u * (2 * P_STAGES + s); };
-    auto tempty_bar = [&](int s) { return bars + 8u * (2 * P_STAGES + 2 + s); };
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + P_BAR_OFFSET + 8 * (2 * P_STAGES + 4));
+    auto empty_bar = [&](int s) { return bars + 8u * (P_MAX_STAGES + s); };
+    auto tfull_bar = [&](int s) { return bars + 8u * (2 * P_MAX_STAGES + s); };
+    auto tempty_bar = [&](int s) { return bars + 8u * (2 * P_MAX_STAGES + 2 + s); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + P_BAR_OFFSET + 8 * (2 * P_MAX_STAGES + 4));
     // the peer CTA's TMEM base: written only by the peer (any time before the cluster barrier below),
     // never by this CTA, so there is no ordering to get wrong
     volatile uint32_t* peer_slot = tmem_slot + 1;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + P_BAR_OFFSET + 8 * (2 * P_STAGES + 4) + 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + P_BAR_OFFSET + 8 * (2 * P_MAX_STAGES + 4) + 8);
+    // res_bar[w]: the residual rows of epilogue warp w's chunks have landed (residual kernels)
+    auto res_bar = [&](int w) { return bars + 8u * (2 * P_MAX_STAGES + 4) + 24u + 8u * w; };
     int* plan = reinterpret_cast<int*>(smem + P_PLAN_OFFSET);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -489,6 +533,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 2 * P_EW); }
+        for (int w = 0; w < P_EW; ++w) mbar_init(res_bar(w), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -605,14 +650,17 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         const int half = (warp - 2) >> 2;
         const uint32_t staging = base + P_STAGING_OFFSET + (uint32_t)(warp - 2) * STAGING_BYTES_PER_WARP;
         int acc = 0;
-        uint32_t acc_phase = 0;
+        uint32_t acc_phase = 0, res_phase = 0;
         uint32_t chunk_no = 0;
         bool ok = true;
         for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
             const int m = 2 * (tile / args.n_tiles) + (int)rank, n = tile % args.n_tiles;
-            ok = epilogue_tile<BN, EPI, HALVES, true, LNF>(args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase,
-                                                      tfull_bar(acc), mapa_cluster(tempty_bar(acc), 0), abort_flag,
-                                                      m, n, quarter, half, lane);
+            ok = epilogue_tile<BN, EPI, HALVES, true, LNF, PairCfg<EPI, RESS>::RES>(
+                args, tm_y, staging, chunk_no, tmem_base, acc, acc_phase, tfull_bar(acc),
+                mapa_cluster(tempty_bar(acc), 0), abort_flag, m, n, quarter, half, lane, &tm_res,
+                base + PairCfg<EPI, RESS>::STAGES * P_STAGE_BYTES + (uint32_t)(warp - 2) * PairCfg<EPI, RESS>::RES_BYTES_PER_WARP,
+                res_bar(warp - 2), res_phase);
+            res_phase ^= 1u;
             if (!ok) break;
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
@@ -959,13 +1007,19 @@ static cudaError_t launch_gemm_epi(const Launch& L, const CUtensorMap& tm_x, con
     }
 }
 
-template <int EPI, bool LNF = false>
+template <int EPI, bool LNF = false, bool RESS = false>
 static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, const CUtensorMap& tm_w,
                                     const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                     const GemmArgs& a, int n_sms) {
+    // the residual tile is fetched by TMA with the output's geometry (32 x 32 boxes, 64B swizzle)
+    CUtensorMap tm_res = tm_y;
+    if (EPI == EPI_RESIDUAL && (const void*)a.residual != (const void*)a.y) {
+        if (!tm_encode_2d(&tm_res, a.residual, a.n_out, a.rows, (uint64_t)a.n_out * 2, 32, 32, 64))
+            return cudaErrorInvalidValue;
+    }
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<EPI, LNF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<EPI, LNF, RESS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              P_SMEM_TOTAL);
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -983,7 +1037,7 @@ static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, co
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     ProfScope ps(L, KC_GEMM);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_pair_kernel<EPI, LNF>, tm_x, tm_w, tm_t, tm_bt, tm_y, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_pair_kernel<EPI, LNF, RESS>, tm_x, tm_w, tm_t, tm_bt, tm_y, tm_res, a);
     BUMP(L);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -998,7 +1052,9 @@ static cudaError_t launch_gemm_pair_epi(const Launch& L, const CUtensorMap& tm_x
     }
     switch (a.epi) {
         case EPI_GELU: return launch_gemm_pair<EPI_GELU>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
-        case EPI_RESIDUAL: return launch_gemm_pair<EPI_RESIDUAL>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+        case EPI_RESIDUAL:
+            if (a.k_in <= 1024) return launch_gemm_pair<EPI_RESIDUAL, false, true>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
+            return launch_gemm_pair<EPI_RESIDUAL>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
         case EPI_PATCH: return launch_gemm_pair<EPI_PATCH>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
         default: return launch_gemm_pair<EPI_NONE>(L, tm_x, tm_w, tm_t, tm_bt, tm_y, a, n_sms);
     }
@@ -1029,7 +1085,7 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
     a.tma_store = (tm_y != nullptr && epi != EPI_PATCH) ? 1 : 0;
     const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced
     const CUtensorMap& ty = a.tma_store ? *tm_y : tm_x;
-    if (lin.has_tm_half && n_sms >= 2) {
+    if (lin.has_tm_half && n_sms >= 2 && (epi != EPI_RESIDUAL || a.tma_store)) {
         a.m_tiles = (rows + 2 * BM - 1) / (2 * BM);       // 256-row tiles
         a.n_tiles = lin.n_out / P_BN;
         return launch_gemm_pair_epi(L, tm_x, lin.tm_w_half, tt, lora ? lin.tm_bt_half : lin.tm_w_half, ty, a, n_sms);
