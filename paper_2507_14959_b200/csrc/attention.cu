@@ -419,14 +419,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tmem_ld32((t_lane + args.o_col) + (uint32_t)(half * 32), v);
                         tmem_ld_wait();
                         if (q_row < T) {
+                            // 32-byte stores: one full sector per row per instruction
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                uint4 o;
-                                o.x = pack2(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
-                                o.y = pack2(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
-                                o.z = pack2(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
-                                o.w = pack2(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
-                                reinterpret_cast<uint4*>(orow + half * 32)[q] = o;
+                            for (int q = 0; q < 2; ++q) {
+                                uint32_t o[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    o[e] = pack2(__uint_as_float(v[q * 16 + 2 * e]) * inv,
+                                                 __uint_as_float(v[q * 16 + 2 * e + 1]) * inv);
+                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                             ::"l"(orow + half * 32 + q * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]),
+                                               "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                                             : "memory");
                             }
                         }
                     }
