@@ -693,6 +693,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 // ---------------------------------------------------------------------------------------
 struct ShrinkArgs {
     int rows, k_in, slab_cap, sg, n_tiles, stages;
+    int reverse;                   // walk the tiles from the last row tile down (see launch_shrink)
     uint32_t acc_cols;             // TMEM columns of one accumulator buffer (power of two >= 16 * sg)
     const int* tile_nslabs;
     const int* tile_slab;
@@ -757,7 +758,8 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < args.n_tiles && ok; tile += gridDim.x) {
+            for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
+                const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
                 const int ns = args.tile_nslabs[tile];
                 for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
                     const int cnt = min(args.sg, ns - g0);
@@ -784,7 +786,8 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < args.n_tiles && ok; tile += gridDim.x) {
+            for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
+                const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
                 const int ns = args.tile_nslabs[tile];
                 for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
                     const int cnt = min(args.sg, ns - g0);
@@ -819,7 +822,8 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < args.n_tiles && ok; tile += gridDim.x) {
+        for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
+            const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
             const int ns = args.tile_nslabs[tile];
             for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
                 const int cnt = min(args.sg, ns - g0);
@@ -950,6 +954,10 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     a.tile_mask = R.tile_mask; a.tbuf = tbuf; a.status = L.status;
     if ((lin.ln_g != nullptr) != (ln_stats != nullptr)) return cudaErrorInvalidValue;
     a.ln_stats = ln_stats; a.ln_c1 = lin.ln_c1; a.ln_c2 = lin.ln_c2;
+    // x larger than the L2 cache was written front to back by the kernel before this one, so its tail
+    // is what the cache still holds: start there, and leave the front in the cache for the GEMM that
+    // follows (which walks front to back)
+    a.reverse = (size_t)rows * lin.k_in * sizeof(bf16) > ((size_t)96 << 20) ? 1 : 0;
     const int smem = a.stages * stage_bytes + 256;
     static int smem_set = 0;
     if (smem > smem_set) {
