@@ -369,7 +369,7 @@ struct pm_handle_s {
     DevBuf cls, pos, ln1_g, ln1_b, ln2_g, ln2_b, lnf_g, lnf_b, head_wt, head_b;
     // activations
     DevBuf X, U, QKV, ATT, H, PATCH, Z, t32, tbuf, status, ln_stats;
-    CUtensorMap tm_patch, tm_u, tm_att, tm_h, tm_t, tm_x_in;
+    CUtensorMap tm_patch, tm_att, tm_h, tm_t, tm_x_in;
     CUtensorMap tm_y_qkv, tm_y_x, tm_y_h;      // outputs, for the TMA-store epilogue
     CUtensorMap tm_att_q, tm_att_kv;           // attention operands over QKV
     int tm_rows = -1;
@@ -438,7 +438,6 @@ int encode_activation_maps(pm_handle_s* h, int rows) {
     const int d = h->cfg.d;
     const int prow = rows / h->tokens * h->g2;
     bool ok = tm_encode_2d(&h->tm_patch, h->PATCH.p, h->patch_dim, prow, (uint64_t)h->patch_dim * 2, 64, PM_TILE_M, 128)
-           && tm_encode_2d(&h->tm_u, h->U.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_x_in, h->X.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_att, h->ATT.p, d, rows, (uint64_t)d * 2, 64, PM_TILE_M, 128)
            && tm_encode_2d(&h->tm_h, h->H.p, h->cfg.mlp, rows, (uint64_t)h->cfg.mlp * 2, 64, PM_TILE_M, 128)
@@ -497,7 +496,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
             CK(linear(h->lin[l * 4 + 0], X, &h->tm_x_in, rows, T_, true, EPI_NONE, nullptr, none, QKV, h->ln_stats.as<float2>()));
         } else {
             CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
-            CK(linear(h->lin[l * 4 + 0], U, &h->tm_u, rows, T_, true, EPI_NONE, nullptr, none, QKV));
+            CK(linear(h->lin[l * 4 + 0], U, nullptr, rows, T_, true, EPI_NONE, nullptr, none, QKV));
         }
         if constexpr (TC) {
             if (attention_tc_supported(T_))
@@ -512,7 +511,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
             CK(linear(h->lin[l * 4 + 2], X, &h->tm_x_in, rows, T_, true, EPI_GELU, nullptr, none, Hb, h->ln_stats.as<float2>()));
         } else {
             CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
-            CK(linear(h->lin[l * 4 + 2], U, &h->tm_u, rows, T_, true, EPI_GELU, nullptr, none, Hb));
+            CK(linear(h->lin[l * 4 + 2], U, nullptr, rows, T_, true, EPI_GELU, nullptr, none, Hb));
         }
         CK(linear(h->lin[l * 4 + 3], Hb, &h->tm_h, rows, T_, true, EPI_RESIDUAL, X, none, X));
     }
@@ -554,13 +553,14 @@ int create_t(pm_handle_s* h, const pm_backbone* w) {
     CK(upload<float>(h->head_b, w->head_b, K));
     const size_t rows = (size_t)c.max_frames * T_;
     const size_t rows_pad = (rows + PM_TILE_M - 1) / PM_TILE_M * PM_TILE_M;
-    CK(h->X.alloc(rows_pad * d * sizeof(T))); CK(h->U.alloc(rows_pad * d * sizeof(T)));
+    // U holds the normalised rows of the fp32 build only (the bf16 build folds LayerNorm into the weights)
+    CK(h->X.alloc(rows_pad * d * sizeof(T))); CK(h->U.alloc(sizeof(T) == 2 ? 0 : rows_pad * d * sizeof(T)));
     CK(h->QKV.alloc(rows_pad * 3 * d * sizeof(T))); CK(h->ATT.alloc(rows_pad * d * sizeof(T)));
     CK(h->H.alloc(rows_pad * m * sizeof(T)));
     CK(h->PATCH.alloc(rows_pad * h->patch_dim * sizeof(T)));
     CK(h->Z.alloc((size_t)c.max_frames * d * sizeof(float)));
     CK(h->ln_stats.alloc(rows_pad * sizeof(float2)));
-    CK(cudaMemset(h->X.p, 0, h->X.bytes)); CK(cudaMemset(h->U.p, 0, h->U.bytes));
+    CK(cudaMemset(h->X.p, 0, h->X.bytes)); if (h->U.p) CK(cudaMemset(h->U.p, 0, h->U.bytes));
     CK(cudaMemset(h->QKV.p, 0, h->QKV.bytes)); CK(cudaMemset(h->ATT.p, 0, h->ATT.bytes));
     CK(cudaMemset(h->H.p, 0, h->H.bytes)); CK(cudaMemset(h->PATCH.p, 0, h->PATCH.bytes));
     rc = h->router.init(c.max_frames, c.max_set, c.max_adapters, h->slabs_max, T_, err);

@@ -199,6 +199,7 @@ constexpr int ATT_MAX_BLOCKS = 3;
 
 struct AttnArgs {
     int tokens, heads, tpad, n_blocks, n_qtiles;
+    int q_split;               // CTAs per (frame, head); each takes a contiguous share of the query tiles
     uint32_t tmem_cols, o_col;
     bf16* out;
     int* status;
@@ -279,7 +280,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
         return;
     }
-    const int f = blockIdx.x / args.heads, h = blockIdx.x % args.heads;
+    const int fh = blockIdx.x / args.q_split, part = blockIdx.x % args.q_split;
+    const int f = fh / args.heads, h = fh % args.heads;
+    const int per = (args.n_qtiles + args.q_split - 1) / args.q_split;
+    const int qt0 = part * per, qt1 = min(args.n_qtiles, qt0 + per);          // this CTA's query tiles
     const int d = args.heads * HD;
     const int T = args.tokens;
     const int n_blocks = args.n_blocks;
@@ -307,7 +311,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tma_load_2d(v_s + b * AKB_BYTES, &tm_kv, 2 * d + h * HD, f * T + b * AKB, kv_bar);
         }
         mbar_expect_tx(q_bar, AQ_BYTES);
-        tma_load_2d(q_s, &tm_q, h * HD, f * T, q_bar);
+        tma_load_2d(q_s, &tm_q, h * HD, f * T + qt0 * AQ, q_bar);
     }
     __syncwarp();
     if (warp == 0) {
@@ -328,9 +332,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const uint64_t dq0 = smem_desc(q_s, 128), dk0 = smem_desc(k_s, 128), dv0 = smem_desc(v_s, 128);
             uint32_t step = 0;
             bool ok = true;
-            for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
-                if (qt == 0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
-                ok = ok && mbar_wait(q_bar, qt & 1, abort_flag, args.status);
+            for (int qt = qt0; qt < qt1 && ok; ++qt) {
+                if (qt == qt0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
+                ok = ok && mbar_wait(q_bar, (qt - qt0) & 1, abort_flag, args.status);
                 if (!ok) break;
                 tc_fence_after();
                 for (int pass = (n_blocks > 1 ? 0 : 1); pass < 2 && ok; ++pass) {
@@ -348,7 +352,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (!ok) break;
                         tc_fence_after();
                         if (pass == 1) {
-                            if (b == n_blocks - 1 && qt + 1 < args.n_qtiles) {
+                            if (b == n_blocks - 1 && qt + 1 < qt1) {
                                 // the last scores of this tile exist, so its query rows are no longer
                                 // needed: fetch the next tile's behind the P V products
                                 mbar_expect_tx(q_bar, AQ_BYTES);
@@ -386,7 +390,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (lane == 0) mbar_arrive(r_bar);
             ++step;
         };
-        for (int qt = 0; qt < args.n_qtiles && ok; ++qt) {
+        for (int qt = qt0; qt < qt1 && ok; ++qt) {
             const int q_row = qt * AQ + quarter * 32 + lane;
             const bool warp_active = qt * AQ + quarter * 32 < T;      // else: no row of this warp exists
             float m = -INFINITY, l = 0.f;
@@ -472,6 +476,9 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
     a.tpad = (tokens + 15) / 16 * 16;
     a.n_blocks = (a.tpad + AKB - 1) / AKB;
     a.n_qtiles = (tokens + AQ - 1) / AQ;
+    // one key block: a CTA per head (three fit an SM).  Several key blocks: one CTA per SM, so each
+    // head's query tiles are spread over several CTAs when there are too few heads to fill the GPU.
+    a.q_split = (a.n_blocks > 1 && n_frames * heads < 4 * 148) ? a.n_qtiles : 1;
     // one block: P (104 columns) replaces S (208) and O takes columns 128..191 of the same 256;
     // several blocks: O must outlive the score blocks and sits in a second group of 256 columns
     a.tmem_cols = a.n_blocks == 1 ? 256u : 512u;
@@ -486,7 +493,7 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
         smem_set = smem;
     }
     ProfScope ps(L, KC_ATTENTION);
-    attention_tc_kernel<<<n_frames * heads, ATT_THREADS, smem, L.st>>>(tm_q, tm_kv, a);
+    attention_tc_kernel<<<n_frames * heads * a.q_split, ATT_THREADS, smem, L.st>>>(tm_q, tm_kv, a);
     BUMP(L);
     return cudaGetLastError();
 }
