@@ -472,7 +472,12 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
         if constexpr (TC) {
             const bool use_lora = lora && R.max_set > 0 && lo.n_adapted > 0;
             if (use_lora) {
-                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>(), h->n_sms, st);
+                // with LayerNorm folded in, the shrink computes the row statistics on its way through x
+                cudaError_t e = launch_shrink(L, lo.dev, R, tmx, (const bf16*)x, nrows, h->tbuf.as<bf16>(), h->n_sms,
+                                              nullptr, const_cast<float2*>(st), c.ln_eps);
+                if (e != cudaSuccess) return e;
+            } else if (st) {
+                cudaError_t e = launch_row_stats(L, (const bf16*)x, const_cast<float2*>(st), nrows, lo.dev.k_in, c.ln_eps);
                 if (e != cudaSuccess) return e;
             }
             const CUtensorMap* tmy = (void*)y == h->QKV.p ? &h->tm_y_qkv
@@ -491,8 +496,8 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     CK(launch_cls_rows<T>(L, h->cls.as<float>(), h->pos.as<float>(), X, n_frames, T_, d));
     for (int l = 0; l < c.layers; ++l) {
         if constexpr (TC) {
-            // LayerNorm 1 is folded into the qkv weights: only the row statistics are computed
-            CK(launch_row_stats(L, (const bf16*)X, h->ln_stats.as<float2>(), rows, d, c.ln_eps));
+            // LayerNorm 1 is folded into the qkv weights: only the row statistics are computed (by the
+            // shrink when there is one, else by a pass of their own)
             CK(linear(h->lin[l * 4 + 0], X, &h->tm_x_in, rows, T_, true, EPI_NONE, nullptr, none, QKV, h->ln_stats.as<float2>()));
         } else {
             CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
@@ -507,7 +512,6 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
         else CK(launch_attention_simple<T>(L, QKV, ATT, n_frames, T_, c.heads));
         CK(linear(h->lin[l * 4 + 1], ATT, &h->tm_att, rows, T_, true, EPI_RESIDUAL, X, none, X));
         if constexpr (TC) {
-            CK(launch_row_stats(L, (const bf16*)X, h->ln_stats.as<float2>(), rows, d, c.ln_eps));
             CK(linear(h->lin[l * 4 + 2], X, &h->tm_x_in, rows, T_, true, EPI_GELU, nullptr, none, Hb, h->ln_stats.as<float2>()));
         } else {
             CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
@@ -865,7 +869,7 @@ int pm_linear_forward(pm_linear l, const void* x, int n_frames, const int32_t* s
             err = "cuTensorMapEncodeTiled failed (y); y must be 16-byte aligned"; return PM_ERR_CUDA;
         }
         const bool lora = R.max_set > 0 && l->lin.dev.lora.At != nullptr;
-        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>(), l->n_sms, nullptr));
+        if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>(), l->n_sms, nullptr, nullptr, 0.f));
         CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, &tm_y, rows, l->epilogue,
                             (const bf16*)residual, none, (bf16*)y, l->n_sms, nullptr));
     } else {

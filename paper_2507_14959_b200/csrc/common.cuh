@@ -142,10 +142,12 @@ cudaError_t launch_naive_linear(const Launch& L, const LinearDev& lin, const Rou
                                 int tokens_per_frame, float* t32, int epi, const T* residual,
                                 const PatchEpi& pe, T* y);
 // tensor-core path (bf16): shrink into the slab buffer, then the fused GEMM
-// ln_stats: per-row (mean, 1/sqrt(var + eps)) of x, required iff lin.ln_g != null
+// A linear with LayerNorm folded in (lin.ln_g != null) needs per-row (mean, 1/sqrt(var + eps)) of x:
+// either ln_stats (already computed) or stats_out (the shrink computes them from the x tiles it
+// streams anyway, uses them and leaves them there for the GEMM), never both.
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
                           const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf, int n_sms,
-                          const float2* ln_stats);
+                          const float2* ln_stats, float2* stats_out, float ln_eps);
 cudaError_t launch_row_stats(const Launch& L, const bf16* x, float2* stats, int rows, int d, float eps);
 // tm_y: [rows, n_out] output map with a (32 x 32) box and 64B swizzle for the TMA-store epilogue, or
 // null to store straight from registers (always the case for EPI_PATCH, whose rows are remapped)

@@ -704,9 +704,14 @@ struct ShrinkArgs {
     // LayerNorm folded into the adapters (x is the raw residual stream, the arena holds gamma o A):
     //   t = s (rstd (x A' - mean c1) + c2);  stored divided by rstd, because the fused GEMM applies
     //   rstd to its whole accumulator, base and LoRA part alike
-    const float2* ln_stats;     // null = not folded
+    const float2* ln_stats;     // null = not folded, or the statistics are computed here (stats_out)
     const float* ln_c1;
     const float* ln_c2;
+    // Statistics mode: the epilogue warps also read every x tile as it passes through shared memory
+    // and produce each row's (mean, 1/sqrt(var + eps)) -- used for t right away and written to
+    // stats_out for the GEMM that follows.  Every row tile is then visited, with or without slabs.
+    float2* stats_out;
+    float ln_eps;
 };
 
 constexpr int SHRINK_MAX_STAGES = 4;
@@ -735,9 +740,14 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = args.k_in / BK;
+    const bool stats = args.stats_out != nullptr;
+    // groups of slabs of a tile; in statistics mode a tile without slabs still makes one pass over x
+    auto n_groups = [&](int ns) { return stats && ns == 0 ? 1 : (ns + args.sg - 1) / args.sg; };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        // a stage is free again when its MMAs are done and, in statistics mode, the four epilogue warps
+        // have read it too
+        for (int s = 0; s < STG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), stats ? 5 : 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -761,8 +771,9 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
                 const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
                 const int ns = args.tile_nslabs[tile];
-                for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
-                    const int cnt = min(args.sg, ns - g0);
+                for (int g = 0; g < n_groups(ns) && ok; ++g) {
+                    const int g0 = g * args.sg;
+                    const int cnt = max(0, min(args.sg, ns - g0));
                     for (int kb = 0; kb < num_kb && ok; ++kb) {
                         ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
                         if (!ok) break;
@@ -789,8 +800,18 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
                 const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
                 const int ns = args.tile_nslabs[tile];
-                for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
-                    const int cnt = min(args.sg, ns - g0);
+                for (int g = 0; g < n_groups(ns) && ok; ++g) {
+                    const int g0 = g * args.sg;
+                    const int cnt = max(0, min(args.sg, ns - g0));
+                    if (cnt == 0) {            // statistics only: hand the stages straight back
+                        for (int kb = 0; kb < num_kb && ok; ++kb) {
+                            ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                            if (!ok) break;
+                            mbar_arrive(empty_bar(stage));
+                            if (++stage == STG) { stage = 0; phase ^= 1u; }
+                        }
+                        continue;
+                    }
                     const uint32_t idesc = instr_desc(cnt * PM_SLAB);
                     ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, args.status);
                     if (!ok) break;
@@ -819,20 +840,64 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;
         const int r = quarter * 32 + lane;
-        int acc = 0;
-        uint32_t acc_phase = 0;
+        int acc = 0, stage = 0;
+        uint32_t acc_phase = 0, phase = 0;
         bool ok = true;
         for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
             const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
             const int ns = args.tile_nslabs[tile];
-            for (int g0 = 0; g0 < ns && ok; g0 += args.sg) {
-                const int cnt = min(args.sg, ns - g0);
+            float mean = 0.f, inv_rstd = 0.f;
+            for (int g = 0; g < n_groups(ns) && ok; ++g) {
+                const int g0 = g * args.sg;
+                const int cnt = max(0, min(args.sg, ns - g0));
+                if (stats) {
+                    // follow the ring: on the tile's first pass every thread sums its row of each x block
+                    // (shifted by the row's first element, which keeps the sum of squares well conditioned)
+                    float pivot = 0.f, s1 = 0.f, s2 = 0.f;
+                    for (int kb = 0; kb < num_kb && ok; ++kb) {
+                        ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                        ok = __all_sync(0xFFFFFFFFu, ok);
+                        if (!ok) break;
+                        if (g == 0) {
+                            const uint32_t row_addr = base + stage * stage_bytes + r * 128;
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                uint4 q;
+                                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w)
+                                             : "r"(row_addr + ((c ^ (r & 7)) << 4)));
+                                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+                                if (kb == 0 && c == 0) pivot = __uint_as_float(w[0] << 16);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float a0 = __uint_as_float(w[e] << 16) - pivot;
+                                    const float a1 = __uint_as_float(w[e] & 0xFFFF0000u) - pivot;
+                                    s1 += a0 + a1;
+                                    s2 = fmaf(a0, a0, fmaf(a1, a1, s2));
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(empty_bar(stage));
+                        if (++stage == STG) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    if (g == 0) {
+                        const float inv_d = 1.f / (float)args.k_in;
+                        const float m1 = s1 * inv_d;
+                        const float var = fmaxf(s2 * inv_d - m1 * m1, 0.f);
+                        const float rstd = rsqrtf(var + args.ln_eps);
+                        mean = pivot + m1;
+                        inv_rstd = 1.f / rstd;
+                        if (tile * BM + r < args.rows) args.stats_out[tile * BM + r] = make_float2(mean, rstd);
+                    }
+                    if (cnt == 0) continue;
+                }
                 ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, args.status);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * args.acc_cols;
-                float mean = 0.f, inv_rstd = 0.f;
                 if (args.ln_stats && tile * BM + r < args.rows) {
                     const float2 st = args.ln_stats[tile * BM + r];
                     mean = st.x;
@@ -845,7 +910,7 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     tmem_ld_wait();
                     const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
                     const float sc = on ? args.tile_scale[slot] : 0.f;
-                    if (args.ln_stats) {
+                    if (args.ln_stats || stats) {
                         const float* c1 = args.ln_c1 + (size_t)args.tile_slab[slot] * PM_SLAB;
                         const float* c2 = args.ln_c2 + (size_t)args.tile_slab[slot] * PM_SLAB;
 #pragma unroll
@@ -938,8 +1003,9 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
                           const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int n_sms,
-                          const float2* ln_stats) {
-    if (R.n_tiles <= 0 || R.slab_cap <= 0) return cudaSuccess;
+                          const float2* ln_stats, float2* stats_out, float ln_eps) {
+    if (R.n_tiles <= 0) return cudaSuccess;
+    if (R.slab_cap <= 0) return stats_out ? cudaErrorInvalidValue : cudaSuccess;   // nothing to shrink
     ShrinkArgs a;
     a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap; a.n_tiles = R.n_tiles;
     // groups of at most 8 slabs: two 128-column accumulators per CTA, so two CTAs share an SM's TMEM
@@ -952,8 +1018,10 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     a.stages = (4 * stage_bytes + 256 <= 112 * 1024) ? 4 : 3;
     a.tile_nslabs = R.tile_nslabs; a.tile_slab = R.tile_slab; a.tile_scale = R.tile_scale;
     a.tile_mask = R.tile_mask; a.tbuf = tbuf; a.status = L.status;
-    if ((lin.ln_g != nullptr) != (ln_stats != nullptr)) return cudaErrorInvalidValue;
+    // a linear with LayerNorm folded in gets the row statistics either ready-made or computed here
+    if ((lin.ln_g != nullptr) != ((ln_stats != nullptr) != (stats_out != nullptr))) return cudaErrorInvalidValue;
     a.ln_stats = ln_stats; a.ln_c1 = lin.ln_c1; a.ln_c2 = lin.ln_c2;
+    a.stats_out = stats_out; a.ln_eps = ln_eps;
     // x larger than the L2 cache was written front to back by the kernel before this one, so its tail
     // is what the cache still holds: start there, and leave the front in the cache for the GEMM that
     // follows (which walks front to back)
