@@ -12,6 +12,8 @@ What follows the paper and where:
                        without merging; the adapter scaling (alpha / r, Sec. 4: r = 16, alpha = 32).
   * forward_frame      the cited ViT/DeiT encoder (pre-LN blocks, CLS token, learned positions),
                        every linear of every block being a lora_linear (Fig. 2a).
+  * forward_branched   Fig. 2b / Fig. 5b read literally: the base model and each active adapter are
+                       separate branches over the frame, merged at the end.
   * heads / compose    Sec. 4 (one head per adapter over its class subset), Fig. 5b (active outputs
                        merged), Sec. 3.2 (base prediction over the full label space).
   * detect_contexts    Algorithm 2, step by step.
@@ -158,6 +160,30 @@ def forward(backbone, adapters, frames, set_offsets, set_ids, heads, patch, ln_e
         base[f] = sigmoid(z @ np.asarray(backbone["head_w"], dtype=dtype)
                           + np.asarray(backbone["head_b"], dtype=dtype))
         scores[f] = compose_scores(z, act, n_classes)
+    return scores, base
+
+
+def forward_branched(backbone, adapters, frames, set_offsets, set_ids, heads, patch, ln_eps, n_classes,
+                     dtype=np.float64):
+    """The per-adapter-branch reading of Fig. 2b / Fig. 5b: the base model and every active adapter
+    process the frame as separate models (each adapter alone on top of the shared backbone), every
+    adapter's head reads its own branch, and the branch outputs are merged as in compose_scores.
+
+    base_scores[f] comes from the branch without any adapter (the plain base model of Sec. 3.2);
+    scores[f, k] = max over active adapters a listing k of adapter a's own score, 0 otherwise.
+    Nothing is shared between branches here: each one is a complete forward of its own, so the
+    result does not depend on where an implementation lets the branches split.
+    """
+    F = len(set_offsets) - 1
+    scores = np.zeros((F, n_classes), dtype=dtype)
+    base = np.zeros((F, n_classes), dtype=dtype)
+    for f in range(F):
+        z0 = cls_feature(backbone, frames[f], [], heads, patch, ln_eps, dtype)
+        base[f] = sigmoid(z0 @ np.asarray(backbone["head_w"], dtype=dtype)
+                          + np.asarray(backbone["head_b"], dtype=dtype))
+        for i in sorted(int(i) for i in set_ids[set_offsets[f]:set_offsets[f + 1]]):
+            za = cls_feature(backbone, frames[f], [adapters[i]], heads, patch, ln_eps, dtype)
+            scores[f] = np.maximum(scores[f], compose_scores(za, [adapters[i]], n_classes))
     return scores, base
 
 

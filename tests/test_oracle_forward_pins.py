@@ -237,6 +237,56 @@ def test_compose_hand_case():
     np.testing.assert_allclose(po.compose_scores(z, [a1, a0], 6), s, atol=0)
 
 
+def test_branched_forward_equals_distinct_merged_models():
+    """Sec. 3.1: merging the adapters means instantiating one distinct model per adapter.  The
+    branch reading (Fig. 2b, Fig. 5b) must therefore equal: the plain base model for the base
+    scores, and for every active adapter a plain model with W + s A B (brute force) whose feature
+    feeds that adapter's own head; maximum where two active adapters list a class."""
+    spec = small_spec(n_classes=10)
+    name = "pin_branch"
+    bb = wl.make_backbone(name, spec)
+    # overlapping class lists so that the merge matters: {0..4}, {3..7}, {6..9}
+    ads = [wl.make_adapter(name, spec, a, r, np.arange(lo, hi), ab_std=0.2)
+           for a, (r, lo, hi) in enumerate([(4, 0, 5), (8, 3, 8), (2, 6, 10)])]
+    frames = wl.make_frames(name, spec, 3)
+    sets = [[0, 1], [], [2, 0, 1]]
+    off, ids = wl.sets_to_csr(sets)
+    s, b = po.forward_branched(bb, ads, frames, off, ids, spec.heads, spec.patch, spec.ln_eps,
+                               spec.n_classes)
+    sg = lambda t: 1.0 / (1.0 + math.exp(-t))
+    for f, st in enumerate(sets):
+        z0 = po.cls_feature(bb, frames[f], [], spec.heads, spec.patch, spec.ln_eps)
+        want_b = [sg(float(z0 @ bb["head_w"][:, k].astype(np.float64) + bb["head_b"][k]))
+                  for k in range(spec.n_classes)]
+        np.testing.assert_allclose(b[f], want_b, atol=1e-12)
+        want = np.zeros(spec.n_classes)
+        for a in st:
+            za = po.cls_feature(merged_backbone(spec, bb, [ads[a]]), frames[f], [], spec.heads,
+                                spec.patch, spec.ln_eps)
+            for j, k in enumerate(ads[a].class_ids):
+                v = sg(float(za @ ads[a].head_w[:, j].astype(np.float64) + ads[a].head_b[j]))
+                want[k] = max(want[k], v)
+        np.testing.assert_allclose(s[f], want, atol=1e-10)
+    # it is a different function from the one-stream forward whenever two adapters are active ...
+    s1, b1 = po.forward(bb, ads, frames, off, ids, spec.heads, spec.patch, spec.ln_eps, spec.n_classes)
+    assert np.abs(s1[0] - s[0]).max() > 1e-4 and np.abs(b1[0] - b[0]).max() > 1e-4
+    # ... and the same function for a frame without adapters
+    np.testing.assert_array_equal(s1[1], s[1])
+    np.testing.assert_array_equal(b1[1], b[1])
+
+
+def test_branched_forward_single_adapter_equals_one_stream_scores():
+    spec, bb, ads = small_model()
+    frames = wl.make_frames("pin_small", spec, 2)
+    off, ids = wl.sets_to_csr([[1], [2]])
+    s, b = po.forward_branched(bb, ads, frames, off, ids, spec.heads, spec.patch, spec.ln_eps, spec.n_classes)
+    s1, _ = po.forward(bb, ads, frames, off, ids, spec.heads, spec.patch, spec.ln_eps, spec.n_classes)
+    off0, ids0 = wl.sets_to_csr([[], []])
+    _, b0 = po.forward(bb, ads, frames, off0, ids0, spec.heads, spec.patch, spec.ln_eps, spec.n_classes)
+    np.testing.assert_allclose(s, s1, atol=1e-13)
+    np.testing.assert_allclose(b, b0, atol=1e-13)
+
+
 # ---------------------------------------------------------------- Table 2
 def read_table2():
     rows = {}
