@@ -124,6 +124,23 @@ int pm_forward(pm_handle h, const void* frames, int n_frames,
                const int32_t* set_offsets, const int32_t* set_ids,
                float* scores_out, float* base_out, void* cuda_stream);
 
+/* The same forward in the per-branch arrangement of Fig. 2b / Fig. 5b (Sec. 3.1, Sec. 3.2): the
+ * first trunk_layers blocks run once per frame without any adapter; from there the base model and
+ * every active adapter continue as separate branches (one adapter alone per branch) through the
+ * remaining blocks; each adapter's head reads its own branch, the base head reads the base branch,
+ * and the branch outputs are merged as in pm_forward (maximum per class, 0 where no active adapter
+ * lists the class).  Arguments as for pm_forward, plus
+ *   trunk_layers  in [0, layers]: blocks shared by all branches.  No registered adapter may carry
+ *                 A/B for a block below trunk_layers (the paper adapts the last 20 % of the blocks).
+ *   base_out      dev fp32 [n_frames, n_classes] or NULL; with NULL no base branch is computed.
+ * Capacity: n_frames + sum_f |S_f| branch slots when base_out is given, n_frames + sum_f max(|S_f|-1, 0)
+ * without it; the total must not exceed max_frames.
+ * Errors: as pm_forward, plus PM_ERR_STATE (an adapter touches a trunk block), PM_ERR_ARG
+ * (trunk_layers out of range), PM_ERR_CAPACITY (too many branches).  No kernel is launched on error. */
+int pm_forward_branched(pm_handle h, const void* frames, int n_frames,
+                        const int32_t* set_offsets, const int32_t* set_ids, int trunk_layers,
+                        float* scores_out, float* base_out, void* cuda_stream);
+
 /* Algorithm 2 (greedy context detection with conditional context copy) for n_frames streams.
  *   scores        dev fp32 [n_frames, n_classes]; Y_t = {k : scores[k] > score_thr}
  *   context_copy  Algorithm 2's flag

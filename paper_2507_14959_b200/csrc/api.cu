@@ -188,11 +188,12 @@ struct Router {
     DevBuf blob;
     void* stage = nullptr;          // pinned host copy of the blob
     size_t blob_bytes = 0;
-    size_t off_perm = 0, off_soff = 0, off_sids = 0, off_tn = 0, off_ts = 0, off_tsc = 0, off_tm = 0;
+    size_t off_perm = 0, off_soff = 0, off_sids = 0, off_src = 0, off_tn = 0, off_ts = 0, off_tsc = 0, off_tm = 0;
     cudaEvent_t uploaded = nullptr;
     bool upload_pending = false;
     RouteDev dev;
     std::vector<int32_t> last_off, last_ids;
+    std::vector<int> last_fixed;     // frame_of_slot then src_of_slot of the cached plan (branched forward)
     int last_frames = -1;
     bool last_sorted = false;
     std::vector<int> perm_host;
@@ -212,6 +213,7 @@ struct Router {
         take(off_perm, sizeof(int) * max_frames);
         take(off_soff, sizeof(int) * (max_frames + 1));
         take(off_sids, sizeof(int) * std::max(1, max_frames * max_set));
+        take(off_src, sizeof(int) * max_frames);
         take(off_tn, sizeof(int) * max_tiles);
         take(off_ts, sizeof(int) * std::max(1, max_tiles * slab_cap));
         take(off_tsc, sizeof(float) * std::max(1, max_tiles * slab_cap));
@@ -223,6 +225,7 @@ struct Router {
         CK(cudaEventCreateWithFlags(&uploaded, cudaEventDisableTiming));
         uint8_t* b = blob.as<uint8_t>();
         dev.perm = (int*)(b + off_perm); dev.slot_off = (int*)(b + off_soff); dev.slot_ids = (int*)(b + off_sids);
+        dev.src_slot = (int*)(b + off_src);
         dev.tile_nslabs = (int*)(b + off_tn); dev.tile_slab = (int*)(b + off_ts);
         dev.tile_scale = (float*)(b + off_tsc); dev.tile_mask = (uint32_t*)(b + off_tm);
         dev.tokens = tokens; dev.slab_cap = slab_cap;
@@ -230,8 +233,12 @@ struct Router {
     }
 
     // offsets/ids: host CSR.  ranks[a] == 0 means "not registered".
+    // frame_of_slot / src_of_slot (both or neither, n_frames entries, sort_frames false): the CSR is
+    // already in slot order; slot i reports to output row frame_of_slot[i] and starts from the trunk
+    // rows of slot src_of_slot[i] (the branched forward's plan).
     int build(int n_frames, const int32_t* offsets, const int32_t* ids, const std::vector<int>& ranks,
-              const std::vector<float>& scales, bool sort_frames, cudaStream_t st, std::string& err) {
+              const std::vector<float>& scales, bool sort_frames, cudaStream_t st, std::string& err,
+              const int* frame_of_slot = nullptr, const int* src_of_slot = nullptr) {
         if (n_frames < 0 || (n_frames > 0 && (!offsets))) { err = "bad frame count or NULL set_offsets"; return PM_ERR_ARG; }
         if (n_frames > max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
         if (n_frames > 0 && offsets[0] != 0) { err = "set_offsets[0] must be 0"; return PM_ERR_ARG; }
@@ -242,9 +249,14 @@ struct Router {
         const int nnz = n_frames > 0 ? offsets[n_frames] : 0;
         if (nnz > 0 && !ids) { err = "NULL set_ids"; return PM_ERR_ARG; }
         // unchanged sets (the common case: temporal continuity) reuse the uploaded plan
+        const bool fixed = frame_of_slot != nullptr;
+        if (fixed && (!src_of_slot || sort_frames)) { err = "inconsistent slot plan"; return PM_ERR_ARG; }
         if (n_frames == last_frames && sort_frames == last_sorted && (int)last_ids.size() == nnz &&
             std::equal(offsets, offsets + n_frames + 1, last_off.begin()) &&
-            std::equal(ids, ids + nnz, last_ids.begin()))
+            std::equal(ids, ids + nnz, last_ids.begin()) &&
+            last_fixed.size() == (fixed ? (size_t)2 * n_frames : 0) &&
+            (!fixed || (std::equal(frame_of_slot, frame_of_slot + n_frames, last_fixed.begin()) &&
+                        std::equal(src_of_slot, src_of_slot + n_frames, last_fixed.begin() + n_frames))))
             return PM_OK;
         std::vector<std::vector<int>> sets(n_frames);
         int widest = 0;
@@ -267,12 +279,14 @@ struct Router {
         if (upload_pending) { CK(cudaEventSynchronize(uploaded)); upload_pending = false; }
         uint8_t* s = (uint8_t*)stage;
         int* h_perm = (int*)(s + off_perm); int* h_soff = (int*)(s + off_soff); int* h_sids = (int*)(s + off_sids);
+        int* h_src = (int*)(s + off_src);
         int* h_tn = (int*)(s + off_tn); int* h_ts = (int*)(s + off_ts);
         float* h_tsc = (float*)(s + off_tsc); uint32_t* h_tm = (uint32_t*)(s + off_tm);
         h_soff[0] = 0;
         for (int i = 0; i < n_frames; ++i) {
             const std::vector<int>& st_ = sets[perm_host[i]];
-            h_perm[i] = perm_host[i];
+            h_perm[i] = fixed ? frame_of_slot[i] : perm_host[i];
+            h_src[i] = fixed ? src_of_slot[i] : i;
             std::copy(st_.begin(), st_.end(), h_sids + h_soff[i]);
             h_soff[i + 1] = h_soff[i] + (int)st_.size();
         }
@@ -312,6 +326,11 @@ struct Router {
         dev.n_frames = n_frames; dev.n_tiles = n_tiles; dev.max_set = widest;
         last_off.assign(offsets, offsets + n_frames + 1);
         last_ids.assign(ids, ids + nnz);
+        last_fixed.clear();
+        if (fixed) {
+            last_fixed.assign(frame_of_slot, frame_of_slot + n_frames);
+            last_fixed.insert(last_fixed.end(), src_of_slot, src_of_slot + n_frames);
+        }
         last_frames = n_frames; last_sorted = sort_frames;
         return PM_OK;
     }
@@ -451,12 +470,17 @@ int encode_activation_maps(pm_handle_s* h, int rows) {
     return PM_OK;
 }
 
+// n_frames frames enter; the first trunk_layers blocks run on them without adapters; then every
+// frame's rows are copied to its further slots (n_slots >= n_frames in all; slot i < n_frames is
+// frame perm[i] itself) and the remaining blocks and the heads run on all slots with the plan's
+// per-slot adapter sets.  The one-stream forward is trunk_layers = 0, n_slots = n_frames.
 template <typename T>
-int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_out, float* base_out,
-              cudaStream_t st) {
+int forward_t(pm_handle_s* h, const void* frames, int n_frames, int n_slots, int trunk_layers,
+              float* scores_out, float* base_out, cudaStream_t st) {
     std::string& err = h->err;
     const pm_config& c = h->cfg;
-    const int T_ = h->tokens, d = c.d, rows = n_frames * T_;
+    const int T_ = h->tokens, d = c.d;
+    int rows = n_frames * T_;
     Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
     const RouteDev& R = h->router.dev;
     constexpr bool TC = sizeof(T) == 2;
@@ -494,32 +518,42 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, float* scores_ou
     CK(launch_im2col<T>(L, (const T*)frames, R.perm, P, n_frames, c.img, c.patch));
     CK(linear(h->patch, P, &h->tm_patch, n_frames * h->g2, h->g2, false, EPI_PATCH, nullptr, pe, X));
     CK(launch_cls_rows<T>(L, h->cls.as<float>(), h->pos.as<float>(), X, n_frames, T_, d));
-    for (int l = 0; l < c.layers; ++l) {
+    int n_cur = n_frames;                     // slots the blocks currently run on
+    for (int l = 0; l <= c.layers; ++l) {
+        if (l == trunk_layers && n_slots != n_cur) {
+            // end of the shared trunk: every further slot starts from its frame's rows
+            CK(launch_fanout_rows<T>(L, X, R.src_slot, n_frames, n_slots, T_, d));
+            n_cur = n_slots;
+            rows = n_slots * T_;
+            if (TC) { int rc = encode_activation_maps(h, rows); if (rc) return rc; }
+        }
+        if (l == c.layers) break;
+        const bool lora = l >= trunk_layers;
         if constexpr (TC) {
             // LayerNorm 1 is folded into the qkv weights: only the row statistics are computed (by the
             // shrink when there is one, else by a pass of their own)
-            CK(linear(h->lin[l * 4 + 0], X, &h->tm_x_in, rows, T_, true, EPI_NONE, nullptr, none, QKV, h->ln_stats.as<float2>()));
+            CK(linear(h->lin[l * 4 + 0], X, &h->tm_x_in, rows, T_, lora, EPI_NONE, nullptr, none, QKV, h->ln_stats.as<float2>()));
         } else {
             CK(launch_layernorm<T>(L, X, h->ln1_g.as<float>() + (size_t)l * d, h->ln1_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
-            CK(linear(h->lin[l * 4 + 0], U, nullptr, rows, T_, true, EPI_NONE, nullptr, none, QKV));
+            CK(linear(h->lin[l * 4 + 0], U, nullptr, rows, T_, lora, EPI_NONE, nullptr, none, QKV));
         }
         if constexpr (TC) {
             if (attention_tc_supported(T_))
-                CK(launch_attention_tc(L, h->tm_att_q, h->tm_att_kv, (bf16*)ATT, n_frames, T_, c.heads));
+                CK(launch_attention_tc(L, h->tm_att_q, h->tm_att_kv, (bf16*)ATT, n_cur, T_, c.heads));
             else
-                CK(launch_attention_mma(L, (const bf16*)QKV, (bf16*)ATT, n_frames, T_, c.heads));
+                CK(launch_attention_mma(L, (const bf16*)QKV, (bf16*)ATT, n_cur, T_, c.heads));
         }
-        else CK(launch_attention_simple<T>(L, QKV, ATT, n_frames, T_, c.heads));
-        CK(linear(h->lin[l * 4 + 1], ATT, &h->tm_att, rows, T_, true, EPI_RESIDUAL, X, none, X));
+        else CK(launch_attention_simple<T>(L, QKV, ATT, n_cur, T_, c.heads));
+        CK(linear(h->lin[l * 4 + 1], ATT, &h->tm_att, rows, T_, lora, EPI_RESIDUAL, X, none, X));
         if constexpr (TC) {
-            CK(linear(h->lin[l * 4 + 2], X, &h->tm_x_in, rows, T_, true, EPI_GELU, nullptr, none, Hb, h->ln_stats.as<float2>()));
+            CK(linear(h->lin[l * 4 + 2], X, &h->tm_x_in, rows, T_, lora, EPI_GELU, nullptr, none, Hb, h->ln_stats.as<float2>()));
         } else {
             CK(launch_layernorm<T>(L, X, h->ln2_g.as<float>() + (size_t)l * d, h->ln2_b.as<float>() + (size_t)l * d, U, rows, d, c.ln_eps));
-            CK(linear(h->lin[l * 4 + 2], U, nullptr, rows, T_, true, EPI_GELU, nullptr, none, Hb));
+            CK(linear(h->lin[l * 4 + 2], U, nullptr, rows, T_, lora, EPI_GELU, nullptr, none, Hb));
         }
-        CK(linear(h->lin[l * 4 + 3], Hb, &h->tm_h, rows, T_, true, EPI_RESIDUAL, X, none, X));
+        CK(linear(h->lin[l * 4 + 3], Hb, &h->tm_h, rows, T_, lora, EPI_RESIDUAL, X, none, X));
     }
-    CK(launch_heads<T>(L, X, n_frames, T_, d, c.ln_eps, h->lnf_g.as<float>(), h->lnf_b.as<float>(),
+    CK(launch_heads<T>(L, X, n_slots, n_frames, n_frames, T_, d, c.ln_eps, h->lnf_g.as<float>(), h->lnf_b.as<float>(),
                        h->Z.as<float>(), h->head_wt.as<T>(), h->head_b.as<float>(), c.n_classes,
                        h->hcat.as<T>(), h->hbias.as<float>(), h->hcls.as<int>(), h->hoff.as<int>(), R,
                        scores_out, base_out));
@@ -719,8 +753,72 @@ int pm_forward(pm_handle h, const void* frames, int n_frames, const int32_t* set
         rc = h->cfg.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
         if (rc) return rc;
     }
-    return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, scores_out, base_out, st)
-                             : forward_t<float>(h, frames, n_frames, scores_out, base_out, st);
+    return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
+                             : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
+}
+
+int pm_forward_branched(pm_handle h, const void* frames, int n_frames, const int32_t* set_offsets,
+                        const int32_t* set_ids, int trunk_layers, float* scores_out, float* base_out,
+                        void* cuda_stream) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    const pm_config& c = h->cfg;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (n_frames < 0 || (n_frames > 0 && (!frames || !set_offsets || !scores_out))) { err = "NULL argument"; return PM_ERR_ARG; }
+    if (trunk_layers < 0 || trunk_layers > c.layers) { err = "trunk_layers out of range"; return PM_ERR_ARG; }
+    if (n_frames == 0) return PM_OK;
+    if (n_frames > c.max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
+    for (int i = 0; i < trunk_layers * 4; ++i)
+        if (h->lin[i].n_adapted > 0) { err = "a registered adapter touches a block of the shared trunk"; return PM_ERR_STATE; }
+    std::vector<int32_t> hoff, hids;
+    const int32_t *o, *ids;
+    int rc = fetch_csr(set_offsets, set_ids, n_frames, st, hoff, hids, &o, &ids, err);
+    if (rc) return rc;
+    if (o[0] != 0) { err = "set_offsets[0] must be 0"; return PM_ERR_ARG; }
+    for (int f = 0; f < n_frames; ++f) {
+        if (o[f + 1] < o[f]) { err = "set_offsets not monotone"; return PM_ERR_ARG; }
+        if (o[f + 1] - o[f] > c.max_set) { err = "a frame has more adapters than max_set"; return PM_ERR_CAPACITY; }
+    }
+    if (o[n_frames] > 0 && !ids) { err = "NULL set_ids"; return PM_ERR_ARG; }
+    // slots [0, F): the frames themselves, in caller order (the trunk's rows); they carry the base
+    // branch when base scores are wanted, else the frame's lowest adapter.  Every other (frame,
+    // adapter) branch gets a slot of its own behind them, grouped by adapter so that neighbouring
+    // rows share LoRA slabs.
+    std::vector<std::pair<int, int>> extra;          // (adapter, frame)
+    std::vector<int32_t> boff(1, 0), bids;
+    std::vector<int> fos, src;
+    for (int f = 0; f < n_frames; ++f) {
+        std::vector<int> s(ids + o[f], ids + o[f + 1]);
+        std::sort(s.begin(), s.end());
+        for (size_t i = 0; i < s.size(); ++i) {
+            if (s[i] < 0 || s[i] >= c.max_adapters) { err = "adapter id out of range"; return PM_ERR_ARG; }
+            if (i > 0 && s[i - 1] == s[i]) { err = "duplicate adapter id in a frame's set"; return PM_ERR_ARG; }
+            if (h->ranks[s[i]] == 0) { err = "adapter id not registered"; return PM_ERR_STATE; }
+        }
+        size_t first_extra = 0;
+        if (!base_out && !s.empty()) { bids.push_back(s[0]); first_extra = 1; }
+        boff.push_back((int32_t)bids.size());
+        fos.push_back(f); src.push_back(f);
+        for (size_t i = first_extra; i < s.size(); ++i) extra.emplace_back(s[i], f);
+    }
+    std::sort(extra.begin(), extra.end());
+    const long long n_slots = (long long)n_frames + (long long)extra.size();
+    if (n_slots > c.max_frames) { err = "frames plus adapter branches exceed max_frames"; return PM_ERR_CAPACITY; }
+    if (c.max_set < 1 && !extra.empty()) { err = "max_set is 0"; return PM_ERR_CAPACITY; }
+    for (auto& e : extra) {
+        bids.push_back(e.first); boff.push_back((int32_t)bids.size());
+        fos.push_back(e.second); src.push_back(e.second);
+    }
+    if (bids.empty()) bids.push_back(0);
+    rc = h->router.build((int)n_slots, boff.data(), bids.data(), h->ranks, h->scales, false, st, err,
+                         fos.data(), src.data());
+    if (rc) return rc;
+    if (h->heads_dirty) {
+        rc = c.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
+        if (rc) return rc;
+    }
+    return c.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st)
+                        : forward_t<float>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st);
 }
 
 int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, int context_copy,

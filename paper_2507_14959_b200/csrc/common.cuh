@@ -54,6 +54,7 @@ struct RouteDev {
     int* perm = nullptr;        // [F] slot -> caller's frame index
     int* slot_off = nullptr;    // [F+1] CSR over slots
     int* slot_ids = nullptr;    // [nnz] ascending adapter ids per slot
+    int* src_slot = nullptr;    // [F] branched forward only: the trunk slot whose rows a branch slot copies
     // tile plan (rows 128*t .. 128*t+127).  Tiles 2p and 2p+1 carry the SAME slab list, the union of
     // what the 256 rows of the pair need (the CTA-pair GEMM applies one slab to both halves); a
     // tile's mask is zero for a slab none of its rows uses.  n_tiles is even.
@@ -155,8 +156,15 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
                              const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
                              int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
                              int n_sms, const float2* ln_stats);
+// x rows of slots [first_slot, n_slots) <- x rows of slot src_slot[slot] (a slot below first_slot)
 template <typename T>
-cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, int d, float eps,
+cudaError_t launch_fanout_rows(const Launch& L, T* x, const int* src_slot, int first_slot, int n_slots,
+                               int tokens, int d);
+// n_slots CLS rows are normalised and feed the adapter heads of their slot; the first n_base_slots
+// also feed the base head; scores_out has n_out_frames rows (several slots may merge into one row)
+template <typename T>
+cudaError_t launch_heads(const Launch& L, const T* x, int n_slots, int n_out_frames, int n_base_slots,
+                         int tokens, int d, float eps,
                          const float* lnf_g, const float* lnf_b, float* z,
                          const T* base_wt, const float* base_b, int n_classes,
                          const T* hcat, const float* hbias, const int* hcls, const int* hoff,

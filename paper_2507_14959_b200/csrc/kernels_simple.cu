@@ -1,6 +1,8 @@
 // Memory-bound and small kernels of the Polymorph forward path: LayerNorm, patch gather, CLS rows,
 // segmented heads + sigmoid + merge, Algorithm 2 selection, and the plain CUDA-core kernels of
 // the fp32 debug build (linear with unmerged LoRA terms, attention).
+#include <algorithm>
+
 #include "common.cuh"
 
 #define BUMP(L) do { if ((L).launches) ++*(L).launches; } while (0)
@@ -411,6 +413,34 @@ template cudaError_t launch_attention_simple<float>(const Launch&, const float*,
 template cudaError_t launch_attention_simple<bf16>(const Launch&, const bf16*, bf16*, int, int, int);
 
 // ---------------------------------------------------------------------------------------
+// branched forward (Fig. 2b): the rows a frame has after the shared trunk are copied to the slots
+// of its adapter branches.  Source slots lie below first_slot, destinations at or above it.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) fanout_rows_kernel(T* __restrict__ x, const int* __restrict__ src_slot,
+                                                          int first_slot, size_t slot_vec) {
+    const int slot = first_slot + blockIdx.y;
+    const uint4* s = reinterpret_cast<const uint4*>(x) + (size_t)src_slot[slot] * slot_vec;
+    uint4* o = reinterpret_cast<uint4*>(x) + (size_t)slot * slot_vec;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < slot_vec; i += (size_t)gridDim.x * blockDim.x)
+        o[i] = s[i];
+}
+
+template <typename T>
+cudaError_t launch_fanout_rows(const Launch& L, T* x, const int* src_slot, int first_slot, int n_slots,
+                               int tokens, int d) {
+    if (n_slots <= first_slot) return cudaSuccess;
+    const size_t slot_vec = (size_t)tokens * d * sizeof(T) / 16;     // d is a multiple of 64
+    ProfScope ps(L, KC_OTHER);
+    dim3 grid((unsigned)std::min<size_t>((slot_vec + 255) / 256, 64), n_slots - first_slot);
+    fanout_rows_kernel<T><<<grid, 256, 0, L.st>>>(x, src_slot, first_slot, slot_vec);
+    BUMP(L);
+    return cudaGetLastError();
+}
+template cudaError_t launch_fanout_rows<float>(const Launch&, float*, const int*, int, int, int, int);
+template cudaError_t launch_fanout_rows<bf16>(const Launch&, bf16*, const int*, int, int, int, int);
+
+// ---------------------------------------------------------------------------------------
 // final LayerNorm on the CLS rows, base head, segmented adapter heads + sigmoid + merge
 // ---------------------------------------------------------------------------------------
 template <typename T>
@@ -496,32 +526,33 @@ __global__ void __launch_bounds__(256) adapter_heads_kernel(const float* __restr
 }
 
 template <typename T>
-cudaError_t launch_heads(const Launch& L, const T* x, int n_frames, int tokens, int d, float eps,
+cudaError_t launch_heads(const Launch& L, const T* x, int n_slots, int n_out_frames, int n_base_slots,
+                         int tokens, int d, float eps,
                          const float* lnf_g, const float* lnf_b, float* z,
                          const T* base_wt, const float* base_b, int n_classes,
                          const T* hcat, const float* hbias, const int* hcls, const int* hoff,
                          const RouteDev& R, float* scores_out, float* base_out) {
-    if (n_frames <= 0) return cudaSuccess;
+    if (n_slots <= 0) return cudaSuccess;
     ProfScope ps(L, KC_OTHER);
-    final_ln_kernel<T><<<(n_frames + 7) / 8, 256, 0, L.st>>>(x, lnf_g, lnf_b, z, n_frames, tokens, d, eps);
+    final_ln_kernel<T><<<(n_slots + 7) / 8, 256, 0, L.st>>>(x, lnf_g, lnf_b, z, n_slots, tokens, d, eps);
     BUMP(L);
-    if (base_out) {
-        dim3 grid((n_classes + 7) / 8, (n_frames + BASE_HEAD_FRAMES - 1) / BASE_HEAD_FRAMES);
-        base_head_kernel<T><<<grid, 256, 0, L.st>>>(z, base_wt, base_b, R.perm, d, n_classes, n_frames, base_out);
+    if (base_out && n_base_slots > 0) {
+        dim3 grid((n_classes + 7) / 8, (n_base_slots + BASE_HEAD_FRAMES - 1) / BASE_HEAD_FRAMES);
+        base_head_kernel<T><<<grid, 256, 0, L.st>>>(z, base_wt, base_b, R.perm, d, n_classes, n_base_slots, base_out);
         BUMP(L);
     }
-    cudaError_t e = cudaMemsetAsync(scores_out, 0, (size_t)n_frames * n_classes * sizeof(float), L.st);
+    cudaError_t e = cudaMemsetAsync(scores_out, 0, (size_t)n_out_frames * n_classes * sizeof(float), L.st);
     if (e != cudaSuccess) return e;
     if (R.max_set > 0) {
-        dim3 grid(R.max_set, n_frames);
+        dim3 grid(R.max_set, n_slots);
         adapter_heads_kernel<T><<<grid, 256, 0, L.st>>>(z, hcat, hbias, hcls, hoff, R.slot_off, R.slot_ids,
                                                        R.perm, d, n_classes, scores_out);
         BUMP(L);
     }
     return cudaGetLastError();
 }
-template cudaError_t launch_heads<float>(const Launch&, const float*, int, int, int, float, const float*, const float*, float*, const float*, const float*, int, const float*, const float*, const int*, const int*, const RouteDev&, float*, float*);
-template cudaError_t launch_heads<bf16>(const Launch&, const bf16*, int, int, int, float, const float*, const float*, float*, const bf16*, const float*, int, const bf16*, const float*, const int*, const int*, const RouteDev&, float*, float*);
+template cudaError_t launch_heads<float>(const Launch&, const float*, int, int, int, int, int, float, const float*, const float*, float*, const float*, const float*, int, const float*, const float*, const int*, const int*, const RouteDev&, float*, float*);
+template cudaError_t launch_heads<bf16>(const Launch&, const bf16*, int, int, int, int, int, float, const float*, const float*, float*, const bf16*, const float*, int, const bf16*, const float*, const int*, const int*, const RouteDev&, float*, float*);
 
 // ---------------------------------------------------------------------------------------
 // Algorithm 2 on the device: one warp per frame, any number of blocks
