@@ -64,6 +64,25 @@ def gemm_flops_per_step(w):
     return base + lora + patch
 
 
+def gemm_flops_per_step_branched(w, trunk_layers):
+    """The same count for the branched arrangement (Fig. 2b): the trunk blocks once per frame, the
+    remaining blocks once per branch (the base branch plus one per active adapter, each adapter
+    alone in its branch)."""
+    s = w.spec
+    T, d, m, L = s.tokens, s.d, s.mlp, s.layers
+    shapes = [(d, 3 * d), (d, d), (d, m), (m, d)]
+    F = w.n_frames
+    per_block = sum(2 * k * n for k, n in shapes) * T
+    branches = F + len(w.set_ids)
+    base = per_block * (F * trunk_layers + branches * (L - trunk_layers))
+    lora = 0
+    for a in w.set_ids:
+        ad = w.adapters[a]
+        for i, (k, n) in enumerate(shapes):
+            lora += 2 * (k + n) * T * ad.rank * sum(1 for l in range(trunk_layers, L) if ad.A[l * 4 + i] is not None)
+    return base + lora + 2 * s.patch_dim * d * (T - 1) * F
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -252,6 +271,10 @@ def main():
     ap.add_argument("--lora-last", type=int, default=None,
                     help="batch workload only: adapters touch the last N blocks only (the paper's cheap "
                          "placement); default: all blocks, the headline configuration")
+    ap.add_argument("--branched", action="store_true",
+                    help="batch workload with --lora-last N only: the paper's arrangement (Fig. 2b) -- the first "
+                         "layers-N blocks run once per frame, then the base model and every active adapter "
+                         "continue as separate branches (pm_forward_branched)")
     ap.add_argument("--workload", default="batch", choices=["batch", "streams"],
                     help="batch: ViT-base 224x224, 256 frames (the headline); streams: ViT-base 384x384, 16 streams "
                          "in closed loop (forward -> Algorithm 2 -> next forward), one step = one frame per stream")
@@ -282,7 +305,10 @@ def main():
         return
 
     w = wl.vit_base_batch(n_frames=args.frames, lora_last=args.lora_last)
-    m = binding.model_from_workload(w, dtype=0)
+    if args.branched and args.lora_last is None:
+        raise SystemExit("--branched needs --lora-last N (adapters may not touch the shared trunk)")
+    trunk = w.spec.layers - args.lora_last if args.branched else 0
+    m = binding.model_from_workload(w, dtype=0, max_frames=w.n_frames + (len(w.set_ids) if args.branched else 0))
     m.set_cover(w.tau)
     F, K = w.n_frames, w.spec.n_classes
     frames_host = torch.from_numpy(w.frames).to(torch.bfloat16).pin_memory()
@@ -298,7 +324,10 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step(i, frames=None):
-        m.forward(frames_dev if frames is None else frames, w.set_offsets, w.set_ids, scores, base)
+        if args.branched:
+            m.forward_branched(frames_dev if frames is None else frames, w.set_offsets, w.set_ids, trunk, scores, base)
+        else:
+            m.forward(frames_dev if frames is None else frames, w.set_offsets, w.set_ids, scores, base)
         prev, nxt = sel[i % 2], sel[(i + 1) % 2]
         m.select(base, 0.5, False, i > 0, labels, prev[0], prev[1], nxt[0], nxt[1])
 
@@ -383,7 +412,7 @@ def main():
     if rank == 0:
         peaks = measured_peaks()
         gemm_ms, gemm_sites = prof["gemm"]
-        flops = gemm_flops_per_step(w) * args.steps
+        flops = (gemm_flops_per_step_branched(w, trunk) if args.branched else gemm_flops_per_step(w)) * args.steps
         achieved = flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
         peak = peaks["bf16_tflops_sustained"]
         out = {
@@ -395,7 +424,9 @@ def main():
                                    "adapters over 800 classes, 1-3 active adapters per frame (60/30/10 %%), "
                                    "forward + Algorithm 2 select" % F,
                        "frames_per_gpu": F, "l2": "activations (~0.9 GB/step) exceed the 126 MB L2; no flush",
-                       "lora_blocks": "all 12" if args.lora_last is None else "last %d" % args.lora_last},
+                       "lora_blocks": "all 12" if args.lora_last is None else "last %d" % args.lora_last,
+                       "arrangement": ("branched: %d shared blocks, then %d branches for %d frames" %
+                                       (trunk, F + len(w.set_ids), F)) if args.branched else "one stream per frame"},
             "e2e": {"value": world * F * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(frames_host.numel() * 2),
                     "d2h_bytes_per_step": int(scores_host.numel() * 4 + base_host.numel() * 4)},
@@ -407,7 +438,7 @@ def main():
                          "peak_source": "bf16_tflops_sustained of %s" % peaks["source"],
                          "launches_timed": gemm_sites, "avg_launch_ms": gemm_ms / max(gemm_sites, 1),
                          "timed_in": "a second pass of the same K steps with CUDA events around each launch site",
-                         "traffic": GEMM_DRAM_TRAFFIC_BYTES},
+                         "traffic": None if args.branched else GEMM_DRAM_TRAFFIC_BYTES},
             "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
             "profiled_pass_ms_per_step": ms_profiled / args.steps,
         }
