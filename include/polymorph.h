@@ -141,6 +141,22 @@ int pm_forward_branched(pm_handle h, const void* frames, int n_frames,
                         const int32_t* set_offsets, const int32_t* set_ids, int trunk_layers,
                         float* scores_out, float* base_out, void* cuda_stream);
 
+/* pm_forward for adapter sets that already live on the device, e.g. the lists pm_select wrote
+ * (Algorithm 2 feeding the next frame, Sec. 3.2): the routing plan is built by kernels on the
+ * stream, nothing is copied to the host and the stream is not synchronised, so forward -> select ->
+ * forward runs without the host in between and the sequence can be recorded in a CUDA graph.
+ *   set_offsets, set_ids   dev int32, as for pm_forward; they are read when the kernels run
+ *   n_frames               at most PM_DEVICE_PLAN_MAX_FRAMES (and max_frames)
+ * The lists cannot be checked on the host: an id that is out of range, not registered or repeated
+ * is skipped, a frame with more than max_set ids keeps its max_set lowest, and the device status
+ * word is set (PM_ERR_ARG / PM_ERR_CAPACITY, read with pm_status).  Frames are bucketed by their
+ * first seven ids; results are the same as pm_forward's.
+ * Errors: PM_ERR_ARG (NULL), PM_ERR_CAPACITY (n_frames).  No kernel is launched on error. */
+#define PM_DEVICE_PLAN_MAX_FRAMES 2048
+int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames,
+                           const int32_t* set_offsets, const int32_t* set_ids,
+                           float* scores_out, float* base_out, void* cuda_stream);
+
 /* Algorithm 2 (greedy context detection with conditional context copy) for n_frames streams.
  *   scores        dev fp32 [n_frames, n_classes]; Y_t = {k : scores[k] > score_thr}
  *   context_copy  Algorithm 2's flag

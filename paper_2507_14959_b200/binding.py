@@ -20,7 +20,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
                -4: "PM_ERR_CUDA", -5: "PM_ERR_TIMEOUT", -6: "PM_ERR_OOM"}
 
 EXPORTS = [
-    "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_select",
+    "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
     "pm_select_static", "pm_status", "pm_last_error", "pm_launch_count", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention",
@@ -75,6 +75,7 @@ def load():
     lib.pm_destroy.argtypes = [vp]
     lib.pm_destroy.restype = None
     lib.pm_forward.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
+    lib.pm_forward_device_sets.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
     lib.pm_forward_branched.argtypes = [vp, vp, ip, vp, vp, ip, vp, vp, vp]
     lib.pm_select.argtypes = [vp, vp, ip, C.c_float, ip, ip, vp, vp, vp, vp, vp, ip, vp]
     lib.pm_select_static.argtypes = [vp, ip, ip, ip, C.c_float, ip, ip, vp, vp, vp, vp, vp, vp, vp, ip, vp, vp]
@@ -172,6 +173,13 @@ class Model:
             set_ids = np.ascontiguousarray(set_ids, dtype=np.int32)
         self._check(self.lib.pm_forward(self.handle, _ptr(frames), n, _ptr(set_offsets), _ptr(set_ids),
                                         _ptr(scores_out), _ptr(base_out), _stream_ptr(stream)), "pm_forward")
+
+    def forward_device_sets(self, frames, set_offsets, set_ids, scores_out, base_out=None, stream=None):
+        """pm_forward_device_sets: the set lists are torch CUDA int32 tensors (e.g. written by
+        select()); the plan is built on the device, nothing synchronises."""
+        self._check(self.lib.pm_forward_device_sets(self.handle, _ptr(frames), int(frames.shape[0]),
+                                                    _ptr(set_offsets), _ptr(set_ids), _ptr(scores_out),
+                                                    _ptr(base_out), _stream_ptr(stream)), "pm_forward_device_sets")
 
     def forward_branched(self, frames, set_offsets, set_ids, trunk_layers, scores_out, base_out=None, stream=None):
         """pm_forward_branched: shared trunk of `trunk_layers` blocks, then one branch per active

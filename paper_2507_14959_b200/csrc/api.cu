@@ -335,6 +335,19 @@ struct Router {
         return PM_OK;
     }
     void invalidate() { last_frames = -1; }
+
+    // The same tables built by kernels from a CSR on the device; the host never sees the sets, so
+    // max_set is the handle's upper bound and the cached host plan is forgotten.
+    int build_on_device(const Launch& L, int n_frames, const int32_t* d_off, const int32_t* d_ids,
+                        const AdapterMeta& meta, std::string& err) {
+        if (n_frames > max_frames || n_frames > PM_DEVICE_PLAN_MAX_FRAMES) { err = "n_frames exceeds the device planner's limit"; return PM_ERR_CAPACITY; }
+        invalidate();
+        dev.n_frames = n_frames;
+        dev.n_tiles = (int)(((long long)n_frames * tokens + 2 * PM_TILE_M - 1) / (2 * PM_TILE_M)) * 2;
+        dev.max_set = max_set;
+        CK(launch_device_plan(L, dev, n_frames, max_set, max_adapters, slabs_max, d_off, d_ids, meta));
+        return PM_OK;
+    }
 };
 
 // Copies a CSR that may live on the device to the host (synchronising the stream if it does).
@@ -753,6 +766,25 @@ int pm_forward(pm_handle h, const void* frames, int n_frames, const int32_t* set
         rc = h->cfg.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
         if (rc) return rc;
     }
+    return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
+                             : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
+}
+
+int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames, const int32_t* set_offsets,
+                           const int32_t* set_ids, float* scores_out, float* base_out, void* cuda_stream) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (n_frames < 0 || (n_frames > 0 && (!frames || !set_offsets || !set_ids || !scores_out))) { err = "NULL argument"; return PM_ERR_ARG; }
+    if (n_frames == 0) return PM_OK;
+    if (n_frames > h->cfg.max_frames) { err = "n_frames exceeds max_frames"; return PM_ERR_CAPACITY; }
+    if (h->heads_dirty) {
+        int rc = h->cfg.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
+        if (rc) return rc;
+    }
+    Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
+    int rc = h->router.build_on_device(L, n_frames, set_offsets, set_ids, h->meta, err);
+    if (rc) return rc;
     return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
                              : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
 }

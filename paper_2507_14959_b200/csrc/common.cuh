@@ -169,6 +169,10 @@ cudaError_t launch_heads(const Launch& L, const T* x, int n_slots, int n_out_fra
                          const T* base_wt, const float* base_b, int n_classes,
                          const T* hcat, const float* hbias, const int* hcls, const int* hoff,
                          const RouteDev& R, float* scores_out, float* base_out);
+// Builds the routing tables of R (perm, slot CSR, tile plan) on the device from a device CSR
+// (plan_device.cu).  Problems found in the lists go to the status word.
+cudaError_t launch_device_plan(const Launch& L, const RouteDev& R, int n_frames, int max_set, int max_adapters,
+                               int slabs_max, const int* off, const int* ids, const AdapterMeta& meta);
 cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, int n_classes,
                           int n_adapters, float thr, int context_copy, int has_prev,
                           uint32_t* prev_labels, const int* prev_off, const int* prev_ids,

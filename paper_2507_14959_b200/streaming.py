@@ -1,7 +1,10 @@
 """Closed-loop streaming driver: for every time step, one pm_forward over the current frame of each
 stream with the adapter sets chosen at the previous step, then pm_select (Algorithm 2) on the base
 scores to choose the sets for the next frame.  The scores never leave the device; the id lists
-produced by pm_select are handed straight back to pm_forward.
+produced by pm_select are handed straight back to the forward.  With ``device_plan`` (the default)
+the forward is pm_forward_device_sets, which also builds its routing plan on the device, so a step
+involves no host synchronisation at all and can be recorded once as a CUDA graph and replayed
+(``capture`` / ``step_graph``); without it pm_forward copies the lists to the host to plan there.
 
 Also counts the two stream-level metrics of the paper on the sets that were actually used:
 AvgCoverage (Eq. 7, mean number of active contexts per frame) and SwitchPenalty (Eq. 8, number of
@@ -16,9 +19,12 @@ class StreamRunner:
     """Owns the per-stream device state (previous label bit sets, two CSR buffers that alternate
     between "sets of this step" and "sets for the next step")."""
 
-    def __init__(self, model, n_streams, n_classes, n_adapters, score_thr=0.5, context_copy=False):
+    def __init__(self, model, n_streams, n_classes, n_adapters, score_thr=0.5, context_copy=False,
+                 device_plan=True):
         import torch
         self.model = model
+        self.device_plan = bool(device_plan)
+        self.graphs = None
         self.S = n_streams
         self.K = n_classes
         self.score_thr = float(score_thr)
@@ -40,10 +46,44 @@ class StreamRunner:
     def step(self, frames):
         """frames: device tensor [n_streams, 3, img, img].  Runs the forward with the current sets and
         selects the next ones.  Returns (scores, base_scores) device tensors (overwritten next step)."""
-        cur, nxt = self.csr[self.t % 2], self.csr[(self.t + 1) % 2]
-        self.model.forward(frames, cur[0], cur[1], self.scores, self.base)
-        self.model.select(self.base, self.score_thr, self.context_copy, self.t > 0, self.labels,
+        self._enqueue(frames, self.t % 2, self.t > 0)
+        self.t += 1
+        return self.scores, self.base
+
+    def _enqueue(self, frames, parity, has_prev):
+        cur, nxt = self.csr[parity], self.csr[1 - parity]
+        fwd = self.model.forward_device_sets if self.device_plan else self.model.forward
+        fwd(frames, cur[0], cur[1], self.scores, self.base)
+        self.model.select(self.base, self.score_thr, self.context_copy, has_prev, self.labels,
                           cur[0], cur[1], nxt[0], nxt[1])
+
+    def capture(self, frames_static):
+        """Records the step (forward from `frames_static`, then select) as two CUDA graphs, one per
+        parity of the alternating list buffers.  Needs device_plan and one eager step before it (so
+        that every kernel has been set up).  Afterwards: write the next frames into `frames_static`,
+        call step_graph()."""
+        import torch
+        if not self.device_plan:
+            raise ValueError("capture needs device_plan (the host planner synchronises the stream)")
+        self.static_frames = frames_static
+        self.graphs, self.graph_launches = [], []
+        for parity in (0, 1):
+            g = torch.cuda.CUDAGraph()
+            n0 = self.model.launch_count()
+            with torch.cuda.graph(g):
+                self._enqueue(frames_static, parity, True)
+            self.graphs.append(g)
+            self.graph_launches.append(self.model.launch_count() - n0)
+        self.replayed_launches = 0
+
+    def step_graph(self):
+        """Replays the recorded step on the frames currently in the static buffer (not the first
+        step of a stream: that one has no previous labels and runs through step())."""
+        if self.t == 0:
+            raise ValueError("the first step of a stream runs through step()")
+        p = self.t % 2
+        self.graphs[p].replay()
+        self.replayed_launches += self.graph_launches[p]
         self.t += 1
         return self.scores, self.base
 
@@ -69,18 +109,26 @@ def switch_penalty(sets_per_step):
     return total
 
 
-def run(model, frames_seq, n_classes, n_adapters, score_thr=0.5, context_copy=False, record=True):
-    """frames_seq: device tensor [n_streams, n_steps, 3, img, img].  Free-running loop over all steps.
-    Returns {"used_sets": per step the sets the forward used, "base": [n_steps, S, K] numpy,
+def run(model, frames_seq, n_classes, n_adapters, score_thr=0.5, context_copy=False, record=True,
+        device_plan=True, graph=False):
+    """frames_seq: device tensor [n_streams, n_steps, 3, img, img].  Free-running loop over all steps
+    (graph: steps after the first are CUDA-graph replays).  Returns {"used_sets": per step the sets the forward used, "base": [n_steps, S, K] numpy,
     "scores": same, "avg_coverage", "switch_penalty"} (records only if `record`)."""
     S, T = int(frames_seq.shape[0]), int(frames_seq.shape[1])
-    r = StreamRunner(model, S, n_classes, n_adapters, score_thr, context_copy)
+    r = StreamRunner(model, S, n_classes, n_adapters, score_thr, context_copy, device_plan)
     r.reset()
     used, base_log, score_log = [], [], []
+    static = frames_seq[:, 0].contiguous() if graph else None
     for t in range(T):
         if record:
             used.append(r.current_sets())
-        scores, base = r.step(frames_seq[:, t].contiguous())
+        if graph and t > 0:
+            if r.graphs is None:
+                r.capture(static)
+            static.copy_(frames_seq[:, t])
+            scores, base = r.step_graph()
+        else:
+            scores, base = r.step(frames_seq[:, t].contiguous())
         if record:
             base_log.append(base.cpu().numpy().copy())
             score_log.append(scores.cpu().numpy().copy())

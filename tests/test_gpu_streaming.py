@@ -53,3 +53,67 @@ def test_free_running_streams_teacher_forced(context_copy):
         assert np.abs(out["scores"][t, s] - so[0]).max() < 1e-2
         assert np.abs(base[t, s] - bo[0]).max() < 1e-2
     m.close()
+
+
+@pytest.mark.gpu
+def test_device_plan_and_graph_replay_match_host_plan():
+    """The same closed loop three ways: plan on the host (pm_forward), plan on the device
+    (pm_forward_device_sets), and the device-plan step replayed from CUDA graphs.  A row's result does
+    not depend on where bucketing puts it, so the sets agree, and the scores agree exactly wherever both
+    ways run the same kernels."""
+    import torch
+    from paper_2507_14959_b200 import binding, streaming
+    w = wl.deit_small_streams()
+    S, T = 8, 6
+    spec = w.spec
+    fr = wl.make_stream_frames("device_plan_streams", spec, S, T)           # [S, T, 3, img, img]
+    # a base-head bias that lets only a few labels per frame cross 0.5: small, non-empty sets
+    bb = wl.make_backbone("device_plan_streams", spec, head_bias_mean=-0.9)
+    w = wl.Workload("device_plan_streams", spec, bb, w.adapters, w.frames, w.set_offsets, w.set_ids)
+    m = binding.model_from_workload(w, dtype=0, max_frames=S, max_set=16)
+    m.set_cover(0.6)
+    fd = torch.from_numpy(fr).cuda().to(torch.bfloat16)
+    outs = [streaming.run(m, fd, spec.n_classes, len(w.adapters), 0.5, False, device_plan=dp, graph=gr)
+            for dp, gr in ((False, False), (True, False), (True, True))]
+    sizes = [len(x) for step in outs[0]["used_sets"][1:] for x in step]
+    assert np.mean(sizes) > 0.5                                     # adapters really are in play
+    for o in outs[1:]:
+        assert o["used_sets"] == outs[0]["used_sets"]
+    # replaying the recorded step launches exactly the kernels of the eager device-plan step
+    np.testing.assert_array_equal(outs[2]["base"], outs[1]["base"])
+    np.testing.assert_array_equal(outs[2]["scores"], outs[1]["scores"])
+    # host plan against device plan: on the first step (no adapters anywhere) the host plan skips the LoRA
+    # path and takes the LayerNorm statistics from a kernel of their own, the device plan from the shrink
+    assert np.abs(outs[1]["base"] - outs[0]["base"]).max() < 5e-3
+    assert np.abs(outs[1]["scores"] - outs[0]["scores"]).max() < 5e-3
+    np.testing.assert_array_equal(outs[1]["base"][2:], outs[0]["base"][2:])
+    assert m.status() == 0
+    m.close()
+
+
+@pytest.mark.gpu
+def test_device_plan_reports_bad_lists():
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    m = binding.model_from_workload(w, dtype=0, max_frames=2, max_set=2)
+    fd = torch.from_numpy(w.frames).cuda().to(torch.bfloat16)
+    K = w.spec.n_classes
+    sc, bs = torch.zeros((2, K), device="cuda"), torch.zeros((2, K), device="cuda")
+    ref_s, ref_b = torch.zeros((2, K), device="cuda"), torch.zeros((2, K), device="cuda")
+    off = torch.tensor([0, 1, 3], dtype=torch.int32, device="cuda")
+    m.forward_device_sets(fd, off, torch.tensor([0, 1, 3], dtype=torch.int32, device="cuda"), ref_s, ref_b)
+    assert m.status() == 0
+    so, bo = po.forward(w.backbone, w.adapters, w.frames, w.set_offsets, w.set_ids, w.spec.heads, w.spec.patch,
+                        w.spec.ln_eps, K)
+    assert np.abs(ref_s.cpu().numpy() - so).max() < 1e-2 and np.abs(ref_b.cpu().numpy() - bo).max() < 1e-2
+    # id 9 is out of range, id 3 repeated: both are skipped and the status word says so
+    m.forward_device_sets(fd, torch.tensor([0, 2, 5], dtype=torch.int32, device="cuda"),
+                          torch.tensor([0, 9, 3, 1, 3], dtype=torch.int32, device="cuda"), sc, bs)
+    assert m.status() == binding.PM_ERR_ARG
+    np.testing.assert_array_equal(sc.cpu().numpy(), ref_s.cpu().numpy())
+    # three ids where max_set is 2: the two lowest are kept
+    m.forward_device_sets(fd, torch.tensor([0, 1, 4], dtype=torch.int32, device="cuda"),
+                          torch.tensor([0, 3, 2, 1], dtype=torch.int32, device="cuda"), sc, bs)
+    assert m.status() == binding.PM_ERR_CAPACITY
+    m.close()
