@@ -195,17 +195,33 @@ def run_streams(args, rank, world, dist):
     import torch
     import workloads as wl
     from paper_2507_14959_b200 import binding, shard, streaming
-    S, T = 16, 30
-    w = wl.vit_base_384_streams(n_streams=S, n_steps=T)
+    T = 30
+    if args.workload == "latency":
+        S = 1
+        w = wl.deit_tiny_stream(n_steps=T, n_streams=S)
+        what = ("deit_tiny_stream: DeiT-tiny 224x224, ONE stream in closed loop (a step = one frame), 11 rank-16 "
+                "query/value adapters on the last 2 blocks, 5 classes each")
+    else:
+        S = 16
+        w = wl.vit_base_384_streams(n_streams=S, n_steps=T)
+        what = ("vit_base_384_streams: ViT-base 384x384 (577 tokens), 16 streams/GPU in closed loop, 64 rank-16 "
+                "adapters over 800 classes")
+    mode = args.loop
     m = binding.model_from_workload(w, dtype=0, max_frames=S, max_set=8)
     m.set_cover(w.tau)
     K = w.spec.n_classes
     frames_host = torch.from_numpy(w.extra["stream_frames"]).to(torch.bfloat16).transpose(0, 1).contiguous().pin_memory()
-    frames_dev = frames_host.cuda()                              # [T, S, 3, 384, 384]
-    r = streaming.StreamRunner(m, S, K, len(w.adapters), 0.5, False)
+    frames_dev = frames_host.cuda()                              # [T, S, 3, img, img]
+    r = streaming.StreamRunner(m, S, K, len(w.adapters), 0.5, False, device_plan=mode != "host")
     stage = torch.empty_like(frames_dev[0])
     scores_host = torch.zeros((S, K)).pin_memory()
     stream = torch.cuda.current_stream()
+    if mode == "graph":
+        # one eager step sets every kernel up; then the step is recorded once per list-buffer parity
+        r.reset()
+        stage.copy_(frames_dev[0])
+        r.step(stage)
+        r.capture(stage)
 
     def barrier():
         torch.cuda.synchronize()
@@ -218,12 +234,16 @@ def run_streams(args, rank, world, dist):
             t = i % T
             if t == 0:
                 r.reset()
-            if e2e:
+            if mode == "graph":
+                stage.copy_(frames_host[t] if e2e else frames_dev[t], non_blocking=True)
+                sc, _ = r.step(stage) if t == 0 else r.step_graph()
+            elif e2e:
                 stage.copy_(frames_host[t], non_blocking=True)
                 sc, _ = r.step(stage)
-                scores_host.copy_(sc, non_blocking=True)
             else:
-                r.step(frames_dev[t])
+                sc, _ = r.step(frames_dev[t])
+            if e2e:
+                scores_host.copy_(sc, non_blocking=True)
 
     loop(max(args.warmup, 3), False)
     assert m.status() == 0
@@ -233,7 +253,8 @@ def run_streams(args, rank, world, dist):
         if e2e:
             loop(2, True)
         barrier()
-        n0 = m.launch_count()
+        count = lambda: m.launch_count() + (r.replayed_launches if mode == "graph" else 0)
+        n0 = count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         loop(args.steps, e2e)
@@ -241,7 +262,7 @@ def run_streams(args, rank, world, dist):
         barrier()
         out_ms.append(e0.elapsed_time(e1))
         if not e2e:
-            launches = m.launch_count() - n0
+            launches = count() - n0
     assert m.status() == 0
     ms, ms_e2e = shard.max_over_ranks(out_ms, device="cuda")
     if rank == 0:
@@ -249,9 +270,13 @@ def run_streams(args, rank, world, dist):
             "metric": METRIC, "value": world * S * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "vit_base_384_streams: ViT-base 384x384 (577 tokens), 16 streams/GPU in closed "
-                                   "loop, 64 rank-16 adapters over 800 classes, sets chosen by Algorithm 2 on the device",
-                       "l2": "one step touches ~0.2 GB of activations; no flush"},
+            "config": {"workload": what + ", sets chosen by Algorithm 2 on the device",
+                       "loop": {"host": "routing plan on the host (a device-to-host copy and a stream synchronisation per step)",
+                                "device": "routing plan built on the device, no host synchronisation",
+                                "graph": "routing plan built on the device; steps after a stream's first are CUDA-graph replays"}[mode],
+                       "l2": "one step's activations fit the 126 MB L2; no flush" if args.workload == "latency"
+                             else "one step touches ~0.2 GB of activations; no flush"},
+            "latency_us_per_step": 1e3 * ms / args.steps,
             "e2e": {"value": world * S * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(stage.numel() * 2), "d2h_bytes_per_step": int(scores_host.numel() * 4)},
             "gpu_launches": int(launches)}))
@@ -275,9 +300,13 @@ def main():
                     help="batch workload with --lora-last N only: the paper's arrangement (Fig. 2b) -- the first "
                          "layers-N blocks run once per frame, then the base model and every active adapter "
                          "continue as separate branches (pm_forward_branched)")
-    ap.add_argument("--workload", default="batch", choices=["batch", "streams"],
+    ap.add_argument("--workload", default="batch", choices=["batch", "streams", "latency"],
                     help="batch: ViT-base 224x224, 256 frames (the headline); streams: ViT-base 384x384, 16 streams "
-                         "in closed loop (forward -> Algorithm 2 -> next forward), one step = one frame per stream")
+                         "in closed loop (forward -> Algorithm 2 -> next forward), one step = one frame per stream; "
+                         "latency: DeiT-tiny, one stream in closed loop (the paper's embedded operating point)")
+    ap.add_argument("--loop", default="graph", choices=["host", "device", "graph"],
+                    help="streams / latency: where the routing plan of a step is built and whether steps are "
+                         "CUDA-graph replays")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "polymorph" else args.warmup
 
@@ -300,7 +329,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    if args.workload == "streams":
+    if args.workload in ("streams", "latency"):
         run_streams(args, rank, world, dist)
         return
 

@@ -289,6 +289,28 @@ def vit_base_384_streams(n_streams=16, n_steps=30, layers=12) -> Workload:
                     extra={"stream_frames": fr, "score_thr": 0.5})
 
 
+def deit_tiny_stream(n_steps=30, n_streams=1) -> Workload:
+    """The paper's embedded operating point as a latency workload (Sec. 4, Table 2): DeiT-tiny, one
+    video stream, 11 contexts of 5 classes each over an 80-class label space (25 classes belong to
+    no context), rank-16 adapters on the query and value projections of the last 2 of 12 blocks,
+    scale 32/16.  The base-head bias is shifted so that about two labels per frame cross 0.5."""
+    name = "deit_tiny_stream"
+    spec = tiny_spec(80)
+    logit_std = float(np.sqrt(spec.d)) * 0.02
+    bb = make_backbone(name, spec, head_bias_mean=-1.96 * logit_std)
+    ads = []
+    for a in range(11):
+        ad = make_adapter(name, spec, a, 16, np.arange(5 * a, 5 * a + 5), layers=range(spec.layers - 2, spec.layers),
+                          projs=("qkv",))
+        for l in range(spec.layers - 2, spec.layers):
+            ad.B[l * 4][:, spec.d:2 * spec.d] = 0.0          # query and value only: the key columns stay untouched
+        ads.append(ad)
+    fr = make_stream_frames(name, spec, n_streams, n_steps)
+    off, ids = sets_to_csr([[] for _ in range(n_streams)])
+    return Workload(name, spec, bb, ads, fr[:, 0].copy(), off, ids, tau=0.6,
+                    extra={"stream_frames": fr, "score_thr": 0.5})
+
+
 # --------------------------------------------------------------------------------------
 # isolated fused base+LoRA linear cells
 # --------------------------------------------------------------------------------------
