@@ -117,3 +117,35 @@ def test_device_plan_reports_bad_lists():
                           torch.tensor([0, 3, 2, 1], dtype=torch.int32, device="cuda"), sc, bs)
     assert m.status() == binding.PM_ERR_CAPACITY
     m.close()
+
+
+@pytest.mark.gpu
+def test_single_stream_latency_shape_teacher_forced():
+    """DeiT-tiny, one stream, query/value adapters on the last two blocks (Sec. 4, Table 2 shape), closed
+    loop as CUDA-graph replays: the oracle, given the sets the GPU used, reproduces every step."""
+    import torch
+    from paper_2507_14959_b200 import binding, streaming
+    T = 5
+    w = wl.deit_tiny_stream(n_steps=T, n_streams=1)
+    m = binding.model_from_workload(w, dtype=0, max_frames=1, max_set=8)
+    m.set_cover(w.tau)
+    fr = w.extra["stream_frames"]
+    fd = torch.from_numpy(fr).cuda().to(torch.bfloat16)
+    out = streaming.run(m, fd, w.spec.n_classes, len(w.adapters), 0.5, False, device_plan=True, graph=True)
+    used, base = out["used_sets"], out["base"]
+    contexts = [a.class_ids for a in w.adapters]
+    accs = [a.acc for a in w.adapters]
+    Y_prev, S_prev = None, None
+    for t in range(T):
+        off, ids = wl.sets_to_csr([used[t][0]])
+        so, bo = po.forward(w.backbone, w.adapters, fr[0:1, t], off, ids, w.spec.heads, w.spec.patch,
+                            w.spec.ln_eps, w.spec.n_classes)
+        assert np.abs(out["scores"][t, 0] - so[0]).max() < 1e-2
+        assert np.abs(base[t, 0] - bo[0]).max() < 1e-2
+        if t + 1 < T:
+            Y = po.labels_from_scores(base[t, 0], 0.5)
+            want = po.detect_contexts(Y, Y_prev, contexts, accs, w.tau, S_prev, False)
+            assert want == used[t + 1][0], t
+            Y_prev, S_prev = Y, want
+    assert sum(len(s[0]) for s in used[1:]) > 0
+    m.close()
