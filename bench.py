@@ -324,6 +324,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
+    # everything runs on a stream of its own: the legacy default stream cannot be recorded into CUDA graphs,
+    # which the library does with its launch sequence once it has seen the same call twice
+    torch.cuda.set_stream(torch.cuda.Stream())
     dist = None
     if world > 1:
         import torch.distributed as dist

@@ -223,7 +223,15 @@ int pm_status(pm_handle h, void* cuda_stream);
 
 const char* pm_last_error(pm_handle h);
 
-/* Number of kernels the library has launched on this handle since creation. */
+/* The forward entry points record their launch sequence as a CUDA graph the second time they are
+ * called with the same buffers, sizes, stream and routing plan, and replay it from then on (the
+ * adapter sets may change between replays only for pm_forward_device_sets, whose plan is built
+ * inside the recorded sequence).  Not on the legacy default stream, not while the caller's stream is
+ * itself being captured, not while pm_profile_enable is on.  pm_set_graphs(h, 0) switches this off
+ * and frees the recorded graphs; default on. */
+int pm_set_graphs(pm_handle h, int on);
+
+/* Number of kernels the library has launched on this handle since creation (kernels of a replayed graph included). */
 long long pm_launch_count(pm_handle h);
 
 /* Device timing of the library's own kernels, by class, with CUDA events recorded on the launching

@@ -21,7 +21,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
 
 EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
-    "pm_select_static", "pm_status", "pm_last_error", "pm_launch_count", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
+    "pm_select_static", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention",
 ]
@@ -83,6 +83,7 @@ def load():
     lib.pm_last_error.argtypes = [vp]
     lib.pm_last_error.restype = C.c_char_p
     lib.pm_launch_count.argtypes = [vp]
+    lib.pm_set_graphs.argtypes = [vp, ip]
     lib.pm_launch_count.restype = C.c_longlong
     lib.pm_profile_enable.argtypes = [vp, ip]
     lib.pm_profile_read.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
@@ -203,6 +204,10 @@ class Model:
 
     def status(self, stream=None):
         return self.lib.pm_status(self.handle, _stream_ptr(stream))
+
+    def set_graphs(self, on):
+        """Switches the recording / replaying of the forward's launch sequence as CUDA graphs."""
+        self._check(self.lib.pm_set_graphs(self.handle, int(on)), "pm_set_graphs")
 
     KERNEL_CLASSES = ("gemm", "shrink", "attention", "layernorm", "other")
 

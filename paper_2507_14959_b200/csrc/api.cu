@@ -194,6 +194,10 @@ struct Router {
     RouteDev dev;
     std::vector<int32_t> last_off, last_ids;
     std::vector<int> last_fixed;     // frame_of_slot then src_of_slot of the cached plan (branched forward)
+    // changes whenever the launch sequence that follows from the plan may change (a new host plan; a
+    // device plan for another frame count): recorded CUDA graphs are keyed by it
+    unsigned long long version = 0;
+    int device_plan_frames = -1;
     int last_frames = -1;
     bool last_sorted = false;
     std::vector<int> perm_host;
@@ -323,6 +327,7 @@ struct Router {
         CK(cudaMemcpyAsync(blob.p, stage, blob_bytes, cudaMemcpyHostToDevice, st));
         CK(cudaEventRecord(uploaded, st));
         upload_pending = true;
+        ++version; device_plan_frames = -1;
         dev.n_frames = n_frames; dev.n_tiles = n_tiles; dev.max_set = widest;
         last_off.assign(offsets, offsets + n_frames + 1);
         last_ids.assign(ids, ids + nnz);
@@ -342,6 +347,7 @@ struct Router {
                         const AdapterMeta& meta, std::string& err) {
         if (n_frames > max_frames || n_frames > PM_DEVICE_PLAN_MAX_FRAMES) { err = "n_frames exceeds the device planner's limit"; return PM_ERR_CAPACITY; }
         invalidate();
+        if (device_plan_frames != n_frames) { ++version; device_plan_frames = n_frames; }
         dev.n_frames = n_frames;
         dev.n_tiles = (int)(((long long)n_frames * tokens + 2 * PM_TILE_M - 1) / (2 * PM_TILE_M)) * 2;
         dev.max_set = max_set;
@@ -420,9 +426,91 @@ struct pm_handle_s {
     long long launches = 0;
     Profiler prof;
     std::string err;
+    // recorded launch sequences of the forward entry points (see run_graphed)
+    struct GraphEntry {
+        const void* key_ptr[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+        int key_int[4] = {0, 0, 0, 0};
+        unsigned long long plan_version = 0;
+        cudaStream_t st = nullptr;
+        cudaGraphExec_t exec = nullptr;     // null: seen once, not recorded yet
+        long long launches = 0;
+        unsigned long long last_use = 0;
+        bool same_key(const GraphEntry& o) const {
+            return std::equal(key_ptr, key_ptr + 5, o.key_ptr) && std::equal(key_int, key_int + 4, o.key_int) &&
+                   plan_version == o.plan_version && st == o.st;
+        }
+    };
+    std::vector<GraphEntry> graphs;
+    bool graphs_on = true;
+    unsigned long long graph_clock = 0;
+    void drop_graphs() {
+        for (GraphEntry& g : graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+        graphs.clear();
+    }
+    ~pm_handle_s() { drop_graphs(); }
 };
 
 namespace {
+
+// Runs `enqueue` (which puts one forward's kernels on `key.st`), recording it as a CUDA graph the
+// second time the same call is seen -- same buffers, sizes, stream and routing plan -- and replaying
+// the graph from then on: back-to-back kernels of a replay start about 2 us closer to each other than
+// individually launched ones.  Falls back to plain launches on the legacy default stream (it cannot
+// be captured), while the caller is itself capturing, and while per-launch profiling is on.
+template <typename F>
+int run_graphed(pm_handle_s* h, pm_handle_s::GraphEntry key, F&& enqueue) {
+    constexpr size_t MAX_GRAPHS = 8;
+    std::string& err = h->err;
+    cudaStream_t st = key.st;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (!h->graphs_on || h->prof.on || st == nullptr || st == cudaStreamLegacy ||
+        cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+        cudaGetLastError();
+        return enqueue();
+    }
+    pm_handle_s::GraphEntry* e = nullptr;
+    for (auto& g : h->graphs) if (g.same_key(key)) e = &g;
+    if (!e) {                                    // first sighting: remember it, launch plainly
+        if (h->graphs.size() >= MAX_GRAPHS) {
+            size_t old = 0;
+            for (size_t i = 1; i < h->graphs.size(); ++i) if (h->graphs[i].last_use < h->graphs[old].last_use) old = i;
+            if (h->graphs[old].exec) cudaGraphExecDestroy(h->graphs[old].exec);
+            h->graphs.erase(h->graphs.begin() + old);
+        }
+        key.last_use = ++h->graph_clock;
+        h->graphs.push_back(key);
+        return enqueue();
+    }
+    e->last_use = ++h->graph_clock;
+    if (!e->exec) {                              // second sighting: record
+        const long long l0 = h->launches;
+        if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+            cudaGetLastError();
+            h->graphs_on = false;
+            return enqueue();
+        }
+        const int rc = enqueue();
+        cudaGraph_t g = nullptr;
+        const cudaError_t ce = cudaStreamEndCapture(st, &g);
+        const long long recorded = h->launches - l0;
+        h->launches = l0;                        // nothing has run yet
+        cudaGraphExec_t exec = nullptr;
+        if (rc == PM_OK && ce == cudaSuccess && g && cudaGraphInstantiate(&exec, g, 0) == cudaSuccess) {
+            e->exec = exec;
+            e->launches = recorded;
+        }
+        if (g) cudaGraphDestroy(g);
+        if (!e->exec) {                          // could not record: never try again on this handle
+            cudaGetLastError();
+            h->graphs_on = false;
+            if (rc != PM_OK) return rc;
+            return enqueue();
+        }
+    }
+    CK(cudaGraphLaunch(e->exec, st));
+    h->launches += e->launches;
+    return PM_OK;
+}
 
 int slabs_for(int max_rank) { return (max_rank + PM_SLAB - 1) / PM_SLAB; }
 
@@ -708,6 +796,7 @@ int pm_register_adapter(pm_handle h, int id, const pm_adapter* a) {
     else h->acc[id].assign(a->n_cls, 1.f);
     h->heads_dirty = true; h->cover_ready = false;
     h->router.invalidate();
+    h->drop_graphs();                 // recorded launch sequences refer to the old adapters and heads
     return sync_meta(h->scale_dev, h->rank_dev, h->scales, h->ranks, err);
 }
 
@@ -766,8 +855,14 @@ int pm_forward(pm_handle h, const void* frames, int n_frames, const int32_t* set
         rc = h->cfg.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
         if (rc) return rc;
     }
-    return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
-                             : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
+    pm_handle_s::GraphEntry key;
+    key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
+    key.key_int[0] = n_frames; key.key_int[1] = 0 /* entry point */;
+    key.plan_version = h->router.version; key.st = st;
+    return run_graphed(h, key, [&]() {
+        return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
+                                 : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
+    });
 }
 
 int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames, const int32_t* set_offsets,
@@ -782,11 +877,20 @@ int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames, const 
         int rc = h->cfg.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
         if (rc) return rc;
     }
-    Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
-    int rc = h->router.build_on_device(L, n_frames, set_offsets, set_ids, h->meta, err);
-    if (rc) return rc;
-    return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
-                             : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
+    if (n_frames > PM_DEVICE_PLAN_MAX_FRAMES) { err = "n_frames exceeds the device planner's limit"; return PM_ERR_CAPACITY; }
+    pm_handle_s::GraphEntry key;
+    key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
+    key.key_ptr[3] = set_offsets; key.key_ptr[4] = set_ids;
+    key.key_int[0] = n_frames; key.key_int[1] = 1 /* entry point */;
+    // the launch sequence of a device plan depends on the frame count only, not on the lists
+    key.plan_version = 0; key.st = st;
+    return run_graphed(h, key, [&]() {
+        Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
+        int rc = h->router.build_on_device(L, n_frames, set_offsets, set_ids, h->meta, err);
+        if (rc) return rc;
+        return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
+                                 : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
+    });
 }
 
 int pm_forward_branched(pm_handle h, const void* frames, int n_frames, const int32_t* set_offsets,
@@ -849,8 +953,15 @@ int pm_forward_branched(pm_handle h, const void* frames, int n_frames, const int
         rc = c.dtype == 0 ? rebuild_heads<bf16>(h) : rebuild_heads<float>(h);
         if (rc) return rc;
     }
-    return c.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st)
-                        : forward_t<float>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st);
+    pm_handle_s::GraphEntry key;
+    key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
+    key.key_int[0] = n_frames; key.key_int[1] = 2 /* entry point */; key.key_int[2] = trunk_layers;
+    key.key_int[3] = (int)n_slots;
+    key.plan_version = h->router.version; key.st = st;
+    return run_graphed(h, key, [&]() {
+        return c.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st)
+                            : forward_t<float>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st);
+    });
 }
 
 int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, int context_copy,
@@ -911,6 +1022,13 @@ int pm_profile_read(pm_handle h, void* cuda_stream, double* ms_by_class, long lo
     return PM_OK;
 }
 long long pm_launch_count(pm_handle h) { return h ? h->launches : 0; }
+
+int pm_set_graphs(pm_handle h, int on) {
+    if (!h) return PM_ERR_ARG;
+    h->graphs_on = on != 0;
+    if (!h->graphs_on) h->drop_graphs();
+    return PM_OK;
+}
 
 // ---- single operators -------------------------------------------------------------------
 int pm_linear_create(int k_in, int n_out, const float* w, const float* bias, int max_adapters,

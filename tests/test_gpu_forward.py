@@ -111,6 +111,62 @@ def test_paper_variant_query_value_last_blocks(dtype):
     m.close()
 
 
+def test_recorded_launch_sequence_replays_identically():
+    """On a stream of its own the forward records its launch sequence the second time it sees the same
+    call and replays it afterwards: same results, same launch count per call; a change of the sets makes
+    a new plan and is honoured; the device-plan entry point replays with lists that change in place."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    m = binding.model_from_workload(w, dtype=0)
+    K = w.spec.n_classes
+    fd = frames_to_dev(w.frames, 0)
+    ref_s, ref_b = run_forward(m, w, 0)                     # legacy default stream: never recorded
+    off2, ids2 = wl.sets_to_csr([[2], [0, 1]])
+    ref2_s, ref2_b = run_forward(m, w, 0, offsets=off2, ids=ids2)
+    side = torch.cuda.Stream()
+    sc = torch.zeros((2, K), device="cuda"); bs = torch.zeros((2, K), device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        counts = []
+        for i in range(4):                                    # plain, record + replay, replay, replay
+            sc.fill_(-1.0); bs.fill_(-1.0)
+            n0 = m.launch_count()
+            m.forward(fd, w.set_offsets, w.set_ids, sc, bs)
+            counts.append(m.launch_count() - n0)
+            side.synchronize()
+            np.testing.assert_array_equal(sc.cpu().numpy(), ref_s.astype(np.float32))
+            np.testing.assert_array_equal(bs.cpu().numpy(), ref_b.astype(np.float32))
+        assert len(set(counts)) == 1 and counts[0] > 0
+        for i in range(3):                                    # other sets: a new plan, a new recording
+            m.forward(fd, off2, ids2, sc, bs)
+            side.synchronize()
+            np.testing.assert_array_equal(sc.cpu().numpy(), ref2_s.astype(np.float32))
+        m.forward(fd, w.set_offsets, w.set_ids, sc, bs)      # and back
+        side.synchronize()
+        np.testing.assert_array_equal(sc.cpu().numpy(), ref_s.astype(np.float32))
+        # device-plan entry point: one recording serves whatever the lists hold at replay time
+        d_off = torch.tensor([0, 1, 3], dtype=torch.int32, device="cuda")
+        d_ids = torch.tensor([0, 1, 3], dtype=torch.int32, device="cuda")
+        for i in range(3):
+            m.forward_device_sets(fd, d_off, d_ids, sc, bs)
+        side.synchronize()
+        first = sc.cpu().numpy().copy()
+        assert np.abs(first - ref_s).max() < 2e-3             # (LayerNorm statistics come from another kernel here)
+        d_off.copy_(torch.tensor([0, 1, 3], dtype=torch.int32)); d_ids.copy_(torch.tensor([2, 0, 1], dtype=torch.int32))
+        m.forward_device_sets(fd, d_off, d_ids, sc, bs)
+        side.synchronize()
+        assert np.abs(sc.cpu().numpy() - ref2_s).max() < 2e-3
+        assert np.abs(sc.cpu().numpy() - first).max() > 1e-2
+        assert m.status(side) == 0
+        # switched off: plain launches again, same numbers
+        m.set_graphs(False)
+        m.forward(fd, w.set_offsets, w.set_ids, sc, bs)
+        side.synchronize()
+        np.testing.assert_array_equal(sc.cpu().numpy(), ref_s.astype(np.float32))
+    m.close()
+
+
 def test_forward_argument_errors():
     import torch
     from paper_2507_14959_b200 import binding
