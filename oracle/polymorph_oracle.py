@@ -17,6 +17,8 @@ What follows the paper and where:
   * heads / compose    Sec. 4 (one head per adapter over its class subset), Fig. 5b (active outputs
                        merged), Sec. 3.2 (base prediction over the full label space).
   * detect_contexts    Algorithm 2, step by step.
+  * build_contexts     Algorithm 1 (context construction from label co-occurrence), step by step.
+  * intra_coherence    Eq. 6.
   * avg_coverage, switch_penalty   Eq. 7 and Eq. 8.
   * model_stats        the parameter / memory / MAC accounting behind Table 2.
 
@@ -245,6 +247,87 @@ def minimum_cover_size(Y, contexts, acc, tau):
             if set().union(*(provs[c] for c in comb)) >= target:
                 return n
     raise AssertionError("unreachable")
+
+
+# --------------------------------------------------------------------------------------
+# Algorithm 1: context construction from a label co-occurrence matrix, and Eq. 6
+# --------------------------------------------------------------------------------------
+def cooccurrence(label_sets, n_labels):
+    """co[i, j] = number of frames whose label set holds both i and j (diagonal: frames holding i).
+    Sec. 3.4: the matrix is built from the training set's per-frame label sets."""
+    co = np.zeros((n_labels, n_labels), dtype=np.float64)
+    for Y in label_sets:
+        for i in Y:
+            for j in Y:
+                co[i, j] += 1.0
+    return co
+
+
+def build_contexts(co, B, M_max, allow_overlap):
+    """Algorithm 1 (BuildContexts), step by step.  Returns the contexts as sorted label lists, in the
+    order they were created.
+
+    Readings where the listing is silent:
+      * valid labels = labels that occur at all (co[l, l] > 0);
+      * they are visited from the most to the least frequent (Sec. 3.4: clusters are centred on
+        frequently occurring labels), ties by ascending label;
+      * the cluster around l = l plus its up to B-1 strongest co-occurring valid neighbours with
+        co[l, j] > 0 (ties by ascending label); without overlap, labels already assigned are no
+        candidates;
+      * unique = not equal, as a set, to a context already kept;
+      * an uncovered label (visited in ascending order) goes to the context with room left whose
+        members co-occur with it most in total, ties by the earlier context; if no context has
+        room it stays uncovered (the size limit wins).
+    """
+    co = np.asarray(co, dtype=np.float64)
+    K = co.shape[0]
+    valid = [l for l in range(K) if co[l, l] > 0]
+    order = sorted(valid, key=lambda l: (-co[l, l], l))
+    contexts, assigned = [], set()
+    for l in order:
+        if not allow_overlap and l in assigned:
+            continue
+        cand = [j for j in valid if j != l and co[l, j] > 0 and (allow_overlap or j not in assigned)]
+        cand.sort(key=lambda j: (-co[l, j], j))
+        cluster = sorted([l] + cand[:max(B - 1, 0)])
+        if cluster not in contexts and len(contexts) < M_max:
+            contexts.append(cluster)
+            if not allow_overlap:
+                assigned |= set(cluster)
+    covered = set().union(*contexts) if contexts else set()
+    for l in valid:
+        if l in covered:
+            continue
+        best, best_fit = -1, -1.0
+        for c, ctx in enumerate(contexts):
+            if len(ctx) >= B:
+                continue
+            fit = sum(co[l, j] for j in ctx)
+            if fit > best_fit:
+                best, best_fit = c, fit
+        if best >= 0:
+            contexts[best] = sorted(contexts[best] + [l])
+            covered.add(l)
+    return contexts
+
+
+def intra_coherence(contexts, co_norm):
+    """Eq. 6: mean over contexts of the mean normalised co-occurrence over ordered pairs i != j of the
+    context.  Reading: a context with a single label has no pair and contributes 0."""
+    if not contexts:
+        return 0.0
+    total = 0.0
+    for ctx in contexts:
+        n = len(ctx)
+        if n < 2:
+            continue
+        s = 0.0
+        for i in ctx:
+            for j in ctx:
+                if i != j:
+                    s += co_norm[i][j]
+        total += s / (n * (n - 1))
+    return total / len(contexts)
 
 
 def avg_coverage(S_seq):
