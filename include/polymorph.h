@@ -243,6 +243,37 @@ long long pm_launch_count(pm_handle h);
 int pm_profile_enable(pm_handle h, int on);
 int pm_profile_read(pm_handle h, void* cuda_stream, double* ms_by_class, long long* launches_by_class);
 
+/* ---- training-time context construction (Sec. 3.4) -------------------------------------- */
+
+/* Label co-occurrence counts from per-frame label bit sets (the layout pm_select keeps in
+ * prev_labels): co[i, j] = number of frames whose set holds both i and j; co[i, i] = frames holding i.
+ *   labels      dev uint32 [n_frames, ceil(n_labels/32)], bit k%32 of word k/32 = label k
+ *   co          dev fp32 [n_labels, n_labels], overwritten (counts are exact: n_frames <= 2^24)
+ *   status_out  dev int32 or NULL: PM_ERR_CAPACITY if a frame carries more than 64 labels (its first
+ *               64 are counted)
+ * Asynchronous on the stream.  Errors: PM_ERR_ARG, PM_ERR_CAPACITY (n_frames), PM_ERR_CUDA. */
+int pm_cooccurrence(const uint32_t* labels, int n_frames, int n_labels, float* co,
+                    int32_t* status_out, void* cuda_stream);
+
+/* Algorithm 1 (BuildContexts).  Host function, host pointers.
+ *   co             host fp32 [n_labels, n_labels] co-occurrence (symmetric; diagonal = label frequency)
+ *   max_size       B: no context holds more labels; max_contexts: M_max; allow_overlap: the flag
+ *   ctx_offsets    host int32 [max_contexts + 1], ctx_ids host int32 [max_contexts * max_size]: the
+ *                  contexts as CSR of ascending label ids, in creation order; *n_contexts their number
+ * Valid labels (co[l, l] > 0) are visited from the most to the least frequent (ties: lower label);
+ * a cluster is the label plus its up to B-1 strongest co-occurring valid neighbours (co > 0; ties:
+ * lower label; without overlap only unassigned ones); a cluster equal to a kept context is dropped;
+ * labels left uncovered go, in ascending order, to the context with room whose members co-occur
+ * with them most (ties: earlier context), or stay uncovered if none has room. */
+int pm_build_contexts(const float* co, int n_labels, int max_size, int max_contexts, int allow_overlap,
+                      int32_t* ctx_offsets, int32_t* ctx_ids, int* n_contexts);
+
+/* IntraCoherence (Eq. 6) of a context set under a normalised co-occurrence matrix (host pointers):
+ * mean over contexts of the mean co_norm[i, j] over ordered pairs i != j; single-label contexts
+ * contribute 0. */
+int pm_intra_coherence(const float* co_norm, int n_labels, const int32_t* ctx_offsets,
+                       const int32_t* ctx_ids, int n_contexts, double* out);
+
 /* ---- single operators (the same kernels pm_forward uses), for unit tests and sweeps ----- */
 
 /* One base + multi-LoRA linear y = epilogue(x W + b + sum_a s_a (x A_a) B_a)   (Sec. 3.1).

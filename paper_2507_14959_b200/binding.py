@@ -23,7 +23,7 @@ EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
     "pm_select_static", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
-    "pm_layernorm", "pm_attention",
+    "pm_layernorm", "pm_attention", "pm_cooccurrence", "pm_build_contexts", "pm_intra_coherence",
 ]
 
 
@@ -83,6 +83,9 @@ def load():
     lib.pm_last_error.argtypes = [vp]
     lib.pm_last_error.restype = C.c_char_p
     lib.pm_launch_count.argtypes = [vp]
+    lib.pm_cooccurrence.argtypes = [vp, ip, ip, vp, vp, vp]
+    lib.pm_build_contexts.argtypes = [_FP, ip, ip, ip, ip, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int)]
+    lib.pm_intra_coherence.argtypes = [_FP, ip, C.POINTER(C.c_int32), C.POINTER(C.c_int32), ip, C.POINTER(C.c_double)]
     lib.pm_set_graphs.argtypes = [vp, ip]
     lib.pm_launch_count.restype = C.c_longlong
     lib.pm_profile_enable.argtypes = [vp, ip]
@@ -325,3 +328,44 @@ def model_from_workload(w, *, dtype=0, max_frames=None, max_set=None):
         m.register_adapter(i, rank=a.rank, scale=a.scale, A=a.A, B=a.B, class_ids=a.class_ids,
                            head_w=a.head_w, head_b=a.head_b, acc=a.acc)
     return m
+
+
+def cooccurrence(labels, n_labels, co, status=None, stream=None):
+    """pm_cooccurrence: labels = torch CUDA int32 [T, ceil(K/32)] bit sets, co = torch CUDA fp32 [K, K]."""
+    rc = load().pm_cooccurrence(_ptr(labels), int(labels.shape[0]), int(n_labels), _ptr(co), _ptr(status),
+                                _stream_ptr(stream))
+    if rc != PM_OK:
+        raise PolymorphError(rc, "pm_cooccurrence")
+
+
+def build_contexts(co, max_size, max_contexts, allow_overlap):
+    """pm_build_contexts (Algorithm 1) on a host matrix; returns the contexts as lists of label ids."""
+    co = np.ascontiguousarray(co, dtype=np.float32)
+    K = co.shape[0]
+    off = np.zeros(max_contexts + 1, dtype=np.int32)
+    ids = np.zeros(max_contexts * max_size, dtype=np.int32)
+    n = C.c_int(0)
+    i32 = C.POINTER(C.c_int32)
+    rc = load().pm_build_contexts(co.ctypes.data_as(_FP), K, int(max_size), int(max_contexts), int(bool(allow_overlap)),
+                                  off.ctypes.data_as(i32), ids.ctypes.data_as(i32), C.byref(n))
+    if rc != PM_OK:
+        raise PolymorphError(rc, "pm_build_contexts")
+    return [ids[off[c]:off[c + 1]].tolist() for c in range(n.value)]
+
+
+def intra_coherence(contexts, co_norm):
+    """pm_intra_coherence (Eq. 6)."""
+    co_norm = np.ascontiguousarray(co_norm, dtype=np.float32)
+    off, ids = [0], []
+    for c in contexts:
+        ids.extend(int(i) for i in c)
+        off.append(len(ids))
+    off = np.asarray(off, dtype=np.int32)
+    ids = np.asarray(ids if ids else [0], dtype=np.int32)
+    out = C.c_double(0.0)
+    i32 = C.POINTER(C.c_int32)
+    rc = load().pm_intra_coherence(co_norm.ctypes.data_as(_FP), co_norm.shape[0], off.ctypes.data_as(i32),
+                                   ids.ctypes.data_as(i32), len(contexts), C.byref(out))
+    if rc != PM_OK:
+        raise PolymorphError(rc, "pm_intra_coherence")
+    return out.value
