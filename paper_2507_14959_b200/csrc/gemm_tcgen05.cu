@@ -28,24 +28,21 @@ constexpr int STAGES = 4;
 constexpr int SHRINK_THREADS = 192;
 constexpr int SLABS_PER_STAGE = 4;
 
-// Exact-erf GELU x * Phi(x) through the rational approximation of Abramowitz & Stegun 7.1.28,
-//   erfc(z) = (1 + a1 z + ... + a6 z^6)^-16 + eps, |eps| <= 3e-7   (z >= 0),
-// with 2^(1/16) folded into the coefficients so that the reciprocal is erfc(z)/2 = Phi(-|x|):
-//   gelu(x) = max(x, 0) - |x| * Phi(-|x|).
-// 12 FP32 operations and one reciprocal per element; absolute error below 1e-6 for finite x.
+// Exact-erf GELU x * Phi(x), evaluated in logistic form: Phi(x) = 1 / (1 + exp(-2 x p(x^2))) holds
+// exactly for p = atanh(erf(x / sqrt 2)) / x, which a quadratic in x^2 fits well enough that
+//   | x / (1 + 2^(x q(x^2))) - gelu(x) | < 2.6e-5   for all x     (q = -2 log2(e) p),
+// far below the bf16 rounding of the stored result except where the result itself is below 1e-2.
+// Seven FP32 operations, one exponential and one reciprocal per element.  The epilogue warps share
+// their issue slots with the thread that issues the MMAs, so every instruction saved here counts.
 __device__ __forceinline__ float gelu_erf(float v) {
-    const float z = fabsf(v) * 0.70710678118654752440f;
-    float p = 4.4970397e-05f;
-    p = fmaf(p, z, 2.8881188e-04f);
-    p = fmaf(p, z, 1.5874455e-04f);
-    p = fmaf(p, z, 9.6809685e-03f);
-    p = fmaf(p, z, 4.4153997e-02f);
-    p = fmaf(p, z, 7.3645402e-02f);
-    p = fmaf(p, z, 1.0442738f);
-    p *= p; p *= p; p *= p; p *= p;
-    float h;                                      // p = +inf (|x| > ~25) gives 0
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(h) : "f"(p));
-    return fmaf(-fabsf(v), h, fmaxf(v, 0.f));
+    // v^2 is capped where Phi has long saturated (the fitted q turns over beyond |v| = 7.2)
+    const float t = fminf(v * v, 50.f);
+    float q = fmaf(t, 1.0142706e-03f, -1.06775776e-01f);
+    q = fmaf(q, t, -2.3011212f);
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(v * q));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.f));      // e = +inf gives 0
+    return v * r;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
