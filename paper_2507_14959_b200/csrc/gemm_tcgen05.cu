@@ -32,17 +32,51 @@ constexpr int SLABS_PER_STAGE = 4;
 // exactly for p = atanh(erf(x / sqrt 2)) / x, which a quadratic in x^2 fits well enough that
 //   | x / (1 + 2^(x q(x^2))) - gelu(x) | < 2.6e-5   for all x     (q = -2 log2(e) p),
 // far below the bf16 rounding of the stored result except where the result itself is below 1e-2.
-// Seven FP32 operations, one exponential and one reciprocal per element.  The epilogue warps share
-// their issue slots with the thread that issues the MMAs, so every instruction saved here counts.
-__device__ __forceinline__ float gelu_erf(float v) {
+// The epilogue warps share their issue slots with the thread that issues the MMAs, so every
+// instruction saved here counts: the arithmetic runs on pairs (packed fp32), six instructions per
+// element including one exponential and one reciprocal.
+
+// Two fp32 values in one 64-bit register, for the packed fp32 arithmetic of sm_100 (one issue slot
+// for two results; each half is the ordinary IEEE operation).
+__device__ __forceinline__ uint64_t pk2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void upk2(uint64_t r, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// the GELU described above, on a pair
+__device__ __forceinline__ uint64_t gelu_erf2(uint64_t v) {
     // v^2 is capped where Phi has long saturated (the fitted q turns over beyond |v| = 7.2)
-    const float t = fminf(v * v, 50.f);
-    float q = fmaf(t, 1.0142706e-03f, -1.06775776e-01f);
-    q = fmaf(q, t, -2.3011212f);
-    float e, r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(v * q));
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.f));      // e = +inf gives 0
-    return v * r;
+    float t0, t1;
+    upk2(mul2(v, v), t0, t1);
+    const uint64_t t = pk2(fminf(t0, 50.f), fminf(t1, 50.f));
+    uint64_t q = fma2(t, pk2(1.0142706e-03f, 1.0142706e-03f), pk2(-1.06775776e-01f, -1.06775776e-01f));
+    q = fma2(q, t, pk2(-2.3011212f, -2.3011212f));
+    float w0, w1, e0, e1, r0, r1;
+    upk2(mul2(v, q), w0, w1);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(w0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(w1));
+    upk2(add2(pk2(e0, e1), pk2(1.f, 1.f)), e0, e1);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(e0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(e1));
+    return mul2(v, pk2(r0, r1));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -159,27 +193,27 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
             __syncwarp();
             if (lane == 0) { if (PAIR) mbar_arrive_cluster(tempty_addr); else mbar_arrive(tempty_addr); }
         }
-        float f[32];
+        // bias (and the folded LayerNorm: rstd (acc - mean g) + b) and GELU, two columns per instruction
+        uint64_t fp[16];                                 // columns (2i, 2i+1) of this chunk
+        const uint64_t rstd2 = pk2(st.y, st.y), nmean2 = pk2(-st.x, -st.x);
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
             const float4 b4 = __ldg(reinterpret_cast<const float4*>(args.bias + n0 + j));
+            uint64_t a0 = pk2(__uint_as_float(v[j + 0]), __uint_as_float(v[j + 1]));
+            uint64_t a1 = pk2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
             if constexpr (LNF) {
                 const float4 g4 = __ldg(reinterpret_cast<const float4*>(args.ln_g + n0 + j));
-                f[j + 0] = fmaf(st.y, fmaf(-st.x, g4.x, __uint_as_float(v[j + 0])), b4.x);
-                f[j + 1] = fmaf(st.y, fmaf(-st.x, g4.y, __uint_as_float(v[j + 1])), b4.y);
-                f[j + 2] = fmaf(st.y, fmaf(-st.x, g4.z, __uint_as_float(v[j + 2])), b4.z);
-                f[j + 3] = fmaf(st.y, fmaf(-st.x, g4.w, __uint_as_float(v[j + 3])), b4.w);
+                a0 = fma2(rstd2, fma2(nmean2, pk2(g4.x, g4.y), a0), pk2(b4.x, b4.y));
+                a1 = fma2(rstd2, fma2(nmean2, pk2(g4.z, g4.w), a1), pk2(b4.z, b4.w));
             } else {
-                f[j + 0] = __uint_as_float(v[j + 0]) + b4.x;
-                f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
-                f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
-                f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+                a0 = add2(a0, pk2(b4.x, b4.y));
+                a1 = add2(a1, pk2(b4.z, b4.w));
             }
+            if constexpr (EPI == EPI_GELU) { a0 = gelu_erf2(a0); a1 = gelu_erf2(a1); }
+            fp[j >> 1] = a0;
+            fp[(j >> 1) + 1] = a1;
         }
-        if constexpr (EPI == EPI_GELU) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) f[j] = gelu_erf(f[j]);
-        } else if constexpr (EPI == EPI_RESIDUAL) {
+        if constexpr (EPI == EPI_RESIDUAL) {
             if constexpr (RES_SMEM) {
                 if (cc == 0) {
                     ok = mbar_wait(res_bar, res_phase, abort_flag, args.status);
@@ -200,27 +234,27 @@ __device__ __forceinline__ bool epilogue_tile(const GemmArgs& args, const CUtens
                 }
                 const uint32_t w[4] = {r4v.x, r4v.y, r4v.z, r4v.w};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    f[q * 8 + 2 * e] += __uint_as_float(w[e] << 16);
-                    f[q * 8 + 2 * e + 1] += __uint_as_float(w[e] & 0xFFFF0000u);
-                }
+                for (int e = 0; e < 4; ++e)
+                    fp[q * 4 + e] = add2(fp[q * 4 + e], pk2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xFFFF0000u)));
             }
         } else if constexpr (EPI == EPI_PATCH) {
             if (row_ok) {
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
                     const float4 p4 = __ldg(reinterpret_cast<const float4*>(pos_row + n0 + j));
-                    f[j + 0] += p4.x; f[j + 1] += p4.y; f[j + 2] += p4.z; f[j + 3] += p4.w;
+                    fp[j >> 1] = add2(fp[j >> 1], pk2(p4.x, p4.y));
+                    fp[(j >> 1) + 1] = add2(fp[(j >> 1) + 1], pk2(p4.z, p4.w));
                 }
             }
         }
         uint4 o[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            o[q].x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
-            o[q].y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
-            o[q].z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
-            o[q].w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
+            float lo, hi;
+            upk2(fp[q * 4 + 0], lo, hi); o[q].x = pack_bf16(lo, hi);
+            upk2(fp[q * 4 + 1], lo, hi); o[q].y = pack_bf16(lo, hi);
+            upk2(fp[q * 4 + 2], lo, hi); o[q].z = pack_bf16(lo, hi);
+            upk2(fp[q * 4 + 3], lo, hi); o[q].w = pack_bf16(lo, hi);
         }
         if (args.tma_store) {
             // [32 rows x 64 B] block, 16-byte chunks XOR-swizzled by (row >> 1) & 3 (64B
