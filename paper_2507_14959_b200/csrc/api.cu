@@ -878,6 +878,9 @@ int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames, const 
         if (rc) return rc;
     }
     if (n_frames > PM_DEVICE_PLAN_MAX_FRAMES) { err = "n_frames exceeds the device planner's limit"; return PM_ERR_CAPACITY; }
+    // the plan tables on the device are about to be rewritten (by the kernels below or by their replay):
+    // whatever host plan was uploaded before is gone
+    h->router.invalidate();
     pm_handle_s::GraphEntry key;
     key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
     key.key_ptr[3] = set_offsets; key.key_ptr[4] = set_ids;

@@ -159,6 +159,12 @@ def test_recorded_launch_sequence_replays_identically():
         assert np.abs(sc.cpu().numpy() - ref2_s).max() < 2e-3
         assert np.abs(sc.cpu().numpy() - first).max() > 1e-2
         assert m.status(side) == 0
+        # a replayed device plan overwrites the plan tables: the host planner must not trust its cache after it
+        m.forward(fd, w.set_offsets, w.set_ids, sc, bs)      # host plan for the first sets, uploaded
+        m.forward_device_sets(fd, d_off, d_ids, sc, bs)      # replay: the tables now hold the second sets
+        m.forward(fd, w.set_offsets, w.set_ids, sc, bs)      # same host sets as two calls ago
+        side.synchronize()
+        np.testing.assert_array_equal(sc.cpu().numpy(), ref_s.astype(np.float32))
         # switched off: plain launches again, same numbers
         m.set_graphs(False)
         m.forward(fd, w.set_offsets, w.set_ids, sc, bs)
