@@ -640,7 +640,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, int n_slots, int
         }
         if constexpr (TC) {
             if (attention_tc_supported(T_))
-                CK(launch_attention_tc(L, h->tm_att_q, h->tm_att_kv, (bf16*)ATT, n_cur, T_, c.heads));
+                CK(launch_attention_tc(L, h->tm_att_q, h->tm_att_kv, (bf16*)ATT, n_cur, T_, c.heads, h->n_sms));
             else
                 CK(launch_attention_mma(L, (const bf16*)QKV, (bf16*)ATT, n_cur, T_, c.heads));
         }
@@ -1171,7 +1171,10 @@ int pm_attention(const void* qkv, void* out, int n_frames, int tokens, int heads
         L.status = status_word;
         CUtensorMap tm_q, tm_kv;
         if (!attention_encode_maps((const bf16*)qkv, n_frames, tokens, heads, &tm_q, &tm_kv)) return PM_ERR_CUDA;
-        e = launch_attention_tc(L, tm_q, tm_kv, (bf16*)out, n_frames, tokens, heads);
+        int dev = 0, n_sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PM_ERR_CUDA;
+        e = launch_attention_tc(L, tm_q, tm_kv, (bf16*)out, n_frames, tokens, heads, n_sms);
     } else {
         e = launch_attention_mma(L, (const bf16*)qkv, (bf16*)out, n_frames, tokens, heads);
     }

@@ -10,6 +10,8 @@
 // 64 with an online softmax in fp32; both contractions run on the tensor cores
 // (mma.sync m16n8k16, bf16 in, fp32 accumulate).  Key blocks are trimmed to the 8-key tile, so
 // 197 tokens cost 200 key columns, not 256.
+#include <algorithm>
+
 #include "common.cuh"
 #include "tcgen05_ptx.cuh"
 
@@ -457,6 +459,270 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 }
 
+// Sweep over the score columns [0, ncols) that start at tensor-memory address t_s (ncols a multiple
+// of 16, `valid` of them real), 16 at a time with the next load in flight.  PROBS = false: running
+// row maximum.  PROBS = true: P (packed bf16, 8 columns per 16 scores) goes to t_p onwards and the
+// row sum of this range is added to acc.
+template <bool PROBS>
+__device__ __forceinline__ float score_range_sweep(uint32_t t_s, uint32_t t_p, int ncols, int valid, float c, float mc,
+                                                   float acc) {
+    uint32_t va[16], vb[16];
+    auto piece = [&](const uint32_t* v, int c0) {
+        const int lim = valid - c0;
+        if (PROBS) {
+            uint32_t pk[8];
+            acc += lim >= 16 ? chunk_probs<16, false>(v, 16, c, mc, pk) : chunk_probs<16, true>(v, lim, c, mc, pk);
+            tmem_st8(t_p + (uint32_t)(c0 >> 1), pk);
+        } else {
+            acc = lim >= 16 ? chunk_max<16, false>(v, 16, acc) : chunk_max<16, true>(v, lim, acc);
+        }
+    };
+    tmem_ld16(t_s, va);
+    tmem_ld_wait();
+#pragma unroll 1
+    for (int c0 = 0; c0 < ncols; c0 += 32) {
+        if (c0 + 16 < ncols) tmem_ld16(t_s + (uint32_t)(c0 + 16), vb);
+        piece(va, c0);
+        tmem_ld_wait();
+        if (c0 + 16 < ncols) {
+            if (c0 + 32 < ncols) tmem_ld16(t_s + (uint32_t)(c0 + 32), va);
+            piece(vb, c0 + 16);
+            tmem_ld_wait();
+        }
+    }
+    return acc;
+}
+
+// ---------------------------------------------------------------------------------------
+// Pipelined variant for sequences of one key block (up to 208 tokens, at most two query tiles):
+// one persistent CTA per SM walks (frame, head) items and keeps two query tiles in flight, each in
+// its own half of tensor memory with its own group of eight softmax warps:
+//     warp 0         TMA: K, V and the query tiles of item j+2 land while items j, j+1 are computed
+//     warp 1         MMA issue:  S(c), then P V of tile c-1, then S(c+1), ...
+//     warps 2..9     softmax + output of the even tiles (tensor-memory columns 0..255)
+//     warps 10..17   the same for the odd tiles (columns 256..511)
+// so the tensor pipe, the two softmax groups and the loads of the following items overlap inside one
+// CTA.  Two warps share each quarter of the 128 rows (a warp reaches the tensor-memory lanes
+// 32 (w mod 4) .. +31 only) and split the key columns: the first seven 16-key pieces and the rest.
+// The sweeps are chains of dependent operations, so what bounds them is how many warps a scheduler
+// can switch between: four per scheduler here against two with one warp per quarter.  The halves
+// exchange their row maxima and row sums through shared memory (mbarriers, bounded waits).
+// Column map of a tile's 256-column slot: scores 0..207; P of the first half over 0..55, P of the
+// second half in 208..255 (so that it never lands on scores the first half still reads); O in
+// 128..191 once both halves are done.  Tile c of a CTA is query tile c % nq of its item c / nq.
+// ---------------------------------------------------------------------------------------
+constexpr int APIPE_GROUP_WARPS = 8;
+constexpr int APIPE_THREADS = 64 + 2 * 32 * APIPE_GROUP_WARPS;      // 576
+constexpr int APIPE_ITEM_BYTES = 2 * AKB_BYTES + 2 * AQ_BYTES;      // K, V, two query tiles
+constexpr int APIPE_SPLIT = 7;                                       // 16-key pieces of the first half
+constexpr int APIPE_XCHG_BYTES = 2 * 2 * 2 * AQ * 4;                 // [max | sum][group][half][row]
+
+struct AttnPipeArgs {
+    int tokens, heads, tpad, nq, n_items;
+    bf16* out;
+    int* status;
+};
+
+__global__ void __launch_bounds__(APIPE_THREADS, 1)
+attention_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
+                      const AttnPipeArgs args) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if (base & 1023u) {                       // swizzled operands need a 1024-byte aligned window
+        if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
+        return;
+    }
+    const int T = args.tokens, nq = args.nq, d = args.heads * HD;
+    const int my_items = (args.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_tiles = my_items * nq;
+    const int n_pieces = args.tpad / 16, split = min(APIPE_SPLIT, n_pieces);
+    auto k_s = [&](int buf) { return base + buf * APIPE_ITEM_BYTES; };
+    auto v_s = [&](int buf) { return base + buf * APIPE_ITEM_BYTES + AKB_BYTES; };
+    auto q_s = [&](int buf, int qt) { return base + buf * APIPE_ITEM_BYTES + 2 * AKB_BYTES + qt * AQ_BYTES; };
+    float* xchg = reinterpret_cast<float*>(smem_raw + 2 * APIPE_ITEM_BYTES);
+    const uint32_t bars = base + 2 * APIPE_ITEM_BYTES + APIPE_XCHG_BYTES;
+    auto kv_full = [&](int b) { return bars + 8u * b; };
+    auto buf_free = [&](int b) { return bars + 16u + 8u * b; };
+    auto s_ready = [&](int sl) { return bars + 32u + 8u * sl; };
+    auto p_ready = [&](int sl) { return bars + 48u + 8u * sl; };
+    auto o_ready = [&](int sl) { return bars + 64u + 8u * sl; };
+    auto slot_free = [&](int sl) { return bars + 80u + 8u * sl; };
+    auto max_bar = [&](int sl) { return bars + 96u + 8u * sl; };
+    auto sum_bar = [&](int sl) { return bars + 112u + 8u * sl; };
+    uint8_t* bar_ptr = smem_raw + (bars - base);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 128);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 136);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(kv_full(i), 1); mbar_init(buf_free(i), 1);
+            mbar_init(s_ready(i), 1); mbar_init(p_ready(i), APIPE_GROUP_WARPS);
+            mbar_init(o_ready(i), 1); mbar_init(slot_free(i), APIPE_GROUP_WARPS);
+            mbar_init(max_bar(i), APIPE_GROUP_WARPS); mbar_init(sum_bar(i), APIPE_GROUP_WARPS);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- TMA producer
+            bool ok = true;
+            for (int j = 0; j < my_items && ok; ++j) {
+                const int buf = j & 1;
+                // the buffer's previous item (j - 2) must be through its last P V product
+                ok = mbar_wait(buf_free(buf), (((uint32_t)j >> 1) & 1u) ^ 1u, abort_flag, args.status);
+                if (!ok) break;
+                const int item = (int)blockIdx.x + j * (int)gridDim.x;
+                const int f = item / args.heads, h = item % args.heads;
+                mbar_expect_tx(kv_full(buf), (uint32_t)(2 * AKB_BYTES + nq * AQ_BYTES));
+                tma_load_2d(k_s(buf), &tm_kv, d + h * HD, f * T, kv_full(buf));
+                for (int qt = 0; qt < nq; ++qt) tma_load_2d(q_s(buf, qt), &tm_q, h * HD, f * T + qt * AQ, kv_full(buf));
+                tma_load_2d(v_s(buf), &tm_kv, 2 * d + h * HD, f * T, kv_full(buf));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- MMA issue
+            const uint32_t idesc_s = instr_desc(args.tpad), idesc_pv = instr_desc_b_mn(HD);
+            bool ok = true;
+            // O(p) = P(p) V: P is the packed bf16 the two halves left in tile p's slot
+            auto issue_pv = [&](int p) {
+                const int slot = p & 1, buf = (p / nq) & 1;
+                ok = mbar_wait(p_ready(slot), ((uint32_t)p >> 1) & 1u, abort_flag, args.status);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t s_tmem = tmem_base + (uint32_t)(slot * 256);
+                const uint64_t dv0 = smem_desc(v_s(buf), 128);
+                for (int kk = 0; kk < n_pieces; ++kk) {
+                    const uint32_t p_col = kk < split ? (uint32_t)(kk * 8) : (uint32_t)(208 + (kk - split) * 8);
+                    umma_bf16_ts(s_tmem + 128u, s_tmem + p_col, dv0 + 128 * kk, idesc_pv, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(o_ready(slot));
+                if (p % nq == nq - 1) umma_commit(buf_free(buf));     // the item's operands are no longer read
+            };
+            for (int c = 0; c < my_tiles && ok; ++c) {
+                const int j = c / nq, qt = c % nq, buf = j & 1, slot = c & 1;
+                if (qt == 0) ok = mbar_wait(kv_full(buf), ((uint32_t)j >> 1) & 1u, abort_flag, args.status);
+                // the slot's previous tile (c - 2) must have been read out
+                ok = ok && mbar_wait(slot_free(slot), (((uint32_t)c >> 1) & 1u) ^ 1u, abort_flag, args.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t dq0 = smem_desc(q_s(buf, qt), 128), dk0 = smem_desc(k_s(buf), 128);
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k)
+                    umma_bf16(tmem_base + (uint32_t)(slot * 256), dq0 + 2 * k, dk0 + 2 * k, idesc_s, k > 0);
+                umma_commit(s_ready(slot));
+                if (c >= 1) issue_pv(c - 1);
+            }
+            if (ok && my_tiles > 0) issue_pv(my_tiles - 1);
+        }
+    } else {
+        // -------------------------------------------------------------------- softmax + output
+        const int group = (warp - 2) / APIPE_GROUP_WARPS;        // 0: even tiles, 1: odd tiles
+        const int half = ((warp - 2) % APIPE_GROUP_WARPS) >> 2;  // which share of the key columns
+        const int quarter = warp & 3;                            // TMEM lanes 32*quarter .. +31
+        const int row = quarter * 32 + lane;                     // row of the query tile
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(group * 256);
+        const int col0 = half == 0 ? 0 : split * 16;             // first key column of this warp
+        const int ncols = half == 0 ? split * 16 : (n_pieces - split) * 16;
+        const uint32_t t_p = t_lane + (half == 0 ? 0u : 208u);   // where this warp's P goes
+        float* my_max = xchg + ((0 * 2 + group) * 2 + half) * AQ;
+        float* other_max = xchg + ((0 * 2 + group) * 2 + (half ^ 1)) * AQ;
+        float* my_sum = xchg + ((1 * 2 + group) * 2 + half) * AQ;
+        float* other_sum = xchg + ((1 * 2 + group) * 2 + (half ^ 1)) * AQ;
+        const float c_ = 0.125f * 1.4426950408889634f;           // 1/sqrt(64) * log2(e)
+        bool ok = true;
+        for (int c = group; c < my_tiles && ok; c += 2) {
+            const uint32_t par = ((uint32_t)c >> 1) & 1u;
+            const int j = c / nq, qt = c % nq;
+            const int item = (int)blockIdx.x + j * (int)gridDim.x;
+            const int f = item / args.heads, h = item % args.heads;
+            const int q_row = qt * AQ + row;
+            const bool warp_active = qt * AQ + quarter * 32 < T;     // else: no row of this warp exists
+            ok = mbar_wait(s_ready(group), par, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            // row maximum: own columns, then the other half's through shared memory
+            float m = -INFINITY;
+            if (warp_active && ncols > 0)
+                m = score_range_sweep<false>(t_lane + (uint32_t)col0, 0u, ncols, T - col0, 0.f, 0.f, m);
+            my_max[row] = m;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(max_bar(group));
+            ok = mbar_wait(max_bar(group), par, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            m = fmaxf(m, other_max[row]);
+            float l = 0.f;
+            if (warp_active && ncols > 0) {
+                l = score_range_sweep<true>(t_lane + (uint32_t)col0, t_p, ncols, T - col0, c_, m * c_, 0.f);
+                tmem_st_wait();
+            }
+            my_sum[row] = l;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(sum_bar(group)); mbar_arrive(p_ready(group)); }
+            ok = mbar_wait(sum_bar(group), par, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            l += other_sum[row];
+            ok = mbar_wait(o_ready(group), par, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            if (warp_active) {
+                // each half writes 32 of the 64 output columns
+                const float inv = 1.f / l;
+                bf16* orow = args.out + ((size_t)f * T + q_row) * d + h * HD + half * 32;
+                uint32_t v[32];
+                tmem_ld32((t_lane + 128u) + (uint32_t)(half * 32), v);
+                tmem_ld_wait();
+                if (q_row < T) {
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        uint32_t o[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            o[e] = pack2(__uint_as_float(v[q * 16 + 2 * e]) * inv,
+                                         __uint_as_float(v[q * 16 + 2 * e + 1]) * inv);
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                     ::"l"(orow + q * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]),
+                                       "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                                     : "memory");
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(slot_free(group));
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);    // let copies / MMAs in flight land
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
 }  // namespace
 
 bool attention_tc_supported(int tokens) { return (tokens + 15) / 16 * 16 <= ATT_MAX_BLOCKS * AKB; }
@@ -469,7 +735,7 @@ bool attention_encode_maps(const bf16* qkv, int n_frames, int tokens, int heads,
 }
 
 cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const CUtensorMap& tm_kv,
-                                bf16* out, int n_frames, int tokens, int heads) {
+                                bf16* out, int n_frames, int tokens, int heads, int n_sms) {
     if (n_frames <= 0) return cudaSuccess;
     AttnArgs a;
     a.tokens = tokens; a.heads = heads;
@@ -484,6 +750,23 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
     a.tmem_cols = a.n_blocks == 1 ? 256u : 512u;
     a.o_col = a.n_blocks == 1 ? 128u : 256u;
     a.out = out; a.status = L.status;
+    if (a.n_blocks == 1 && a.n_qtiles <= 2 && n_sms > 0) {
+        // one key block: the pipelined persistent kernel
+        AttnPipeArgs pa;
+        pa.tokens = tokens; pa.heads = heads; pa.tpad = a.tpad; pa.nq = a.n_qtiles;
+        pa.n_items = n_frames * heads; pa.out = out; pa.status = L.status;
+        const size_t psmem = 2 * (size_t)APIPE_ITEM_BYTES + APIPE_XCHG_BYTES + 192;
+        static bool pipe_set = false;
+        if (!pipe_set) {
+            cudaError_t e = cudaFuncSetAttribute(attention_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psmem);
+            if (e != cudaSuccess) return e;
+            pipe_set = true;
+        }
+        ProfScope ps(L, KC_ATTENTION);
+        attention_pipe_kernel<<<std::min(pa.n_items, n_sms), APIPE_THREADS, psmem, L.st>>>(tm_q, tm_kv, pa);
+        BUMP(L);
+        return cudaGetLastError();
+    }
     // one block: 68 KB, three CTAs per SM (two computing, the third loading while it waits for TMEM)
     size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
     static size_t smem_set = 0;

@@ -128,8 +128,9 @@ cudaError_t launch_attention_mma(const Launch& L, const bf16* qkv, bf16* out, in
 bool attention_tc_supported(int tokens);
 bool attention_encode_maps(const bf16* qkv, int n_frames, int tokens, int heads, CUtensorMap* tm_q,
                            CUtensorMap* tm_kv);
+// n_sms > 0 selects the pipelined persistent kernel where it applies (one key block); 0 = never
 cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const CUtensorMap& tm_kv,
-                                bf16* out, int n_frames, int tokens, int heads);
+                                bf16* out, int n_frames, int tokens, int heads, int n_sms);
 template <typename T>
 cudaError_t launch_im2col(const Launch& L, const T* frames, const int* perm, T* out, int n_frames,
                           int img, int patch);
