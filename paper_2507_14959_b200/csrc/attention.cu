@@ -194,7 +194,11 @@ __global__ void __launch_bounds__(512) attention_mma_kernel(const bf16* __restri
 // ---------------------------------------------------------------------------------------
 constexpr int AQ = 128;                    // query rows per tile
 constexpr int AKB = 208;                   // keys per score block
-constexpr int ATT_THREADS = 160;           // warp 0: TMEM owner, TMA + MMA issue; warps 1..4: softmax
+constexpr int ATT_MAX_SHARES = 3;          // softmax warps per lane quarter (they split the key columns)
+#ifndef PM_ATT_SHARES
+#define PM_ATT_SHARES 2
+#endif
+constexpr int ATT_SHARES = PM_ATT_SHARES;  // the multi-block kernel's choice: block = 32 + 128 * ATT_SHARES threads
 constexpr int AQ_BYTES = AQ * 128;
 constexpr int AKB_BYTES = AKB * 128;
 constexpr int ATT_MAX_BLOCKS = 3;
@@ -238,42 +242,49 @@ __device__ __forceinline__ float chunk_probs(const uint32_t* v, int lim, float c
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
-// One sweep over a score block of nb columns (a multiple of 16), 16 columns at a time, with the
-// tensor-memory load of the next chunk in flight while the current one is processed.
-// PROBS = false: running row maximum (acc in, acc out).  PROBS = true: writes P (packed bf16) over
-// the scores and returns acc + the row sum of this block.  Columns at or beyond `valid` are ignored.
+// Sweep over the score columns [0, ncols) that start at tensor-memory address t_s (ncols a multiple
+// of 16, `valid` of them real), 16 at a time with the next load in flight.  PROBS = false: running
+// row maximum.  PROBS = true: P (packed bf16, 8 columns per 16 scores) goes to t_p onwards and the
+// row sum of this range is added to acc.
 template <bool PROBS>
-__device__ __forceinline__ float score_chunk(uint32_t t_lane, const uint32_t* v, int c0, int valid, float c,
-                                             float mc, float acc) {
-    const int lim = valid - c0;
-    if (PROBS) {
-        uint32_t pk[8];
-        acc += lim >= 16 ? chunk_probs<16, false>(v, 16, c, mc, pk) : chunk_probs<16, true>(v, lim, c, mc, pk);
-        tmem_st8(t_lane + (uint32_t)(c0 >> 1), pk);
-        return acc;
-    }
-    return lim >= 16 ? chunk_max<16, false>(v, 16, acc) : chunk_max<16, true>(v, lim, acc);
-}
-template <bool PROBS>
-__device__ __forceinline__ float score_block_sweep(uint32_t t_lane, int nb, int valid, float c, float mc, float acc) {
+__device__ __forceinline__ float score_range_sweep(uint32_t t_s, uint32_t t_p, int ncols, int valid, float c, float mc,
+                                                   float acc) {
     uint32_t va[16], vb[16];
-    tmem_ld16(t_lane, va);
+    auto piece = [&](const uint32_t* v, int c0) {
+        const int lim = valid - c0;
+        if (PROBS) {
+            uint32_t pk[8];
+            acc += lim >= 16 ? chunk_probs<16, false>(v, 16, c, mc, pk) : chunk_probs<16, true>(v, lim, c, mc, pk);
+            tmem_st8(t_p + (uint32_t)(c0 >> 1), pk);
+        } else {
+            acc = lim >= 16 ? chunk_max<16, false>(v, 16, acc) : chunk_max<16, true>(v, lim, acc);
+        }
+    };
+    tmem_ld16(t_s, va);
     tmem_ld_wait();
 #pragma unroll 1
-    for (int c0 = 0; c0 < nb; c0 += 32) {
-        if (c0 + 16 < nb) tmem_ld16(t_lane + (uint32_t)(c0 + 16), vb);
-        acc = score_chunk<PROBS>(t_lane, va, c0, valid, c, mc, acc);
+    for (int c0 = 0; c0 < ncols; c0 += 32) {
+        if (c0 + 16 < ncols) tmem_ld16(t_s + (uint32_t)(c0 + 16), vb);
+        piece(va, c0);
         tmem_ld_wait();
-        if (c0 + 16 < nb) {
-            if (c0 + 32 < nb) tmem_ld16(t_lane + (uint32_t)(c0 + 32), va);
-            acc = score_chunk<PROBS>(t_lane, vb, c0 + 16, valid, c, mc, acc);
+        if (c0 + 16 < ncols) {
+            if (c0 + 32 < ncols) tmem_ld16(t_s + (uint32_t)(c0 + 32), va);
+            piece(vb, c0 + 16);
             tmem_ld_wait();
         }
     }
     return acc;
 }
 
-__global__ void __launch_bounds__(ATT_THREADS, 3)
+// Share k of `shares` takes the 16-key pieces [att_first(shares, k), att_first(shares, k + 1)) of a key
+// block (capped to the block's pieces) and leaves its P at the start of its own score columns.
+__host__ __device__ constexpr int att_first(int shares, int k) {
+    return shares == 1 ? (k == 0 ? 0 : 13) : shares == 2 ? (k == 0 ? 0 : k == 1 ? 7 : 13)
+                                                         : (k == 0 ? 0 : k == 1 ? 5 : k == 2 ? 9 : 13);
+}
+
+template <int SHARES>
+__global__ void __launch_bounds__(32 + 128 * SHARES, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kv,
                     const AttnArgs args) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -294,13 +305,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t v_s = k_s + n_blocks * AKB_BYTES;
     const uint32_t bars = v_s + n_blocks * AKB_BYTES;
     const uint32_t kv_bar = bars, s_bar = bars + 8, r_bar = bars + 16, q_bar = bars + 24;
+    const uint32_t max_bar = bars + 48, sum_bar = bars + 56;
     uint8_t* bar_ptr = smem_raw + (bars - base);
+    float* xchg = reinterpret_cast<float*>(bar_ptr + 64);        // [max | sum][share][row]
+    constexpr int shares = SHARES;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 40);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(kv_bar, 1); mbar_init(q_bar, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4);
+        mbar_init(kv_bar, 1); mbar_init(q_bar, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4 * shares);
+        mbar_init(max_bar, 4 * shares); mbar_init(sum_bar, 4 * shares);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -360,9 +375,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                 mbar_expect_tx(q_bar, AQ_BYTES);
                                 tma_load_2d(q_s, &tm_q, h * HD, f * T + (qt + 1) * AQ, q_bar);
                             }
-                            for (int kk = 0; kk < nb / 16; ++kk)
-                                umma_bf16_ts(o_tmem, tmem_base + (uint32_t)(kk * 8), dv0 + bo + 128 * kk, idesc_pv,
+                            // P of piece kk sits where its share left it: at the start of that share's columns
+                            uint32_t p_col = 0;
+                            for (int kk = 0; kk < nb / 16; ++kk) {
+                                if (kk == att_first(shares, 1) || kk == att_first(shares, 2)) p_col = (uint32_t)(kk * 16);
+                                umma_bf16_ts(o_tmem, tmem_base + p_col, dv0 + bo + 128 * kk, idesc_pv,
                                              (b > 0 || kk > 0) ? 1u : 0u);
+                                p_col += 8;
+                            }
                             umma_commit(s_bar);
                             ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
                             ++step;
@@ -374,11 +394,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
         }
     } else {
-        // ---------------------------------------------------------- softmax + output (warps 1..4)
+        // ---------------------------------------------------------- softmax + output
         const int quarter = warp & 3;                            // TMEM lanes 32*quarter .. +31
+        const int share = (warp - 1) >> 2;                       // which share of the key columns
+        const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const float c = 0.125f * 1.4426950408889634f;            // 1/sqrt(64) * log2(e)
-        uint32_t step = 0;
+        float* maxes = xchg;                                     // [share][row]
+        float* sums = xchg + ATT_MAX_SHARES * AQ;
+        uint32_t step = 0, tile_no = 0;
         bool ok = true;
         auto begin_step = [&]() {
             ok = mbar_wait(s_bar, step & 1u, abort_flag, args.status);
@@ -392,51 +416,89 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (lane == 0) mbar_arrive(r_bar);
             ++step;
         };
-        for (int qt = qt0; qt < qt1 && ok; ++qt) {
-            const int q_row = qt * AQ + quarter * 32 + lane;
+        // this warp's columns of key block b: [col0, col0 + ncols), `valid` of them real
+        auto my_cols = [&](int b, int& col0, int& ncols, int& valid) {
+            const int np = min(AKB, args.tpad - b * AKB) / 16;
+            const int p0 = min(att_first(shares, share), np), p1 = min(att_first(shares, share + 1), np);
+            col0 = p0 * 16; ncols = (p1 - p0) * 16; valid = T - b * AKB - col0;
+        };
+        for (int qt = qt0; qt < qt1 && ok; ++qt, ++tile_no) {
+            const int q_row = qt * AQ + row;
             const bool warp_active = qt * AQ + quarter * 32 < T;      // else: no row of this warp exists
             float m = -INFINITY, l = 0.f;
+            int col0, ncols, valid;
             if (n_blocks > 1) {
                 for (int b = 0; b < n_blocks; ++b) {
                     if (!begin_step()) break;
-                    if (warp_active)
-                        m = score_block_sweep<false>(t_lane, min(AKB, args.tpad - b * AKB), T - b * AKB, 0.f, 0.f, m);
+                    my_cols(b, col0, ncols, valid);
+                    if (warp_active && ncols > 0)
+                        m = score_range_sweep<false>(t_lane + (uint32_t)col0, 0u, ncols, valid, 0.f, 0.f, m);
                     end_step();
                 }
                 if (!ok) break;
             }
             for (int b = 0; b < n_blocks; ++b) {
-                const int nb = min(AKB, args.tpad - b * AKB), valid = T - b * AKB;
                 if (!begin_step()) break;
-                if (warp_active) {
-                    if (n_blocks == 1) m = score_block_sweep<false>(t_lane, nb, valid, 0.f, 0.f, m);
-                    l = score_block_sweep<true>(t_lane, nb, valid, c, m * c, l);
+                my_cols(b, col0, ncols, valid);
+                if (b == 0) {
+                    if (n_blocks == 1 && warp_active && ncols > 0)
+                        m = score_range_sweep<false>(t_lane + (uint32_t)col0, 0u, ncols, valid, 0.f, 0.f, m);
+                    if (shares > 1) {
+                        // the row maximum over all keys: every share's part, through shared memory
+                        maxes[share * AQ + row] = m;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(max_bar);
+                        ok = mbar_wait(max_bar, tile_no & 1u, abort_flag, args.status);
+                        ok = __all_sync(0xFFFFFFFFu, ok);
+                        if (!ok) break;
+#pragma unroll
+                        for (int k = 0; k < shares; ++k) m = fmaxf(m, maxes[k * AQ + row]);
+                    }
+                }
+                if (warp_active && ncols > 0) {
+                    l = score_range_sweep<true>(t_lane + (uint32_t)col0, t_lane + (uint32_t)col0, ncols, valid, c, m * c, l);
                     tmem_st_wait();
+                }
+                if (shares > 1 && b == n_blocks - 1) {
+                    sums[share * AQ + row] = l;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sum_bar);
                 }
                 end_step();
                 // O (+)= P V_b is issued now; after the last block the finished rows are written out
                 if (!begin_step()) break;
-                if (b == n_blocks - 1 && warp_active) {
-                    const float inv = 1.f / l;
-                    bf16* orow = args.out + ((size_t)f * T + q_row) * d + h * HD;
+                if (b == n_blocks - 1) {
+                    if (shares > 1) {
+                        ok = mbar_wait(sum_bar, tile_no & 1u, abort_flag, args.status);
+                        ok = __all_sync(0xFFFFFFFFu, ok);
+                        if (!ok) break;
+                        l = 0.f;
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t v[32];
-                        tmem_ld32((t_lane + args.o_col) + (uint32_t)(half * 32), v);
-                        tmem_ld_wait();
-                        if (q_row < T) {
-                            // 32-byte stores: one full sector per row per instruction
+                        for (int k = 0; k < shares; ++k) l += sums[k * AQ + row];
+                    }
+                    // the output columns are split between the first two shares (all 64 to the only one)
+                    const int ocols = shares == 1 ? 64 : 32;
+                    if (warp_active && share * ocols < 64) {
+                        const float inv = 1.f / l;
+                        bf16* orow = args.out + ((size_t)f * T + q_row) * d + h * HD + share * ocols;
+                        for (int part = 0; part < ocols / 32; ++part) {
+                            uint32_t v[32];
+                            tmem_ld32((t_lane + args.o_col) + (uint32_t)(share * ocols + part * 32), v);
+                            tmem_ld_wait();
+                            if (q_row < T) {
+                                // 32-byte stores: one full sector per row per instruction
 #pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                uint32_t o[8];
+                                for (int q = 0; q < 2; ++q) {
+                                    uint32_t o[8];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e)
-                                    o[e] = pack2(__uint_as_float(v[q * 16 + 2 * e]) * inv,
-                                                 __uint_as_float(v[q * 16 + 2 * e + 1]) * inv);
-                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                                             ::"l"(orow + half * 32 + q * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]),
-                                               "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
-                                             : "memory");
+                                    for (int e = 0; e < 8; ++e)
+                                        o[e] = pack2(__uint_as_float(v[q * 16 + 2 * e]) * inv,
+                                                     __uint_as_float(v[q * 16 + 2 * e + 1]) * inv);
+                                    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                                 ::"l"(orow + part * 32 + q * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]),
+                                                   "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                                                 : "memory");
+                                }
                             }
                         }
                     }
@@ -457,40 +519,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc_fence_after();
         tmem_dealloc(tmem_base, args.tmem_cols);
     }
-}
-
-// Sweep over the score columns [0, ncols) that start at tensor-memory address t_s (ncols a multiple
-// of 16, `valid` of them real), 16 at a time with the next load in flight.  PROBS = false: running
-// row maximum.  PROBS = true: P (packed bf16, 8 columns per 16 scores) goes to t_p onwards and the
-// row sum of this range is added to acc.
-template <bool PROBS>
-__device__ __forceinline__ float score_range_sweep(uint32_t t_s, uint32_t t_p, int ncols, int valid, float c, float mc,
-                                                   float acc) {
-    uint32_t va[16], vb[16];
-    auto piece = [&](const uint32_t* v, int c0) {
-        const int lim = valid - c0;
-        if (PROBS) {
-            uint32_t pk[8];
-            acc += lim >= 16 ? chunk_probs<16, false>(v, 16, c, mc, pk) : chunk_probs<16, true>(v, lim, c, mc, pk);
-            tmem_st8(t_p + (uint32_t)(c0 >> 1), pk);
-        } else {
-            acc = lim >= 16 ? chunk_max<16, false>(v, 16, acc) : chunk_max<16, true>(v, lim, acc);
-        }
-    };
-    tmem_ld16(t_s, va);
-    tmem_ld_wait();
-#pragma unroll 1
-    for (int c0 = 0; c0 < ncols; c0 += 32) {
-        if (c0 + 16 < ncols) tmem_ld16(t_s + (uint32_t)(c0 + 16), vb);
-        piece(va, c0);
-        tmem_ld_wait();
-        if (c0 + 16 < ncols) {
-            if (c0 + 32 < ncols) tmem_ld16(t_s + (uint32_t)(c0 + 32), va);
-            piece(vb, c0 + 16);
-            tmem_ld_wait();
-        }
-    }
-    return acc;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -768,15 +796,15 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
         return cudaGetLastError();
     }
     // one block: 68 KB, three CTAs per SM (two computing, the third loading while it waits for TMEM)
-    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64;
+    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64 + 2 * ATT_MAX_SHARES * AQ * sizeof(float);
     static size_t smem_set = 0;
     if (smem > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<ATT_SHARES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     ProfScope ps(L, KC_ATTENTION);
-    attention_tc_kernel<<<n_frames * heads * a.q_split, ATT_THREADS, smem, L.st>>>(tm_q, tm_kv, a);
+    attention_tc_kernel<ATT_SHARES><<<n_frames * heads * a.q_split, 32 + 128 * ATT_SHARES, smem, L.st>>>(tm_q, tm_kv, a);
     BUMP(L);
     return cudaGetLastError();
 }

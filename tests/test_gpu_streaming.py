@@ -59,8 +59,7 @@ def test_free_running_streams_teacher_forced(context_copy):
 def test_device_plan_and_graph_replay_match_host_plan():
     """The same closed loop three ways: plan on the host (pm_forward), plan on the device
     (pm_forward_device_sets), and the device-plan step replayed from CUDA graphs.  A row's result does
-    not depend on where bucketing puts it, so the sets agree, and the scores agree exactly wherever both
-    ways run the same kernels."""
+    not depend on where bucketing puts it; eager and replayed device-plan loops agree bit for bit."""
     import torch
     from paper_2507_14959_b200 import binding, streaming
     w = wl.deit_small_streams()
@@ -77,16 +76,26 @@ def test_device_plan_and_graph_replay_match_host_plan():
             for dp, gr in ((False, False), (True, False), (True, True))]
     sizes = [len(x) for step in outs[0]["used_sets"][1:] for x in step]
     assert np.mean(sizes) > 0.5                                     # adapters really are in play
-    for o in outs[1:]:
-        assert o["used_sets"] == outs[0]["used_sets"]
     # replaying the recorded step launches exactly the kernels of the eager device-plan step
+    assert outs[2]["used_sets"] == outs[1]["used_sets"]
     np.testing.assert_array_equal(outs[2]["base"], outs[1]["base"])
     np.testing.assert_array_equal(outs[2]["scores"], outs[1]["scores"])
-    # host plan against device plan: on the first step (no adapters anywhere) the host plan skips the LoRA
-    # path and takes the LayerNorm statistics from a kernel of their own, the device plan from the shrink
-    assert np.abs(outs[1]["base"] - outs[0]["base"]).max() < 5e-3
-    assert np.abs(outs[1]["scores"] - outs[0]["scores"]).max() < 5e-3
-    np.testing.assert_array_equal(outs[1]["base"][2:], outs[0]["base"][2:])
+    # host plan against device plan: the first step (no adapters anywhere) runs the same frames through
+    # slightly different arithmetic (the host plan skips the LoRA path and takes the LayerNorm statistics
+    # from a kernel of their own, the device plan from the shrink), so scores agree to rounding only and
+    # a label next to the threshold may flip; from then on each loop follows its own sets.  Every loop
+    # must be consistent with Algorithm 2 applied to its own base scores.
+    assert np.abs(outs[1]["base"][0] - outs[0]["base"][0]).max() < 5e-3
+    contexts = [a.class_ids for a in w.adapters]
+    accs = [a.acc for a in w.adapters]
+    for o in outs:
+        for st in range(S):
+            Y_prev, S_prev = None, None
+            for t in range(T - 1):
+                Y = po.labels_from_scores(o["base"][t, st], 0.5)
+                want = po.detect_contexts(Y, Y_prev, contexts, accs, 0.6, S_prev, False)
+                assert want == o["used_sets"][t + 1][st], (st, t)
+                Y_prev, S_prev = Y, want
     assert m.status() == 0
     m.close()
 
