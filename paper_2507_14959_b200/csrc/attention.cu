@@ -1,8 +1,8 @@
 // Attention of the bf16 build: softmax(q k^T / 8) v per (frame, head), head dim 64.
 //
-// Two kernels.  attention_tc_kernel (below, used up to 624 tokens) runs both contractions on the
-// tcgen05 tensor cores with the scores in tensor memory; attention_mma_kernel is the register-level
-// version kept for longer sequences:
+// Three kernels.  attention_pipe_kernel (up to 208 tokens) and attention_tc_kernel (up to 624 tokens)
+// run both contractions on the tcgen05 tensor cores with the scores in tensor memory;
+// attention_mma_kernel is the register-level version kept for longer sequences:
 //
 // One CTA owns one (frame, head) (or a slice of its query rows when there are more than 256):
 // K and V of the head are staged once in shared memory (16-byte chunks XOR-swizzled by row so
@@ -189,8 +189,9 @@ __global__ void __launch_bounds__(512) attention_mma_kernel(const bf16* __restri
 // yields each row's maximum over all keys, the second forms P against that final maximum and
 // accumulates O over the blocks, so no rescaling of O is ever needed.
 // The issuing thread and the softmax warps alternate through two mbarriers (scores / O ready,
-// rows done); with one key block three CTAs fit an SM: two hold tensor memory and compute while the
-// third, whose loads were issued before it asked for tensor memory, waits for columns.
+// rows done).  ATT_SHARES softmax warps per lane quarter split the key columns of a block; they
+// exchange row maxima and row sums through shared memory.  (One key block goes to the pipelined
+// kernel further down.)
 // ---------------------------------------------------------------------------------------
 constexpr int AQ = 128;                    // query rows per tile
 constexpr int AKB = 208;                   // keys per score block
