@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 METRIC = "frames/sec (ViT-base, 1-3 LoRA adapters/frame)"
 UNIT = "frames/s"
 # DRAM bytes per fused-GEMM launch from the ncu capture summarised in profiles/ (None until taken)
-GEMM_DRAM_TRAFFIC_BYTES = 317e6     # mean over qkv / proj / fc1 / fc2 launches
+GEMM_DRAM_TRAFFIC_BYTES = 318e6     # mean over qkv / proj / fc1 / fc2 launches
 
 
 def measured_peaks():
