@@ -173,6 +173,35 @@ def test_recorded_launch_sequence_replays_identically():
     m.close()
 
 
+@pytest.mark.parametrize("dtype", [1, 0])
+def test_ragged_ranks_odd_frame_count_full_sets(dtype):
+    """Edge shapes in one batch: 3 frames (591 rows: a ragged last tile), adapter ranks that are not
+    multiples of the 16-rank slab (4, 24, 16, 40: one to three slabs, the last one partly empty), one frame
+    with every adapter active (|S| = max_set), one with none, one with a single multi-slab adapter."""
+    from paper_2507_14959_b200 import binding
+    name = "deit_tiny_ragged"
+    spec = wl.tiny_spec(32)
+    bb = wl.make_backbone(name, spec)
+    ads = [wl.make_adapter(name, spec, a, r, np.arange(8 * a, 8 * a + 8), ab_std=0.05)
+           for a, r in enumerate([4, 24, 16, 40])]
+    off, ids = wl.sets_to_csr([[0, 1, 2, 3], [], [3]])
+    w = wl.Workload(name, spec, bb, ads, wl.make_frames(name, spec, 3), off, ids)
+    m = binding.model_from_workload(w, dtype=dtype, max_frames=3, max_set=4)
+    s_, b_ = run_forward(m, w, dtype)
+    so, bo = oracle_rows(w, range(3))
+    assert np.abs(s_ - so).max() < SCORE_TOL[dtype]
+    assert np.abs(b_ - bo).max() < SCORE_TOL[dtype]
+    assert np.all(s_[1] == 0) and np.all(s_[2, :24] == 0) and np.all(s_[0] > 0)
+    # the adapters matter at this size of A and B: dropping them moves the base scores well past the tolerance
+    off0, ids0 = wl.sets_to_csr([[], [], []])
+    _, bo_plain = oracle_rows(w, range(3), offsets=off0, ids=ids0)
+    assert np.abs(bo[0] - bo_plain[0]).max() > 3e-2
+    # one frame alone (a single, mostly empty tile)
+    s1, b1 = run_forward(m, w, dtype, frames=w.frames[:1], offsets=off[:2], ids=ids[:4])
+    assert np.abs(s1 - so[:1]).max() < SCORE_TOL[dtype] and np.abs(b1 - bo[:1]).max() < SCORE_TOL[dtype]
+    m.close()
+
+
 def test_forward_argument_errors():
     import torch
     from paper_2507_14959_b200 import binding
