@@ -468,10 +468,12 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ z, const T* _
 
 __device__ __forceinline__ float sigmoidf_acc(float v) { return 1.f / (1.f + expf(-v)); }
 
-// grid (ceil(K/8), ceil(F/32)): a warp keeps the weight row of one class in registers and walks 32
-// slots, so the weights are read once per 32 frames; base_out rows are in the caller's order
-constexpr int BASE_HEAD_FRAMES = 32;
-template <typename T>
+// grid (ceil(K/8), ceil(F/8)): a warp keeps the weight row of one class in registers and walks 8
+// slots (a longer walk is a longer chain of load latencies); base_out rows are in the caller's order.
+// NV = ceil(d / 32) values per lane.  All loads of a z row are issued before the first multiply-add
+// (the walk is bound by the latency of those loads), and the dot product runs in four chains.
+constexpr int BASE_HEAD_FRAMES = 8;
+template <typename T, int NV>
 __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict__ z, const T* __restrict__ wt,
                                                         const float* __restrict__ bias,
                                                         const int* __restrict__ perm, int d, int n_classes,
@@ -479,10 +481,9 @@ __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict_
     const int k = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (k >= n_classes) return;
-    constexpr int MAXV = 32;                      // d <= 1024: at most 32 weights per lane
-    float w[MAXV];
+    float w[NV];
 #pragma unroll
-    for (int i = 0; i < MAXV; ++i) {
+    for (int i = 0; i < NV; ++i) {
         const int c = lane + 32 * i;
         w[i] = c < d ? to_f(wt[(size_t)k * d + c]) : 0.f;
     }
@@ -490,14 +491,17 @@ __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict_
     const int s0 = blockIdx.y * BASE_HEAD_FRAMES, s1 = min(n_frames, s0 + BASE_HEAD_FRAMES);
     for (int slot = s0; slot < s1; ++slot) {
         const float* zr = z + (size_t)slot * d;
-        float acc = 0.f;
+        float zv[NV];
 #pragma unroll
-        for (int i = 0; i < MAXV; ++i) {
+        for (int i = 0; i < NV; ++i) {
             const int c = lane + 32 * i;
-            if (c < d) acc = fmaf(zr[c], w[i], acc);
+            zv[i] = c < d ? __ldg(zr + c) : 0.f;
         }
-        acc = warp_sum(acc);
-        if (lane == 0) base_out[(size_t)perm[slot] * n_classes + k] = sigmoidf_acc(acc + bk);
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < NV; ++i) acc[i & 3] = fmaf(zv[i], w[i], acc[i & 3]);
+        const float dot = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
+        if (lane == 0) base_out[(size_t)perm[slot] * n_classes + k] = sigmoidf_acc(dot + bk);
     }
 }
 
@@ -538,7 +542,10 @@ cudaError_t launch_heads(const Launch& L, const T* x, int n_slots, int n_out_fra
     BUMP(L);
     if (base_out && n_base_slots > 0) {
         dim3 grid((n_classes + 7) / 8, (n_base_slots + BASE_HEAD_FRAMES - 1) / BASE_HEAD_FRAMES);
-        base_head_kernel<T><<<grid, 256, 0, L.st>>>(z, base_wt, base_b, R.perm, d, n_classes, n_base_slots, base_out);
+        const int nv = (d + 31) / 32;                  // d <= 1024
+        auto kern = nv <= 6 ? base_head_kernel<T, 6> : nv <= 12 ? base_head_kernel<T, 12>
+                  : nv <= 24 ? base_head_kernel<T, 24> : base_head_kernel<T, 32>;
+        kern<<<grid, 256, 0, L.st>>>(z, base_wt, base_b, R.perm, d, n_classes, n_base_slots, base_out);
         BUMP(L);
     }
     cudaError_t e = cudaMemsetAsync(scores_out, 0, (size_t)n_out_frames * n_classes * sizeof(float), L.st);
