@@ -168,7 +168,11 @@ int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames,
  *   next_offsets  dev int32 [n_frames+1]; next_ids dev int32 [ids_capacity]: CSR of S_t,
  *                 ascending ids.  If the result needs more than ids_capacity entries the lists are
  *                 truncated and PM_ERR_CAPACITY is recorded in the status word.
- * Needs pm_set_cover.  prev_* and next_* must not alias. */
+ * Needs pm_set_cover.  prev_* and next_* must not alias.  n_frames may differ from call to call.
+ * An id in prev_ids outside [0, max_adapters), or a malformed prev_offsets pair, is skipped and
+ * PM_ERR_ARG is recorded in the status word.  Calls on one handle share scratch memory: enqueue them
+ * on one stream (or order them).
+ * Every call also adds to the handle's stream-metric counters (see pm_metrics_read). */
 int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, int context_copy,
               int has_prev, uint32_t* prev_labels,
               const int32_t* prev_offsets, const int32_t* prev_ids,
@@ -196,14 +200,17 @@ int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, i
  *   provider   dev uint64 [n_classes, ceil(n_adapters/64)]: bit a of row k set iff adapter a lists
  *              class k with accuracy >= tau (the tables pm_set_cover builds inside a handle)
  *   status_out dev int32 or NULL: cleared by the call, then PM_ERR_CAPACITY is stored if the id list
- *              did not fit in ids_capacity (the lists are truncated).  With NULL the condition is
- *              not reported.
- * Errors: PM_ERR_ARG (NULL / non-positive sizes), PM_ERR_CAPACITY (n_frames >
- * PM_SELECT_STATIC_MAX_FRAMES or n_adapters > PM_SELECT_STATIC_MAX_ADAPTERS; nothing is launched),
- * PM_ERR_CUDA.
+ *              did not fit in ids_capacity (the lists are truncated), or PM_ERR_ARG if `first` or
+ *              the previous lists hold an adapter id outside [0, n_adapters) or a malformed offset
+ *              pair (such entries are skipped, nothing is read or written out of range because of
+ *              them).  With NULL the conditions are not reported.
+ * Errors: PM_ERR_ARG (NULL / non-positive sizes; a stream that belongs to another device than the
+ * current one), PM_ERR_CAPACITY (n_frames > PM_SELECT_STATIC_MAX_FRAMES or n_adapters >
+ * PM_SELECT_STATIC_MAX_ADAPTERS; nothing is launched), PM_ERR_CUDA.
  * Set-up: the first call on each device looks up the device address of the array (with that
  * device current -- make the stream's device current before calling).  Make that first call
- * before starting any stream capture.
+ * before starting any stream capture.  Host threads may call concurrently (subject to the sharing
+ * rule below); threads that race through a device's first call each do the look-up.
  * Sharing: all calls on a device use the same array and it keeps the previous call's contents.
  * The call clears the two words that must start at zero (status, block counter) on the stream; every
  * other word it reads it has written first.  Two calls whose kernels may overlap on the GPU --
@@ -216,6 +223,16 @@ int pm_select_static(const float* scores, int n_frames, int n_classes, int n_ada
                      const int32_t* first, const uint64_t* provider,
                      int32_t* next_offsets, int32_t* next_ids, int ids_capacity,
                      int32_t* status_out, void* cuda_stream);
+
+/* Stream metrics of Sec. 3.4, counted on the device by pm_select over the sets it chooses:
+ *   frames    number of (stream, step) selections made
+ *   contexts  sum of |S_t| over them          -> AvgCoverage (Eq. 7) = contexts / frames
+ *   switches  number of selections with has_prev whose S_t differs from S_{t-1}   (SwitchPenalty, Eq. 8)
+ * pm_metrics_reset zeroes the counters on the stream; pm_metrics_read synchronises the stream and
+ * copies them out (host pointers, each may be NULL).  Replayed CUDA graphs of pm_select count too. */
+int pm_metrics_reset(pm_handle h, void* cuda_stream);
+int pm_metrics_read(pm_handle h, void* cuda_stream, long long* frames, long long* contexts,
+                    long long* switches);
 
 /* Synchronises the stream and returns the device status word (PM_OK or the first recorded
  * error), then clears it. */

@@ -21,7 +21,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
 
 EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
-    "pm_select_static", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
+    "pm_select_static", "pm_metrics_reset", "pm_metrics_read", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention", "pm_cooccurrence", "pm_build_contexts", "pm_intra_coherence",
 ]
@@ -80,6 +80,8 @@ def load():
     lib.pm_select.argtypes = [vp, vp, ip, C.c_float, ip, ip, vp, vp, vp, vp, vp, ip, vp]
     lib.pm_select_static.argtypes = [vp, ip, ip, ip, C.c_float, ip, ip, vp, vp, vp, vp, vp, vp, vp, ip, vp, vp]
     lib.pm_status.argtypes = [vp, vp]
+    lib.pm_metrics_reset.argtypes = [vp, vp]
+    lib.pm_metrics_read.argtypes = [vp, vp, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)]
     lib.pm_last_error.argtypes = [vp]
     lib.pm_last_error.restype = C.c_char_p
     lib.pm_launch_count.argtypes = [vp]
@@ -207,6 +209,16 @@ class Model:
 
     def status(self, stream=None):
         return self.lib.pm_status(self.handle, _stream_ptr(stream))
+
+    def metrics_reset(self, stream=None):
+        self._check(self.lib.pm_metrics_reset(self.handle, _stream_ptr(stream)), "pm_metrics_reset")
+
+    def metrics_read(self, stream=None):
+        """(frames, contexts, switches) counted by select() since the last reset; synchronises."""
+        f, c, s = C.c_longlong(0), C.c_longlong(0), C.c_longlong(0)
+        self._check(self.lib.pm_metrics_read(self.handle, _stream_ptr(stream), C.byref(f), C.byref(c), C.byref(s)),
+                    "pm_metrics_read")
+        return int(f.value), int(c.value), int(s.value)
 
     def set_graphs(self, on):
         """Switches the recording / replaying of the forward's launch sequence as CUDA graphs."""

@@ -421,7 +421,7 @@ struct pm_handle_s {
     AdapterMeta meta;
     bool heads_dirty = true;
     // cover tables
-    DevBuf first, provider, mask_scratch;
+    DevBuf first, provider, mask_scratch, metrics;
     bool cover_ready = false;
     long long launches = 0;
     Profiler prof;
@@ -822,9 +822,13 @@ int pm_set_cover(pm_handle h, float tau) {
         }
     CK(h->first.alloc(first.size() * sizeof(int)));
     CK(h->provider.alloc(prov.size() * sizeof(uint64_t)));
-    // per-frame adapter masks + the select kernel's block counter (zero between launches)
-    CK(h->mask_scratch.alloc(((size_t)h->cfg.max_frames * AW + 1) * sizeof(uint64_t)));
+    // the select kernel's block counter (word 0, zero between launches) + per-frame adapter masks
+    CK(h->mask_scratch.alloc((1 + (size_t)h->cfg.max_frames * AW) * sizeof(uint64_t)));
     CK(cudaMemset(h->mask_scratch.p, 0, h->mask_scratch.bytes));
+    if (!h->metrics.p) {
+        CK(h->metrics.alloc(3 * sizeof(unsigned long long)));
+        CK(cudaMemset(h->metrics.p, 0, h->metrics.bytes));
+    }
     CK(cudaMemcpy(h->first.p, first.data(), first.size() * sizeof(int), cudaMemcpyHostToDevice));
     CK(cudaMemcpy(h->provider.p, prov.data(), prov.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
     h->cover_ready = true;
@@ -981,7 +985,28 @@ int pm_select(pm_handle h, const float* scores, int n_frames, float score_thr, i
     CK(launch_select(L, scores, n_frames, h->cfg.n_classes, h->cfg.max_adapters, score_thr, context_copy,
                      has_prev, prev_labels, prev_offsets, prev_ids, h->first.as<int>(),
                      h->provider.as<uint64_t>(), h->mask_scratch.as<uint64_t>(), next_offsets, next_ids,
-                     ids_capacity));
+                     ids_capacity, h->metrics.as<unsigned long long>()));
+    return PM_OK;
+}
+
+int pm_metrics_reset(pm_handle h, void* cuda_stream) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    if (!h->metrics.p) { err = "pm_set_cover has not been called"; return PM_ERR_STATE; }
+    CK(cudaMemsetAsync(h->metrics.p, 0, h->metrics.bytes, (cudaStream_t)cuda_stream));
+    return PM_OK;
+}
+
+int pm_metrics_read(pm_handle h, void* cuda_stream, long long* frames, long long* contexts, long long* switches) {
+    if (!h) return PM_ERR_ARG;
+    std::string& err = h->err;
+    if (!h->metrics.p) { err = "pm_set_cover has not been called"; return PM_ERR_STATE; }
+    unsigned long long v[3] = {0, 0, 0};
+    CK(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    CK(cudaMemcpy(v, h->metrics.p, sizeof(v), cudaMemcpyDeviceToHost));
+    if (frames) *frames = (long long)v[0];
+    if (contexts) *contexts = (long long)v[1];
+    if (switches) *switches = (long long)v[2];
     return PM_OK;
 }
 

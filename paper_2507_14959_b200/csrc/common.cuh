@@ -178,7 +178,8 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
                           int n_adapters, float thr, int context_copy, int has_prev,
                           uint32_t* prev_labels, const int* prev_off, const int* prev_ids,
                           const int* first, const uint64_t* provider, uint64_t* mask_scratch,
-                          int* next_off, int* next_ids, int ids_capacity);
+                          int* next_off, int* next_ids, int ids_capacity,
+                          unsigned long long* metrics = nullptr);   // [frames, sum |S_t|, switches] or null
 
 // tensor-map helpers (gemm_tcgen05.cu); return false if the driver entry point is unavailable
 bool tm_encode_2d(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer,

@@ -2,6 +2,7 @@
 // segmented heads + sigmoid + merge, Algorithm 2 selection, and the plain CUDA-core kernels of
 // the fp32 debug build (linear with unmerged LoRA terms, attention).
 #include <algorithm>
+#include <atomic>
 
 #include "common.cuh"
 
@@ -569,8 +570,11 @@ template cudaError_t launch_heads<bf16>(const Launch&, const bf16*, int, int, in
 // in visiting order, so it reduces to a table lookup and a bit-mask OR.
 // Phase 1 (all blocks): threshold -> label bit set -> keep / copy / greedy -> adapter bit mask and
 // its population count per frame.  Phase 2 (the block that finishes last, found with a counter in
-// the scratch area): prefix sum of the counts and emission of the sorted id lists.  `masks` holds
-// n_frames * ceil(n_adapters/64) words followed by one counter word that is zero between launches.
+// the scratch area): prefix sum of the counts and emission of the sorted id lists.  `scratch` holds
+// the counter in word 0 (zero between launches; its place does not depend on the frame count, so
+// calls with different batch sizes may follow each other on one scratch area) and, from word 1 on,
+// n_frames * ceil(n_adapters/64) mask words.  Adapter ids read from prev_ids / first that fall
+// outside [0, n_adapters) are skipped and reported as PM_ERR_ARG in the status word.
 constexpr int SELECT_THREADS = 256;
 
 __global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __restrict__ scores, int n_frames,
@@ -581,24 +585,34 @@ __global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __r
                                                       const int* __restrict__ prev_ids,
                                                       const int* __restrict__ first,
                                                       const uint64_t* __restrict__ provider,
-                                                      uint64_t* masks,
+                                                      uint64_t* scratch,
                                                       int* next_off,
                                                       int* __restrict__ next_ids, int ids_capacity,
-                                                      int* __restrict__ status) {
+                                                      int* __restrict__ status,
+                                                      unsigned long long* __restrict__ metrics) {
     __shared__ int partial[SELECT_THREADS];
     __shared__ int is_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = SELECT_THREADS >> 5;
     const int NW = (n_classes + 31) / 32;
     const int AW = (n_adapters + 63) / 64;     // <= 4 (checked on the host)
-    unsigned int* done = reinterpret_cast<unsigned int*>(masks + (size_t)n_frames * AW);
+    unsigned int* done = reinterpret_cast<unsigned int*>(scratch);
+    uint64_t* masks = scratch + 1;
 
     const int f = blockIdx.x * nwarps + warp;
     if (f < n_frames) {
         uint64_t prev_mask[4] = {0, 0, 0, 0}, greedy[4] = {0, 0, 0, 0};
         if (has_prev) {
-            for (int i = prev_off[f] + lane; i < prev_off[f + 1]; i += 32) {
-                const int a = prev_ids[i];
-                prev_mask[a >> 6] |= 1ull << (a & 63);
+            // a valid S_{t-1} has at most n_adapters distinct ids; anything else is a caller error
+            const int p0 = prev_off[f];
+            int pn = prev_off[f + 1] - p0;
+            if (p0 < 0 || pn < 0 || pn > n_adapters) {
+                if (lane == 0) atomicCAS(status, 0, (int)PM_ERR_ARG);
+                pn = 0;
+            }
+            for (int i = lane; i < pn; i += 32) {
+                const int a = prev_ids[p0 + i];
+                if ((unsigned)a < (unsigned)n_adapters) prev_mask[a >> 6] |= 1ull << (a & 63);
+                else atomicCAS(status, 0, (int)PM_ERR_ARG);
             }
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
@@ -631,8 +645,9 @@ __global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __r
                     bool cov = false;
                     for (int q = 0; q < AW; ++q) cov |= (provider[(size_t)k * AW + q] & prev_mask[q]) != 0;
                     if (!cov) covered = false;
-                    const int a = first[k];
-                    if (a >= 0) greedy[a >> 6] |= 1ull << (a & 63);
+                    const int a = first[k];                 // -1: nobody provides this label
+                    if ((unsigned)a < (unsigned)n_adapters) greedy[a >> 6] |= 1ull << (a & 63);
+                    else if (a != -1) atomicCAS(status, 0, (int)PM_ERR_ARG);
                 }
             }
         }
@@ -645,12 +660,16 @@ __global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __r
         }
         const bool keep = has_prev && ((prev_labels != nullptr && same) || (context_copy && covered));
         int cnt = 0;
+        bool changed = false;
         for (int q = 0; q < AW; ++q) {
             const uint64_t m = keep ? prev_mask[q] : greedy[q];
             cnt += __popcll(m);
+            changed |= m != prev_mask[q];
             if (lane == 0) masks[(size_t)f * AW + q] = m;
         }
         if (lane == 0) next_off[f + 1] = cnt;
+        // Eq. 8: one switch per stream and step whose chosen set differs from the previous one
+        if (lane == 0 && metrics && has_prev && changed) atomicAdd(metrics + 2, 1ull);
     }
     // ---- the last block to arrive here does the scan and the emission
     __threadfence();
@@ -676,6 +695,11 @@ __global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __r
     }
     int run = partial[threadIdx.x] - s;        // exclusive prefix of this chunk
     if (threadIdx.x == 0) { voff[0] = 0; *done = 0u; }
+    if (threadIdx.x == SELECT_THREADS - 1 && metrics) {
+        // Eq. 7: frames seen and active contexts chosen (their ratio is AvgCoverage)
+        atomicAdd(metrics + 0, (unsigned long long)n_frames);
+        atomicAdd(metrics + 1, (unsigned long long)partial[threadIdx.x]);
+    }
     for (int g = lo; g < hi; ++g) {
         run += voff[g + 1];
         voff[g + 1] = run;
@@ -703,12 +727,12 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
                           int n_adapters, float thr, int context_copy, int has_prev,
                           uint32_t* prev_labels, const int* prev_off, const int* prev_ids,
                           const int* first, const uint64_t* provider, uint64_t* mask_scratch,
-                          int* next_off, int* next_ids, int ids_capacity) {
+                          int* next_off, int* next_ids, int ids_capacity, unsigned long long* metrics) {
     ProfScope ps(L, KC_OTHER);
     const int blocks = n_frames > 0 ? (n_frames + SELECT_THREADS / 32 - 1) / (SELECT_THREADS / 32) : 1;
     select_kernel<<<blocks, SELECT_THREADS, 0, L.st>>>(scores, n_frames, n_classes, n_adapters, thr, context_copy,
                                         has_prev, prev_labels, prev_off, prev_ids, first, provider,
-                                        mask_scratch, next_off, next_ids, ids_capacity, L.status);
+                                        mask_scratch, next_off, next_ids, ids_capacity, L.status, metrics);
     BUMP(L);
     return cudaGetLastError();
 }
@@ -724,14 +748,17 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
 // can still run the selection.  Every GPU that loads the library carries the array until exit.
 #define PM_SELECT_STATIC_WORDS (PM_SELECT_STATIC_MAX_FRAMES * (PM_SELECT_STATIC_MAX_ADAPTERS / 64))
 
-static __device__ __align__(256) unsigned long long pm_select_static_masks[PM_SELECT_STATIC_WORDS + 1];   // + block counter
+static __device__ __align__(256) unsigned long long pm_select_static_masks[1 + PM_SELECT_STATIC_WORDS];   // block counter, then the masks
 static __device__ __align__(256) int pm_select_static_status[64];   // word 0: status when the caller passes none
 
 namespace {
 constexpr int STATIC_MAX_DEVICES = 64;
 struct StaticScratch { uint64_t* masks; int* status; };
 StaticScratch g_static_scratch[STATIC_MAX_DEVICES];       // device addresses, per device ordinal
-bool g_static_ready[STATIC_MAX_DEVICES];
+// set (release) once a device's addresses are stored; host threads that see it (acquire) may use them.
+// Two threads racing through the first call on a device both look the addresses up and store the
+// same values.
+std::atomic<bool> g_static_ready[STATIC_MAX_DEVICES];
 }  // namespace
 
 extern "C" int pm_select_static(const float* scores, int n_frames, int n_classes, int n_adapters,
@@ -748,7 +775,14 @@ extern "C" int pm_select_static(const float* scores, int n_frames, int n_classes
         return PM_ERR_CAPACITY;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return PM_ERR_CUDA;
-    if (!g_static_ready[dev]) {
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (st != nullptr && st != cudaStreamLegacy && st != cudaStreamPerThread) {
+        // the scratch array is per device: the stream must belong to the current one
+        int sdev = -1;
+        if (cudaStreamGetDevice(st, &sdev) != cudaSuccess) { cudaGetLastError(); return PM_ERR_CUDA; }
+        if (sdev != dev) return PM_ERR_ARG;
+    }
+    if (!g_static_ready[dev].load(std::memory_order_acquire)) {
         // The array's name is only a host-side stand-in here: ask the runtime for the device address
         // of this device's copy (the current device is the one the stream belongs to).
         void *m = nullptr, *s = nullptr;
@@ -759,15 +793,13 @@ extern "C" int pm_select_static(const float* scores, int n_frames, int n_classes
         }
         g_static_scratch[dev].masks = static_cast<uint64_t*>(m);
         g_static_scratch[dev].status = static_cast<int*>(s);
-        g_static_ready[dev] = true;
+        g_static_ready[dev].store(true, std::memory_order_release);
     }
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int* status = status_out ? status_out : g_static_scratch[dev].status;
-    // what must start at zero: the status word and the kernel's block counter (the word after the
-    // last mask word of this call); the mask words themselves are all rewritten before they are read
-    const size_t counter_at = (size_t)n_frames * ((n_adapters + 63) / 64);
+    // what must start at zero: the status word and the kernel's block counter (word 0 of the array);
+    // the mask words themselves are all rewritten before they are read
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess ||
-        cudaMemsetAsync(g_static_scratch[dev].masks + counter_at, 0, sizeof(uint64_t), st) != cudaSuccess)
+        cudaMemsetAsync(g_static_scratch[dev].masks, 0, sizeof(uint64_t), st) != cudaSuccess)
         return PM_ERR_CUDA;
     Launch L;
     L.st = st;

@@ -6,9 +6,10 @@ the forward is pm_forward_device_sets, which also builds its routing plan on the
 involves no host synchronisation at all and can be recorded once as a CUDA graph and replayed
 (``capture`` / ``step_graph``); without it pm_forward copies the lists to the host to plan there.
 
-Also counts the two stream-level metrics of the paper on the sets that were actually used:
-AvgCoverage (Eq. 7, mean number of active contexts per frame) and SwitchPenalty (Eq. 8, number of
-steps at which a stream's set changed).
+The two stream-level metrics of the paper -- AvgCoverage (Eq. 7, mean number of active contexts per
+frame) and SwitchPenalty (Eq. 8, number of steps at which a stream's set changed) -- are counted on
+the device by pm_select over the sets it chooses (pm_metrics_read); nothing here touches the id lists
+on the host unless ``record`` asks for them.
 """
 from __future__ import annotations
 
@@ -95,29 +96,19 @@ class StreamRunner:
         return [list(map(int, i[o[f]:o[f + 1]])) for f in range(self.S)]
 
 
-def avg_coverage(sets_per_step):
-    """Eq. 7 over all streams: mean |S_t| per frame."""
-    n = sum(len(step) for step in sets_per_step)
-    return sum(len(s) for step in sets_per_step for s in step) / max(n, 1)
-
-
-def switch_penalty(sets_per_step):
-    """Eq. 8 summed over streams: number of (stream, t >= 1) with S_t != S_{t-1}."""
-    total = 0
-    for t in range(1, len(sets_per_step)):
-        total += sum(1 for a, b in zip(sets_per_step[t - 1], sets_per_step[t]) if sorted(a) != sorted(b))
-    return total
-
-
 def run(model, frames_seq, n_classes, n_adapters, score_thr=0.5, context_copy=False, record=True,
         device_plan=True, graph=False):
     """frames_seq: device tensor [n_streams, n_steps, 3, img, img].  Free-running loop over all steps
     (graph: steps after the first are CUDA-graph replays).  Returns {"used_sets": per step the sets the forward used, "base": [n_steps, S, K] numpy,
-    "scores": same, "avg_coverage", "switch_penalty"} (records only if `record`)."""
+    "chosen_sets": per step the sets pm_select chose for the next frame, "scores": same} (only if
+    `record`; recording copies the lists to the host every step) and always "avg_coverage" (Eq. 7) and
+    "switch_penalty" (Eq. 8, summed over streams) of the chosen sets, read once from the device counters
+    after the last step."""
     S, T = int(frames_seq.shape[0]), int(frames_seq.shape[1])
     r = StreamRunner(model, S, n_classes, n_adapters, score_thr, context_copy, device_plan)
     r.reset()
-    used, base_log, score_log = [], [], []
+    model.metrics_reset()
+    used, chosen, base_log, score_log = [], [], [], []
     static = frames_seq[:, 0].contiguous() if graph else None
     for t in range(T):
         if record:
@@ -130,12 +121,13 @@ def run(model, frames_seq, n_classes, n_adapters, score_thr=0.5, context_copy=Fa
         else:
             scores, base = r.step(frames_seq[:, t].contiguous())
         if record:
+            chosen.append(r.current_sets())
             base_log.append(base.cpu().numpy().copy())
             score_log.append(scores.cpu().numpy().copy())
     if model.status() != 0:
         raise RuntimeError("device status word set during the streaming loop")
-    out = {"runner": r}
+    n, contexts, switches = model.metrics_read()
+    out = {"runner": r, "avg_coverage": contexts / max(n, 1), "switch_penalty": switches}
     if record:
-        out.update(used_sets=used, base=np.stack(base_log), scores=np.stack(score_log),
-                   avg_coverage=avg_coverage(used), switch_penalty=switch_penalty(used))
+        out.update(used_sets=used, chosen_sets=chosen, base=np.stack(base_log), scores=np.stack(score_log))
     return out

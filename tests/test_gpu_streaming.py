@@ -9,22 +9,23 @@ import workloads as wl
 from oracle import polymorph_oracle as po
 
 
-def test_stream_metrics_match_eq7_eq8():
-    from paper_2507_14959_b200 import streaming
-    # 2 streams, 4 steps
-    steps = [[[0], [1, 2]], [[0], [1, 2]], [[0, 3], [2]], [[0, 3], []]]
-    per_stream = [[s[i] for s in steps] for i in range(2)]
-    assert streaming.avg_coverage(steps) == pytest.approx(
-        sum(po.avg_coverage(seq) * len(seq) for seq in per_stream) / 8)
-    assert streaming.switch_penalty(steps) == sum(po.switch_penalty(seq) for seq in per_stream)
+def check_device_metrics(out, n_streams):
+    """AvgCoverage (Eq. 7) and SwitchPenalty (Eq. 8) counted on the device by pm_select against the
+    oracle's definitions applied, per stream, to the sequence of sets Algorithm 2 chose."""
+    chosen = out["chosen_sets"]
+    per_stream = [[step[s] for step in chosen] for s in range(n_streams)]
+    total = sum(len(seq) for seq in per_stream)
+    assert out["avg_coverage"] == pytest.approx(sum(po.avg_coverage(seq) * len(seq) for seq in per_stream) / total)
+    assert out["switch_penalty"] == sum(po.switch_penalty(seq) for seq in per_stream)
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("context_copy", [False, True])
-def test_free_running_streams_teacher_forced(context_copy):
+@pytest.mark.parametrize("context_copy,T", [(False, 30), (True, 5)])
+def test_free_running_streams_teacher_forced(context_copy, T):
+    """T = 30 is the full length of the streaming configuration (16 streams x 30 frames)."""
     import torch
     from paper_2507_14959_b200 import binding, streaming
-    S, T = 16, 5
+    S = 16
     w = wl.vit_base_384_streams(n_streams=S, n_steps=T)
     m = binding.model_from_workload(w, dtype=0, max_frames=S, max_set=8)
     m.set_cover(w.tau)
@@ -45,6 +46,8 @@ def test_free_running_streams_teacher_forced(context_copy):
             Y_prev, S_prev = Y, want
     sizes = [len(x) for step in used[1:] for x in step]
     assert 0 < np.mean(sizes) <= 8
+    assert out["chosen_sets"][:-1] == used[1:]                      # what select chose is what the next forward used
+    check_device_metrics(out, S)
     # forward: the oracle, given the sets the GPU used, reproduces sampled rows
     for (t, s) in [(1, 0), (T - 1, S - 1), (2, 7)]:
         off, ids = wl.sets_to_csr([used[t][s]])
@@ -96,6 +99,15 @@ def test_device_plan_and_graph_replay_match_host_plan():
                 want = po.detect_contexts(Y, Y_prev, contexts, accs, 0.6, S_prev, False)
                 assert want == o["used_sets"][t + 1][st], (st, t)
                 Y_prev, S_prev = Y, want
+    # the device-plan loop against the oracle, teacher-forced with the sets that loop used
+    for (t, st) in [(2, 1), (T - 1, S - 1)]:
+        off, ids = wl.sets_to_csr([outs[1]["used_sets"][t][st]])
+        so, bo = po.forward(w.backbone, w.adapters, fr[st:st + 1, t], off, ids, spec.heads, spec.patch,
+                            spec.ln_eps, spec.n_classes)
+        assert np.abs(outs[1]["scores"][t, st] - so[0]).max() < 1e-2
+        assert np.abs(outs[1]["base"][t, st] - bo[0]).max() < 1e-2
+    for o in outs:
+        check_device_metrics(o, S)
     assert m.status() == 0
     m.close()
 
