@@ -240,6 +240,16 @@ int pm_status(pm_handle h, void* cuda_stream);
 
 const char* pm_last_error(pm_handle h);
 
+/* Self-test of the bounded device-side waits (no counterpart in the paper: library diagnostics).
+ * Launches one small CTA built from the same wait helper as the tensor-core kernels: one thread waits,
+ * with a limit of limit_cycles GPU clock cycles (1 .. 1e8), on a barrier that is never signalled, the
+ * other warps wait on a second such barrier with the library's own limit.  Expected outcome, read
+ * after synchronising the stream: *status == PM_ERR_TIMEOUT (it is only written if it was 0),
+ * trace[0] == 1 (the wait gave up), trace[1] == 3 (the other warps left through the abort flag),
+ * trace[2] == 1 (tensor memory released).  Nothing faults and the context stays usable.
+ *   status  dev int32, trace dev int32 [3] (cleared by the call). */
+int pm_selftest_wait_timeout(long long limit_cycles, int32_t* status, int32_t* trace, void* cuda_stream);
+
 /* The forward entry points record their launch sequence as a CUDA graph the second time they are
  * called with the same buffers, sizes, stream and routing plan, and replay it from then on (the
  * adapter sets may change between replays only for pm_forward_device_sets, whose plan is built

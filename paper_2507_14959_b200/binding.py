@@ -23,7 +23,7 @@ EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
     "pm_select_static", "pm_metrics_reset", "pm_metrics_read", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
-    "pm_layernorm", "pm_attention", "pm_cooccurrence", "pm_build_contexts", "pm_intra_coherence",
+    "pm_layernorm", "pm_attention", "pm_selftest_wait_timeout", "pm_cooccurrence", "pm_build_contexts", "pm_intra_coherence",
 ]
 
 
@@ -102,6 +102,7 @@ def load():
     lib.pm_linear_destroy.restype = None
     lib.pm_layernorm.argtypes = [vp, vp, vp, vp, ip, ip, C.c_float, ip, vp]
     lib.pm_attention.argtypes = [vp, vp, ip, ip, ip, ip, vp]
+    lib.pm_selftest_wait_timeout.argtypes = [C.c_longlong, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -308,6 +309,13 @@ def attention(qkv, out, n_frames, tokens, heads, dtype, stream=None):
     rc = load().pm_attention(_ptr(qkv), _ptr(out), n_frames, tokens, heads, dtype, _stream_ptr(stream))
     if rc != PM_OK:
         raise PolymorphError(rc, "pm_attention")
+
+
+def selftest_wait_timeout(limit_cycles, status, trace, stream=None):
+    """pm_selftest_wait_timeout: status = torch CUDA int32 [1], trace = torch CUDA int32 [3]."""
+    rc = load().pm_selftest_wait_timeout(int(limit_cycles), _ptr(status), _ptr(trace), _stream_ptr(stream))
+    if rc != PM_OK:
+        raise PolymorphError(rc, "pm_selftest_wait_timeout")
 
 
 def select_static(scores, n_adapters, score_thr, context_copy, has_prev, prev_labels, prev_offsets, prev_ids,

@@ -1188,17 +1188,24 @@ int pm_attention(const void* qkv, void* out, int n_frames, int tokens, int heads
     } else if (attention_tc_supported(tokens)) {
         // the operator has no handle, hence no status word of its own: a bounded wait that expires is
         // reported through the return code of a later call on the same device
-        static int* status_word = nullptr;
+        // (one word per device, allocated on first use)
+        static std::atomic<int*> status_words[64];
+        int dev = 0, n_sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 ||
+            cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PM_ERR_CUDA;
+        int* status_word = status_words[dev].load(std::memory_order_acquire);
         if (!status_word) {
             if (cudaMalloc(&status_word, sizeof(int)) != cudaSuccess) return PM_ERR_OOM;
             if (cudaMemset(status_word, 0, sizeof(int)) != cudaSuccess) return PM_ERR_CUDA;
+            int* expected = nullptr;
+            if (!status_words[dev].compare_exchange_strong(expected, status_word, std::memory_order_acq_rel)) {
+                cudaFree(status_word);                    // another thread got there first
+                status_word = expected;
+            }
         }
         L.status = status_word;
         CUtensorMap tm_q, tm_kv;
         if (!attention_encode_maps((const bf16*)qkv, n_frames, tokens, heads, &tm_q, &tm_kv)) return PM_ERR_CUDA;
-        int dev = 0, n_sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return PM_ERR_CUDA;
         e = launch_attention_tc(L, tm_q, tm_kv, (bf16*)out, n_frames, tokens, heads, n_sms);
     } else {
         e = launch_attention_mma(L, (const bf16*)qkv, (bf16*)out, n_frames, tokens, heads);

@@ -1,8 +1,10 @@
 // Attention of the bf16 build: softmax(q k^T / 8) v per (frame, head), head dim 64.
 //
-// Three kernels.  attention_pipe_kernel (up to 208 tokens) and attention_tc_kernel (up to 624 tokens)
-// run both contractions on the tcgen05 tensor cores with the scores in tensor memory;
-// attention_mma_kernel is the register-level version kept for longer sequences:
+// Three kernels.  The two that serve the model shapes, attention_pipe_kernel (one key block, up to
+// 208 tokens: persistent, two query tiles in flight) and attention_tc_kernel (up to 624 tokens, several
+// key blocks), run both contractions on the tcgen05 tensor cores with scores and probabilities in
+// tensor memory; they are described where they are defined.  attention_mma_kernel is the
+// register-level kernel for sequences beyond 624 tokens:
 //
 // One CTA owns one (frame, head) (or a slice of its query rows when there are more than 256):
 // K and V of the head are staged once in shared memory (16-byte chunks XOR-swizzled by row so
@@ -785,12 +787,8 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
         pa.tokens = tokens; pa.heads = heads; pa.tpad = a.tpad; pa.nq = a.n_qtiles;
         pa.n_items = n_frames * heads; pa.out = out; pa.status = L.status;
         const size_t psmem = 2 * (size_t)APIPE_ITEM_BYTES + APIPE_XCHG_BYTES + 192;
-        static bool pipe_set = false;
-        if (!pipe_set) {
-            cudaError_t e = cudaFuncSetAttribute(attention_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psmem);
-            if (e != cudaSuccess) return e;
-            pipe_set = true;
-        }
+        static SmemGrant grant;
+        if (cudaError_t e = grant.ensure(attention_pipe_kernel, (int)psmem); e != cudaSuccess) return e;
         ProfScope ps(L, KC_ATTENTION);
         attention_pipe_kernel<<<std::min(pa.n_items, n_sms), APIPE_THREADS, psmem, L.st>>>(tm_q, tm_kv, pa);
         BUMP(L);
@@ -798,12 +796,8 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
     }
     // one block: 68 KB, three CTAs per SM (two computing, the third loading while it waits for TMEM)
     size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64 + 2 * ATT_MAX_SHARES * AQ * sizeof(float);
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<ATT_SHARES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        smem_set = smem;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant.ensure(attention_tc_kernel<ATT_SHARES>, (int)smem); e != cudaSuccess) return e;
     ProfScope ps(L, KC_ATTENTION);
     attention_tc_kernel<ATT_SHARES><<<n_frames * heads * a.q_split, 32 + 128 * ATT_SHARES, smem, L.st>>>(tm_q, tm_kv, a);
     BUMP(L);
@@ -819,12 +813,8 @@ cudaError_t launch_attention_mma(const Launch& L, const bf16* qkv, bf16* out, in
     const int tpad = groups * 16;
     const size_t smem = (size_t)tpad * 256;
     if (smem > 227 * 1024) return launch_attention_simple<bf16>(L, qkv, out, n_frames, tokens, heads);
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        smem_set = smem;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant.ensure(attention_mma_kernel, (int)smem); e != cudaSuccess) return e;
     ProfScope ps(L, KC_ATTENTION);
     dim3 grid(slices, n_frames * heads);
     attention_mma_kernel<<<grid, warps * 32, smem, L.st>>>(qkv, out, tokens, heads, tpad, warps * 16);

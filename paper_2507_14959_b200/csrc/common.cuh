@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <string>
 #include <vector>
 
@@ -180,6 +181,25 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
                           const int* first, const uint64_t* provider, uint64_t* mask_scratch,
                           int* next_off, int* next_ids, int ids_capacity,
                           unsigned long long* metrics = nullptr);   // [frames, sum |S_t|, switches] or null
+
+// cudaFuncSetAttribute acts on the current device only, so "already set" is remembered per device
+// ordinal: the largest dynamic shared-memory size granted to one kernel on each device.
+struct SmemGrant {
+    std::atomic<int> granted[64];
+    template <typename Kernel>
+    cudaError_t ensure(Kernel kernel, int bytes) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        std::atomic<int>& g = granted[dev & 63];
+        if (bytes <= g.load(std::memory_order_acquire)) return cudaSuccess;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e != cudaSuccess) return e;
+        int cur = g.load(std::memory_order_relaxed);
+        while (cur < bytes && !g.compare_exchange_weak(cur, bytes, std::memory_order_release)) {}
+        return cudaSuccess;
+    }
+};
 
 // tensor-map helpers (gemm_tcgen05.cu); return false if the driver entry point is unavailable
 bool tm_encode_2d(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer,

@@ -977,6 +977,53 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     }
 }
 
+// Exercises the give-up path of the bounded waits without any fault: one CTA with the warp roles of
+// the kernels above allocates tensor memory, then its "MMA" thread waits -- with the caller's cycle
+// limit -- on an mbarrier nothing ever arrives on.  The wait must expire, raise the abort flag and
+// record PM_ERR_TIMEOUT; the other warps, parked on a second barrier, must see the abort flag and
+// leave too; the CTA drains, frees its tensor memory and returns.  trace[0] = the timed-out wait
+// returned false, trace[1] = warps that left through the abort flag, trace[2] = 1 after the release.
+__global__ void __launch_bounds__(128) wait_timeout_selftest_kernel(long long limit, int* status, int* trace) {
+    __shared__ __align__(8) uint64_t bars[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars[0]), 1);
+        mbar_init(smem_u32(&bars[1]), 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_slot), 32);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    if (warp == 1) {
+        if (lane == 0) {
+            const bool ok = mbar_wait(smem_u32(&bars[0]), 0u, abort_flag, status, limit);
+            trace[0] = ok ? 0 : 1;
+        }
+    } else {
+        // like an epilogue warp waiting for an accumulator that never comes: ends through the abort flag
+        bool ok = mbar_wait(smem_u32(&bars[1]), 0u, abort_flag, status);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok && lane == 0) atomicAdd(&trace[1], 1);
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 32);
+        if (lane == 0) trace[2] = 1;
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -1004,6 +1051,15 @@ CUtensorMapSwizzle swz(int bytes) {
 }
 
 }  // namespace
+
+extern "C" int pm_selftest_wait_timeout(long long limit_cycles, int32_t* status, int32_t* trace, void* cuda_stream) {
+    // the other warps' own limit is the library's (~2 s): the test limit must stay far below it
+    if (!status || !trace || limit_cycles <= 0 || limit_cycles > 100000000ll) return PM_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(trace, 0, 3 * sizeof(int32_t), st) != cudaSuccess) return PM_ERR_CUDA;
+    wait_timeout_selftest_kernel<<<1, 128, 0, st>>>(limit_cycles, status, trace);
+    return cudaGetLastError() == cudaSuccess ? PM_OK : PM_ERR_CUDA;
+}
 
 bool tm_encode_2d(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer,
                   uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, int swizzle) {
@@ -1058,12 +1114,8 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     // follows (which walks front to back)
     a.reverse = (size_t)rows * lin.k_in * sizeof(bf16) > ((size_t)96 << 20) ? 1 : 0;
     const int smem = a.stages * stage_bytes + 256;
-    static int smem_set = 0;
-    if (smem > smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(shrink_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        smem_set = smem;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant.ensure(shrink_tc_kernel, smem); e != cudaSuccess) return e;
     const int per_sm = (2 * smem + 4096 <= 227 * 1024 && 4 * cols <= 512) ? 2 : 1;
     const int grid = R.n_tiles < n_sms * per_sm ? R.n_tiles : n_sms * per_sm;
     ProfScope ps(L, KC_SHRINK);
@@ -1082,13 +1134,8 @@ static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, cons
                                   const CUtensorMap& tm_t, const CUtensorMap& tm_bt, const CUtensorMap& tm_y,
                                   const GemmArgs& a, int n_sms) {
     constexpr int EW = GEMM_EPI_WARPS;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(lora_gemm_kernel<BN, EPI, EW, LNF>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, EW>::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant.ensure(lora_gemm_kernel<BN, EPI, EW, LNF>, Smem<BN, EW>::TOTAL); e != cudaSuccess) return e;
     const int total = a.m_tiles * a.n_tiles;
     const int grid = total < n_sms ? total : n_sms;
     ProfScope ps(L, KC_GEMM);
@@ -1124,13 +1171,8 @@ static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, co
         if (!tm_encode_2d(&tm_res, a.residual, a.n_out, a.rows, (uint64_t)a.n_out * 2, 32, 32, 64))
             return cudaErrorInvalidValue;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<EPI, LNF, RESS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             P_SMEM_TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant.ensure(lora_gemm_pair_kernel<EPI, LNF, RESS>, P_SMEM_TOTAL); e != cudaSuccess) return e;
     const int total = a.m_tiles * a.n_tiles;
     const int pairs = total < n_sms / 2 ? total : n_sms / 2;
     cudaLaunchConfig_t cfg = {};

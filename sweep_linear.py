@@ -1,8 +1,8 @@
 """Isolated fused base+LoRA linear sweep (the single-linear workload): times pm_linear_forward
 (shrink + fused GEMM) per cell and reports algorithmic TFLOP/s.
 
-  python -m paper_2507_14959_b200.sweep                      # the whole grid
-  python -m paper_2507_14959_b200.sweep --k 768 --n 2304 --frames 256 --rank 16 --sets unif --iters 3
+  python sweep_linear.py                      # the whole grid
+  python sweep_linear.py --k 768 --n 2304 --frames 256 --rank 16 --sets unif --iters 3
 
 Cells: M = 197*B tokens, B in {16, 64, 256}; K->N in {768->2304, 768->3072, 3072->768}; 128 registered
 adapters of rank in {8, 16, 32, 64}; 1-8 active adapters per frame, uniform or Zipf(1.2)-clustered;
@@ -17,7 +17,7 @@ import sys
 
 import numpy as np
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

@@ -45,7 +45,9 @@ def test_layernorm(dtype, rows, d):
 
 
 @pytest.mark.parametrize("dtype", [0, 1])
-@pytest.mark.parametrize("frames,tokens,heads", [(3, 197, 3), (1, 577, 2), (2, 10, 1), (2, 64, 2), (1, 130, 1)])
+@pytest.mark.parametrize("frames,tokens,heads", [(3, 197, 3), (1, 577, 2), (2, 10, 1), (2, 64, 2), (1, 130, 1),
+                                                 (2, 626, 2),      # beyond the tcgen05 kernels' 624 tokens
+                                                 (1, 785, 1)])     # 448x448 frames: several query slices
 def test_attention(dtype, frames, tokens, heads):
     import torch
     from paper_2507_14959_b200 import binding
@@ -132,26 +134,45 @@ def test_lora_linear(dtype, case):
     lin.close()
 
 
-def test_lora_linear_full_size_sampled():
-    """One cell of the single-linear grid at full size (256 frames x 197 tokens, 768 -> 2304, 128
-    rank-16 adapters, 1-8 active per frame) in the launch configuration the sweep times; the oracle
-    computes sampled rows one by one (first and last row tiles, frame boundaries, the ragged tail)."""
+FULL_SIZE_CELLS = [
+    # k_in, n_out, rank, clustered, epilogue
+    (768, 2304, 16, False, 0),
+    (3072, 768, 64, False, 2),      # rank 64 with up to 8 active adapters: the largest LoRA share
+    (768, 3072, 64, False, 1),
+    (768, 2304, 32, True, 0),       # Zipf-clustered sets
+    (3072, 768, 8, True, 2),        # rank below one slab
+]
+
+
+@pytest.mark.parametrize("k_in,n_out,rank,clustered,epi", FULL_SIZE_CELLS,
+                         ids=[f"{c[0]}x{c[1]}_r{c[2]}_{'zipf' if c[3] else 'unif'}_e{c[4]}" for c in FULL_SIZE_CELLS])
+def test_lora_linear_full_size_sampled(k_in, n_out, rank, clustered, epi):
+    """Cells of the single-linear grid at full size (256 frames x 197 tokens, 128 adapters of one
+    rank, 1-8 active per frame) in the launch configuration the sweep times; the oracle computes
+    sampled rows one by one: first and last row tiles, frame boundaries, the ragged tail, rows of
+    the frames with the most active adapters, and random rows."""
     import torch
     from paper_2507_14959_b200 import binding
-    cell = wl.linear_cell(768, 2304, 256, 16, clustered=False)
-    lin = binding.Linear(cell.w, cell.b, max_adapters=128, max_rank=16, max_set=8, max_frames=256,
-                         tokens=cell.tokens, epilogue=0, dtype=0)
+    cell = wl.linear_cell(k_in, n_out, 256, rank, clustered=clustered)
+    lin = binding.Linear(cell.w, cell.b, max_adapters=128, max_rank=rank, max_set=8, max_frames=256,
+                         tokens=cell.tokens, epilogue=epi, dtype=0)
     for a in range(128):
-        lin.register(a, 16, cell.scale, cell.A[a], cell.B[a])
+        lin.register(a, rank, cell.scale, cell.A[a], cell.B[a])
     rows = 256 * cell.tokens
     xd = to_dev(cell.x, 0)
-    yd = torch.full((rows, 2304), float("nan"), device="cuda", dtype=torch.bfloat16)
-    lin.forward(xd, 256, cell.set_offsets, cell.set_ids, yd)
+    res = wl.normal((rows, n_out), 1.0, cell.name, "res") if epi == 2 else None
+    rd = to_dev(res, 0) if epi == 2 else None
+    yd = torch.full((rows, n_out), float("nan"), device="cuda", dtype=torch.bfloat16)
+    lin.forward(xd, 256, cell.set_offsets, cell.set_ids, yd, residual=rd)
     assert lin.status() == 0
     assert not torch.isnan(yd.float()).any()
-    g = wl.rng_for("full_size_rows")
+    g = wl.rng_for("full_size_rows", k_in, n_out, rank)
+    sizes = np.diff(cell.set_offsets)
+    assert sizes.max() == 8
+    widest = [int(f) for f in np.argsort(-sizes, kind="stable")[:3]]
     sample = sorted(set([0, 127, 128, 196, 197, 198, rows - 1, rows - 65, rows - 128, rows - 129]
-                        + [int(r) for r in g.integers(0, rows, 54)]))
+                        + [f * cell.tokens + t for f in widest for t in (0, 100, 196)]
+                        + [int(r) for r in g.integers(0, rows, 48)]))
     got = to_np(yd[sample])
     w64, b64 = cell.w.astype(np.float64), cell.b.astype(np.float64)
     for i, r in enumerate(sample):
@@ -159,6 +180,10 @@ def test_lora_linear_full_size_sampled():
         act = [(cell.scale, cell.A[a].astype(np.float64), cell.B[a].astype(np.float64))
                for a in sorted(cell.set_ids[cell.set_offsets[f]:cell.set_offsets[f + 1]])]
         want = po.lora_linear(cell.x[r:r + 1].astype(np.float64), w64, b64, act)[0]
+        if epi == 1:
+            want = po.gelu(want)
+        elif epi == 2:
+            want = want + wl.round_bf16(res[r]).astype(np.float64)
         np.testing.assert_allclose(got[i], want, **TOL[0])
     lin.close()
 
@@ -212,3 +237,27 @@ def test_linear_argument_errors():
         lin.register(1, 32, 1.0, np.zeros((64, 32), np.float32), np.zeros((32, 64), np.float32))
     assert e.value.code == binding.PM_ERR_CAPACITY
     lin.close()
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A wait on a barrier that nothing signals runs into its limit, records PM_ERR_TIMEOUT, takes the
+    other warps of the CTA out through the abort flag and releases tensor memory; nothing faults and
+    the next kernel on the device runs normally."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    trace = torch.full((3,), -1, dtype=torch.int32, device="cuda")
+    binding.selftest_wait_timeout(100000, status, trace)
+    torch.cuda.synchronize()
+    assert int(status.item()) == binding.PM_ERR_TIMEOUT
+    assert trace.cpu().tolist() == [1, 3, 1]
+    # the context is intact: an ordinary operator right after
+    x = wl.normal((64, 128), 1.0, "after_timeout")
+    y = torch.zeros((64, 128), device="cuda")
+    binding.layernorm(torch.from_numpy(x).cuda(), torch.ones(128, device="cuda"), torch.zeros(128, device="cuda"),
+                      y, 1e-6, 1)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(y.cpu().numpy(), po.layernorm(x.astype(np.float64), np.ones(128), np.zeros(128), 1e-6),
+                               atol=2e-4)
+    with pytest.raises(binding.PolymorphError):
+        binding.selftest_wait_timeout(10 ** 12, status, trace)       # limits beyond 1e8 cycles are refused
