@@ -251,9 +251,9 @@ const char* pm_last_error(pm_handle h);
 int pm_selftest_wait_timeout(long long limit_cycles, int32_t* status, int32_t* trace, void* cuda_stream);
 
 /* The forward entry points record their launch sequence as a CUDA graph the second time they are
- * called with the same buffers, sizes, stream and routing plan, and replay it from then on (the
- * adapter sets may change between replays only for pm_forward_device_sets, whose plan is built
- * inside the recorded sequence).  Not on the legacy default stream, not while the caller's stream is
+ * called with the same buffers, sizes and stream and the same widest adapter set, and replay it
+ * from then on; the adapter sets themselves may change between replays (a new routing plan is
+ * uploaded, or built by the recorded kernels for pm_forward_device_sets, before the replay reads it).  Not on the legacy default stream, not while the caller's stream is
  * itself being captured, not while pm_profile_enable is on.  pm_set_graphs(h, 0) switches this off
  * and frees the recorded graphs; default on. */
 int pm_set_graphs(pm_handle h, int on);
@@ -263,12 +263,20 @@ long long pm_launch_count(pm_handle h);
 
 /* Device timing of the library's own kernels, by class, with CUDA events recorded on the launching
  * stream around each launch site: class 0 fused base+LoRA GEMM (patch embed included), 1 LoRA
- * shrink, 2 attention, 3 LayerNorm, 4 everything else (patch gather, CLS rows, heads, select).
- * pm_profile_enable(h, 1) clears and starts recording, (h, 0) stops.  pm_profile_read synchronises
- * the stream, returns total milliseconds and launch-site counts per class (arrays of 5) since the
- * last read, and clears them. */
+ * shrink, 2 attention, 3 LayerNorm / row statistics, 4 patch gather, CLS rows and branch fan-out,
+ * 5 final LayerNorm + heads + sigmoid + merge, 6 Algorithm 2 selection, 7 routing plan built on the
+ * device.  pm_profile_enable(h, 1) clears and starts recording, (h, 0) stops.  pm_profile_read
+ * synchronises the stream, returns total milliseconds and launch-site counts per class (arrays of
+ * PM_PROFILE_CLASSES) since the last read, and clears them. */
+#define PM_PROFILE_CLASSES 8
 int pm_profile_enable(pm_handle h, int on);
 int pm_profile_read(pm_handle h, void* cuda_stream, double* ms_by_class, long long* launches_by_class);
+
+/* Host-side cost of the routing plan (Sec. 3.2: frames are bucketed by adapter set before the fused
+ * linears run): number of plans pm_forward / pm_forward_branched have built on the host since the
+ * handle was created (a call whose sets equal the previous call's reuses the uploaded plan and builds
+ * nothing) and the total host time spent building them, in milliseconds.  Either pointer may be NULL. */
+int pm_plan_stats(pm_handle h, long long* plans_built, double* host_ms);
 
 /* ---- training-time context construction (Sec. 3.4) -------------------------------------- */
 

@@ -21,7 +21,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
 
 EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
-    "pm_select_static", "pm_metrics_reset", "pm_metrics_read", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_linear_create", "pm_linear_register",
+    "pm_select_static", "pm_metrics_reset", "pm_metrics_read", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_plan_stats", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention", "pm_selftest_wait_timeout", "pm_cooccurrence", "pm_build_contexts", "pm_intra_coherence",
 ]
@@ -92,6 +92,7 @@ def load():
     lib.pm_launch_count.restype = C.c_longlong
     lib.pm_profile_enable.argtypes = [vp, ip]
     lib.pm_profile_read.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
+    lib.pm_plan_stats.argtypes = [vp, C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
     lib.pm_linear_create.argtypes = [ip, ip, _FP, _FP, ip, ip, ip, ip, ip, ip, ip, C.POINTER(vp)]
     lib.pm_linear_register.argtypes = [vp, ip, ip, C.c_float, _FP, _FP]
     lib.pm_linear_forward.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
@@ -225,17 +226,23 @@ class Model:
         """Switches the recording / replaying of the forward's launch sequence as CUDA graphs."""
         self._check(self.lib.pm_set_graphs(self.handle, int(on)), "pm_set_graphs")
 
-    KERNEL_CLASSES = ("gemm", "shrink", "attention", "layernorm", "other")
+    KERNEL_CLASSES = ("gemm", "shrink", "attention", "layernorm", "other", "heads", "select", "plan")
 
     def profile_enable(self, on):
         self._check(self.lib.pm_profile_enable(self.handle, int(on)), "pm_profile_enable")
 
     def profile_read(self, stream=None):
         """{class: (total_ms, launch_sites)} since the last read; synchronises the stream."""
-        ms = (C.c_double * 5)()
-        n = (C.c_longlong * 5)()
+        ms = (C.c_double * len(self.KERNEL_CLASSES))()
+        n = (C.c_longlong * len(self.KERNEL_CLASSES))()
         self._check(self.lib.pm_profile_read(self.handle, _stream_ptr(stream), ms, n), "pm_profile_read")
         return {k: (ms[i], int(n[i])) for i, k in enumerate(self.KERNEL_CLASSES)}
+
+    def plan_stats(self):
+        """(plans built on the host, total host milliseconds spent building them)."""
+        n, ms = C.c_longlong(0), C.c_double(0.0)
+        self._check(self.lib.pm_plan_stats(self.handle, C.byref(n), C.byref(ms)), "pm_plan_stats")
+        return int(n.value), float(ms.value)
 
     def launch_count(self):
         return int(self.lib.pm_launch_count(self.handle))

@@ -2,6 +2,7 @@
 // (bucketing of frames by adapter set, tile -> LoRA slab lists) and the launch sequences.
 #include <algorithm>
 #include <array>
+#include <chrono>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -201,6 +202,8 @@ struct Router {
     int last_frames = -1;
     bool last_sorted = false;
     std::vector<int> perm_host;
+    long long plans_built = 0;       // host plans built (cache misses) and the host time they took
+    double plan_host_ms = 0.0;
 
     ~Router() {
         if (stage) cudaFreeHost(stage);
@@ -262,6 +265,7 @@ struct Router {
             (!fixed || (std::equal(frame_of_slot, frame_of_slot + n_frames, last_fixed.begin()) &&
                         std::equal(src_of_slot, src_of_slot + n_frames, last_fixed.begin() + n_frames))))
             return PM_OK;
+        const auto t_start = std::chrono::steady_clock::now();
         std::vector<std::vector<int>> sets(n_frames);
         int widest = 0;
         for (int f = 0; f < n_frames; ++f) {
@@ -337,6 +341,8 @@ struct Router {
             last_fixed.insert(last_fixed.end(), src_of_slot, src_of_slot + n_frames);
         }
         last_frames = n_frames; last_sorted = sort_frames;
+        ++plans_built;
+        plan_host_ms += std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_start).count();
         return PM_OK;
     }
     void invalidate() { last_frames = -1; }
@@ -862,7 +868,10 @@ int pm_forward(pm_handle h, const void* frames, int n_frames, const int32_t* set
     pm_handle_s::GraphEntry key;
     key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
     key.key_int[0] = n_frames; key.key_int[1] = 0 /* entry point */;
-    key.plan_version = h->router.version; key.st = st;
+    // the kernels read the plan from device tables at fixed addresses; of its contents only the widest
+    // set shapes the launch sequence, so a recorded sequence is replayed for any sets of the same width
+    key.key_int[2] = h->router.dev.max_set;
+    key.plan_version = 0; key.st = st;
     return run_graphed(h, key, [&]() {
         return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
                                  : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
@@ -964,7 +973,7 @@ int pm_forward_branched(pm_handle h, const void* frames, int n_frames, const int
     key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
     key.key_int[0] = n_frames; key.key_int[1] = 2 /* entry point */; key.key_int[2] = trunk_layers;
     key.key_int[3] = (int)n_slots;
-    key.plan_version = h->router.version; key.st = st;
+    key.plan_version = (unsigned long long)h->router.dev.max_set; key.st = st;
     return run_graphed(h, key, [&]() {
         return c.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st)
                             : forward_t<float>(h, frames, n_frames, (int)n_slots, trunk_layers, scores_out, base_out, st);
@@ -1050,6 +1059,13 @@ int pm_profile_read(pm_handle h, void* cuda_stream, double* ms_by_class, long lo
     return PM_OK;
 }
 long long pm_launch_count(pm_handle h) { return h ? h->launches : 0; }
+
+int pm_plan_stats(pm_handle h, long long* plans_built, double* host_ms) {
+    if (!h) return PM_ERR_ARG;
+    if (plans_built) *plans_built = h->router.plans_built;
+    if (host_ms) *host_ms = h->router.plan_host_ms;
+    return PM_OK;
+}
 
 int pm_set_graphs(pm_handle h, int on) {
     if (!h) return PM_ERR_ARG;

@@ -82,7 +82,8 @@ struct PatchEpi {               // EPI_PATCH: GEMM row i = patch (i % g2) of slo
 // every function enqueues on `st`, bumps *launches per kernel and returns a cudaError_t
 // ---------------------------------------------------------------------------------------
 // Optional per-kernel-class device timing (CUDA events on the launching stream).
-enum { KC_GEMM = 0, KC_SHRINK = 1, KC_ATTENTION = 2, KC_LAYERNORM = 3, KC_OTHER = 4, KC_COUNT = 5 };
+enum { KC_GEMM = 0, KC_SHRINK = 1, KC_ATTENTION = 2, KC_LAYERNORM = 3, KC_OTHER = 4, KC_HEADS = 5, KC_SELECT = 6,
+       KC_PLAN = 7, KC_COUNT = PM_PROFILE_CLASSES };
 struct Profiler {
     bool on = false;
     std::vector<cudaEvent_t> ev;     // pairs: 2*i start, 2*i+1 stop

@@ -538,7 +538,7 @@ cudaError_t launch_heads(const Launch& L, const T* x, int n_slots, int n_out_fra
                          const T* hcat, const float* hbias, const int* hcls, const int* hoff,
                          const RouteDev& R, float* scores_out, float* base_out) {
     if (n_slots <= 0) return cudaSuccess;
-    ProfScope ps(L, KC_OTHER);
+    ProfScope ps(L, KC_HEADS);
     final_ln_kernel<T><<<(n_slots + 7) / 8, 256, 0, L.st>>>(x, lnf_g, lnf_b, z, n_slots, tokens, d, eps);
     BUMP(L);
     if (base_out && n_base_slots > 0) {
@@ -728,7 +728,7 @@ cudaError_t launch_select(const Launch& L, const float* scores, int n_frames, in
                           uint32_t* prev_labels, const int* prev_off, const int* prev_ids,
                           const int* first, const uint64_t* provider, uint64_t* mask_scratch,
                           int* next_off, int* next_ids, int ids_capacity, unsigned long long* metrics) {
-    ProfScope ps(L, KC_OTHER);
+    ProfScope ps(L, KC_SELECT);
     const int blocks = n_frames > 0 ? (n_frames + SELECT_THREADS / 32 - 1) / (SELECT_THREADS / 32) : 1;
     select_kernel<<<blocks, SELECT_THREADS, 0, L.st>>>(scores, n_frames, n_classes, n_adapters, thr, context_copy,
                                         has_prev, prev_labels, prev_off, prev_ids, first, provider,

@@ -193,7 +193,7 @@ cudaError_t launch_device_plan(const Launch& L, const RouteDev& R, int n_frames,
                                int slabs_max, const int* off, const int* ids, const AdapterMeta& meta) {
     if (n_frames <= 0) return cudaSuccess;
     if (n_frames > PM_DEVICE_PLAN_MAX_FRAMES) return cudaErrorInvalidValue;
-    ProfScope ps(L, KC_OTHER);
+    ProfScope ps(L, KC_PLAN);
     plan_slots_kernel<<<1, PLAN_THREADS, 0, L.st>>>(n_frames, max_set, max_adapters, off, ids, meta.rank, R, L.status);
     BUMP(L);
     const long long rows = (long long)n_frames * R.tokens;

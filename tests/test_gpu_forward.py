@@ -69,6 +69,42 @@ def test_deit_tiny_2frames(dtype):
     m.close()
 
 
+def test_recorded_sequence_follows_changing_sets():
+    """On a stream of its own the third identical call replays a recorded launch sequence.  When the
+    sets then change (same widest set) the replay must use the newly uploaded routing plan: results
+    follow the new sets, checked against the oracle, and changing back gives the first bits again."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_2frames()
+    m = binding.model_from_workload(w, dtype=0)
+    fd = frames_to_dev(w.frames, 0)
+    K = w.spec.n_classes
+    side = torch.cuda.Stream()
+    sc, bs = torch.zeros((2, K), device="cuda"), torch.zeros((2, K), device="cuda")
+    torch.cuda.synchronize()
+    results = {}
+    plans0, _ = m.plan_stats()
+    with torch.cuda.stream(side):
+        n_before = m.launch_count()
+        for name, sets, reps in (("a", [[0], [1, 3]], 3), ("b", [[2, 3], [0]], 2), ("c", [[1], [0, 2]], 1),
+                                 ("a2", [[0], [1, 3]], 1)):
+            off, ids = wl.sets_to_csr(sets)
+            for _ in range(reps):
+                sc.fill_(-1.0)
+                m.forward(fd, off, ids, sc, bs)
+            assert m.status(side) == 0
+            results[name] = (sc.cpu().numpy().astype(np.float64), bs.cpu().numpy().astype(np.float64), off, ids)
+    assert m.plan_stats()[0] - plans0 == 4                 # one host plan per change of the sets
+    for name in ("a", "b", "c"):
+        s, b, off, ids = results[name]
+        so, bo = oracle_rows(w, range(2), offsets=off, ids=ids)
+        assert np.abs(s - so).max() < 1e-2 and np.abs(b - bo).max() < 1e-2
+    assert np.abs(results["a"][0] - results["b"][0]).max() > 1e-2     # the sets really differ in effect
+    np.testing.assert_array_equal(results["a2"][0], results["a"][0])
+    np.testing.assert_array_equal(results["a2"][1], results["a"][1])
+    m.close()
+
+
 @pytest.mark.parametrize("dtype", [1, 0])
 def test_paper_variant_query_value_last_blocks(dtype):
     """The paper's own placement of the adapters (Sec. 3.1, Sec. 4): LoRA on the query and value

@@ -201,6 +201,19 @@ def draw_set(g: np.random.Generator, n_adapters: int, size_probs=(0.6, 0.3, 0.1)
     return sorted(int(a) for a in g.choice(n_adapters, size=size, replace=False))
 
 
+def changing_sets(sets, n_steps: int, p: float, n_adapters: int, tag: str = ""):
+    """n_steps set lists starting from `sets`: at every step each frame redraws its set with
+    probability p (sizes 1/2/3 with probability 0.6/0.3/0.1, uniform distinct ids), else keeps it --
+    the slowly changing sets of a video stream (temporal continuity)."""
+    g = rng_for("changing_sets", tag, n_steps, p, n_adapters)
+    cur = [list(s) for s in sets]
+    out = []
+    for _ in range(n_steps):
+        cur = [draw_set(g, n_adapters) if g.random() < p else s for s in cur]
+        out.append(sets_to_csr(cur))
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # the workloads
 # --------------------------------------------------------------------------------------
