@@ -5,7 +5,6 @@
 #include <chrono>
 #include <cstdio>
 #include <cstring>
-#include <map>
 #include <new>
 
 #include "common.cuh"
@@ -187,11 +186,15 @@ struct Router {
     int max_frames = 0, max_set = 0, max_adapters = 0, slabs_max = 0, tokens = 0;
     int slab_cap = 0, max_tiles = 0;
     DevBuf blob;
-    void* stage = nullptr;          // pinned host copy of the blob
+    // pinned host copies of the blob, used in turn: the host may plan a few steps ahead of the GPU
+    // without waiting for an earlier upload to have left its staging buffer
+    static constexpr int N_STAGE = 4;
+    void* stage[N_STAGE] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t uploaded[N_STAGE] = {nullptr, nullptr, nullptr, nullptr};
+    bool upload_pending[N_STAGE] = {false, false, false, false};
+    int stage_next = 0;
     size_t blob_bytes = 0;
     size_t off_perm = 0, off_soff = 0, off_sids = 0, off_src = 0, off_tn = 0, off_ts = 0, off_tsc = 0, off_tm = 0;
-    cudaEvent_t uploaded = nullptr;
-    bool upload_pending = false;
     RouteDev dev;
     std::vector<int32_t> last_off, last_ids;
     std::vector<int> last_fixed;     // frame_of_slot then src_of_slot of the cached plan (branched forward)
@@ -201,13 +204,17 @@ struct Router {
     int device_plan_frames = -1;
     int last_frames = -1;
     bool last_sorted = false;
-    std::vector<int> perm_host;
+    std::vector<int> perm_host, sorted_ids;
+    struct SlabRows { int slab; uint32_t mask[8]; };     // arena slab -> 256-bit mask of the pair's rows using it
+    std::vector<SlabRows> pair_slabs;                    // scratch of build(): the slabs of the pair at hand
     long long plans_built = 0;       // host plans built (cache misses) and the host time they took
     double plan_host_ms = 0.0;
 
     ~Router() {
-        if (stage) cudaFreeHost(stage);
-        if (uploaded) cudaEventDestroy(uploaded);
+        for (int i = 0; i < N_STAGE; ++i) {
+            if (stage[i]) cudaFreeHost(stage[i]);
+            if (uploaded[i]) cudaEventDestroy(uploaded[i]);
+        }
     }
 
     int init(int max_frames_, int max_set_, int max_adapters_, int slabs_max_, int tokens_, std::string& err) {
@@ -227,9 +234,11 @@ struct Router {
         take(off_tm, sizeof(uint32_t) * 4 * std::max(1, max_tiles * slab_cap));
         CK(blob.alloc(blob_bytes));
         CK(cudaMemset(blob.p, 0, blob_bytes));
-        CK(cudaMallocHost(&stage, blob_bytes));
-        memset(stage, 0, blob_bytes);
-        CK(cudaEventCreateWithFlags(&uploaded, cudaEventDisableTiming));
+        for (int i = 0; i < N_STAGE; ++i) {
+            CK(cudaMallocHost(&stage[i], blob_bytes));
+            memset(stage[i], 0, blob_bytes);
+            CK(cudaEventCreateWithFlags(&uploaded[i], cudaEventDisableTiming));
+        }
         uint8_t* b = blob.as<uint8_t>();
         dev.perm = (int*)(b + off_perm); dev.slot_off = (int*)(b + off_soff); dev.slot_ids = (int*)(b + off_sids);
         dev.src_slot = (int*)(b + off_src);
@@ -265,72 +274,97 @@ struct Router {
             (!fixed || (std::equal(frame_of_slot, frame_of_slot + n_frames, last_fixed.begin()) &&
                         std::equal(src_of_slot, src_of_slot + n_frames, last_fixed.begin() + n_frames))))
             return PM_OK;
+        const int si = stage_next;
+        stage_next = (stage_next + 1) % N_STAGE;
+        if (upload_pending[si]) { CK(cudaEventSynchronize(uploaded[si])); upload_pending[si] = false; }
         const auto t_start = std::chrono::steady_clock::now();
-        std::vector<std::vector<int>> sets(n_frames);
+        // per frame: sorted ids, validated
+        sorted_ids.resize(nnz);
         int widest = 0;
         for (int f = 0; f < n_frames; ++f) {
-            sets[f].assign(ids + offsets[f], ids + offsets[f + 1]);
-            std::sort(sets[f].begin(), sets[f].end());
-            for (size_t i = 0; i < sets[f].size(); ++i) {
-                const int a = sets[f][i];
+            int* b = sorted_ids.data() + offsets[f];
+            const int n = offsets[f + 1] - offsets[f];
+            std::copy(ids + offsets[f], ids + offsets[f + 1], b);
+            std::sort(b, b + n);
+            for (int i = 0; i < n; ++i) {
+                const int a = b[i];
                 if (a < 0 || a >= max_adapters) { err = "adapter id out of range"; return PM_ERR_ARG; }
-                if (i > 0 && sets[f][i - 1] == a) { err = "duplicate adapter id in a frame's set"; return PM_ERR_ARG; }
+                if (i > 0 && b[i - 1] == a) { err = "duplicate adapter id in a frame's set"; return PM_ERR_ARG; }
                 if (ranks[a] == 0) { err = "adapter id not registered"; return PM_ERR_STATE; }
             }
-            widest = std::max(widest, (int)sets[f].size());
+            widest = std::max(widest, n);
         }
+        auto set_of = [&](int f) { return std::make_pair(sorted_ids.data() + offsets[f], sorted_ids.data() + offsets[f + 1]); };
         perm_host.resize(n_frames);
         for (int f = 0; f < n_frames; ++f) perm_host[f] = f;
         if (sort_frames)
-            std::stable_sort(perm_host.begin(), perm_host.end(),
-                             [&](int a, int b) { return sets[a] < sets[b]; });
-        if (upload_pending) { CK(cudaEventSynchronize(uploaded)); upload_pending = false; }
-        uint8_t* s = (uint8_t*)stage;
+            std::stable_sort(perm_host.begin(), perm_host.end(), [&](int a, int b) {
+                const auto sa = set_of(a), sb = set_of(b);
+                return std::lexicographical_compare(sa.first, sa.second, sb.first, sb.second);
+            });
+        uint8_t* s = (uint8_t*)stage[si];
         int* h_perm = (int*)(s + off_perm); int* h_soff = (int*)(s + off_soff); int* h_sids = (int*)(s + off_sids);
         int* h_src = (int*)(s + off_src);
         int* h_tn = (int*)(s + off_tn); int* h_ts = (int*)(s + off_ts);
         float* h_tsc = (float*)(s + off_tsc); uint32_t* h_tm = (uint32_t*)(s + off_tm);
         h_soff[0] = 0;
         for (int i = 0; i < n_frames; ++i) {
-            const std::vector<int>& st_ = sets[perm_host[i]];
+            const auto st_ = set_of(perm_host[i]);
             h_perm[i] = fixed ? frame_of_slot[i] : perm_host[i];
             h_src[i] = fixed ? src_of_slot[i] : i;
-            std::copy(st_.begin(), st_.end(), h_sids + h_soff[i]);
-            h_soff[i + 1] = h_soff[i] + (int)st_.size();
+            std::copy(st_.first, st_.second, h_sids + h_soff[i]);
+            h_soff[i + 1] = h_soff[i] + (int)(st_.second - st_.first);
         }
         const long long rows = (long long)n_frames * tokens;
         const int n_pairs = (int)((rows + 2 * PM_TILE_M - 1) / (2 * PM_TILE_M));
         const int n_tiles = 2 * n_pairs;
+        pair_slabs.resize(std::max(slab_cap, 1));
+        SlabRows* ps = pair_slabs.data();
         for (int p = 0; p < n_pairs; ++p) {
             const long long r0 = (long long)p * 2 * PM_TILE_M, r1 = std::min(rows, r0 + 2 * PM_TILE_M);
-            std::map<int, std::array<uint32_t, 8>> slabs;      // arena slab -> 256-bit row mask, ascending
+            int n_ps = 0;                                   // kept in ascending slab order
             for (int slot = (int)(r0 / tokens); slot <= (int)((r1 - 1) / tokens); ++slot) {
-                const long long a0 = std::max(r0, (long long)slot * tokens);
-                const long long a1 = std::min(r1, (long long)(slot + 1) * tokens);
-                for (int a : sets[perm_host[slot]]) {
-                    const int ns = (ranks[a] + PM_SLAB - 1) / PM_SLAB;
+                const int b0 = (int)(std::max(r0, (long long)slot * tokens) - r0);
+                const int b1 = (int)(std::min(r1, (long long)(slot + 1) * tokens) - r0);     // bits [b0, b1)
+                uint32_t m[8];
+                for (int q = 0; q < 8; ++q) {
+                    const int lo = std::max(b0, 32 * q) - 32 * q, hi = std::min(b1, 32 * q + 32) - 32 * q;
+                    m[q] = hi <= lo ? 0u : (hi - lo == 32 ? 0xFFFFFFFFu : ((1u << (hi - lo)) - 1u) << lo);
+                }
+                const auto st_ = set_of(perm_host[slot]);
+                for (const int* ap = st_.first; ap != st_.second; ++ap) {
+                    const int ns = (ranks[*ap] + PM_SLAB - 1) / PM_SLAB;
                     for (int j = 0; j < ns; ++j) {
-                        auto& m = slabs[a * slabs_max + j];
-                        for (long long r = a0; r < a1; ++r) m[(r - r0) >> 5] |= 1u << ((r - r0) & 31);
+                        const int slab = *ap * slabs_max + j;
+                        int at = 0;
+                        while (at < n_ps && ps[at].slab < slab) ++at;
+                        if (at == n_ps || ps[at].slab != slab) {
+                            if (n_ps >= slab_cap) { err = "tile needs more LoRA slabs than the plan capacity"; return PM_ERR_CAPACITY; }
+                            for (int i = n_ps; i > at; --i) ps[i] = ps[i - 1];
+                            ps[at].slab = slab;
+                            for (int q = 0; q < 8; ++q) ps[at].mask[q] = 0u;
+                            ++n_ps;
+                        }
+                        for (int q = 0; q < 8; ++q) ps[at].mask[q] |= m[q];
                     }
                 }
             }
-            if ((int)slabs.size() > slab_cap) { err = "tile needs more LoRA slabs than the plan capacity"; return PM_ERR_CAPACITY; }
             for (int half = 0; half < 2; ++half) {
                 const int t = 2 * p + half;
-                h_tn[t] = (int)slabs.size();
-                int i = 0;
-                for (auto& kv : slabs) {
-                    const size_t at = (size_t)t * slab_cap + i++;
-                    h_ts[at] = kv.first;
-                    h_tsc[at] = scales[kv.first / slabs_max];
-                    for (int q = 0; q < 4; ++q) h_tm[at * 4 + q] = kv.second[half * 4 + q];
+                h_tn[t] = n_ps;
+                for (int i = 0; i < n_ps; ++i) {
+                    const size_t at = (size_t)t * slab_cap + i;
+                    h_ts[at] = ps[i].slab;
+                    h_tsc[at] = scales[ps[i].slab / slabs_max];
+                    for (int q = 0; q < 4; ++q) h_tm[at * 4 + q] = ps[i].mask[half * 4 + q];
                 }
             }
         }
-        CK(cudaMemcpyAsync(blob.p, stage, blob_bytes, cudaMemcpyHostToDevice, st));
-        CK(cudaEventRecord(uploaded, st));
-        upload_pending = true;
+        plan_host_ms += std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_start).count();
+        ++plans_built;
+        CK(cudaMemcpyAsync(blob.p, stage[si], blob_bytes, cudaMemcpyHostToDevice, st));
+        CK(cudaEventRecord(uploaded[si], st));
+        upload_pending[si] = true;
         ++version; device_plan_frames = -1;
         dev.n_frames = n_frames; dev.n_tiles = n_tiles; dev.max_set = widest;
         last_off.assign(offsets, offsets + n_frames + 1);
@@ -341,8 +375,6 @@ struct Router {
             last_fixed.insert(last_fixed.end(), src_of_slot, src_of_slot + n_frames);
         }
         last_frames = n_frames; last_sorted = sort_frames;
-        ++plans_built;
-        plan_host_ms += std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_start).count();
         return PM_OK;
     }
     void invalidate() { last_frames = -1; }

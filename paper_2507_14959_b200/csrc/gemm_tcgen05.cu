@@ -714,18 +714,19 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 // ---------------------------------------------------------------------------------------
 // shrink on the tensor cores: t[tile][s][row][j] = mask(row) * s_a * sum_k x[row,k] A_a[k, 16 s' + j]
 //
-// Persistent: each CTA walks 128-row tiles (tile = blockIdx.x, += gridDim.x) and, inside a tile,
-// groups of up to `sg` LoRA slabs.  For each (tile, group) the x tile streams through shared
-// memory once (TMA, 128B swizzle) next to the group's A^T slabs (16 arena rows per slab, stacked),
-// one UMMA of N = 16 * slabs per 16 K-columns accumulates into one of two TMEM buffers, and the
-// epilogue warps scale, mask, round to bf16 and store each slab as a [128 x 16] block -- the
-// layout the fused GEMM fetches as a 32B-swizzled operand.  The TMA ring and the accumulator
-// buffers carry on across tiles, so loads of the next tile run under the arithmetic of this one.
+// One CTA per 128-row tile, three CTAs per SM, so every tile of a batch is in flight at once and the
+// kernel runs at the speed of its one pass over x (a persistent walk of a few tiles per CTA spent
+// most of a launch ramping up and waiting for the CTAs that drew one tile more).  Inside a tile the
+// LoRA slabs are taken in groups of up to eight: per group the x tile streams through shared memory
+// once (TMA, 128B swizzle) next to the group's A^T slabs (16 arena rows per slab, stacked), one UMMA
+// of N = 16 * slabs per 16 K-columns accumulates in tensor memory, and the epilogue warps scale,
+// mask, round to bf16 and store each slab as a [128 x 16] block -- the layout the fused GEMM fetches
+// as a 32B-swizzled operand.  The ring's stage size follows the tile's own slab count, so a tile with
+// few slabs gets more stages out of the same shared memory.
 // ---------------------------------------------------------------------------------------
 struct ShrinkArgs {
-    int rows, k_in, slab_cap, sg, n_tiles, stages;
-    int reverse;                   // walk the tiles from the last row tile down (see launch_shrink)
-    uint32_t acc_cols;             // TMEM columns of one accumulator buffer (power of two >= 16 * sg)
+    int rows, k_in, slab_cap, n_tiles;
+    int reverse;                   // visit the tiles from the last row tile down (see launch_shrink)
     const int* tile_nslabs;
     const int* tile_slab;
     const float* tile_scale;
@@ -738,7 +739,7 @@ struct ShrinkArgs {
     const float2* ln_stats;     // null = not folded, or the statistics are computed here (stats_out)
     const float* ln_c1;
     const float* ln_c2;
-    // Statistics mode: the epilogue warps also read every x tile as it passes through shared memory
+    // Statistics mode: the epilogue warps also read every x block as it passes through shared memory
     // and produce each row's (mean, 1/sqrt(var + eps)) -- used for t right away and written to
     // stats_out for the GEMM that follows.  Every row tile is then visited, with or without slabs.
     float2* stats_out;
@@ -746,8 +747,11 @@ struct ShrinkArgs {
 };
 
 constexpr int SHRINK_MAX_STAGES = 4;
-constexpr int SHRINK_X_BYTES = BM * BK * 2;          // 16 KB
+constexpr int SHRINK_GROUP = 8;                       // slabs per pass over x: 128 accumulator columns
+constexpr int SHRINK_X_BYTES = BM * BK * 2;           // 16 KB
 constexpr int SHRINK_A_SLAB_BYTES = PM_SLAB * BK * 2; // 2 KB: 16 arena rows x 64 K-columns
+constexpr int SHRINK_RING_BYTES = 72 * 1024;          // 4 stages with one slab, 3 up to four, 2 up to eight
+constexpr int SHRINK_SMEM_BYTES = SHRINK_RING_BYTES + 256;
 
 __global__ void __launch_bounds__(SHRINK_THREADS)
 shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_at,
@@ -758,40 +762,47 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
         return;
     }
-    const int STG = args.stages;
-    const int stage_bytes = SHRINK_X_BYTES + args.sg * SHRINK_A_SLAB_BYTES;
-    const int bar_off = STG * stage_bytes;
-    const uint32_t bars = base + bar_off;
+    const int tile = args.reverse ? args.n_tiles - 1 - (int)blockIdx.x : (int)blockIdx.x;
+    const int ns = args.tile_nslabs[tile];
+    const bool stats = args.stats_out != nullptr;
+    if (ns == 0 && !stats) return;            // nothing to do for this tile (the whole CTA leaves)
+    const int sg = min(ns, SHRINK_GROUP);
+    const int stage_bytes = SHRINK_X_BYTES + sg * SHRINK_A_SLAB_BYTES;
+    const int STG = min(SHRINK_MAX_STAGES, SHRINK_RING_BYTES / stage_bytes);
+    // groups of slabs; in statistics mode a tile without slabs still makes one pass over x
+    const int n_groups = ns == 0 ? 1 : (ns + SHRINK_GROUP - 1) / SHRINK_GROUP;
+    uint32_t acc_cols = 32;                   // power of two >= 16 * sg
+    while ((int)acc_cols < sg * PM_SLAB) acc_cols <<= 1;
+
+    const uint32_t bars = base + SHRINK_RING_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (SHRINK_MAX_STAGES + s); };
-    auto tfull_bar = [&](int a) { return bars + 8u * (2 * SHRINK_MAX_STAGES + a); };
-    auto tempty_bar = [&](int a) { return bars + 8u * (2 * SHRINK_MAX_STAGES + 2 + a); };
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + bar_off + 8 * (2 * SHRINK_MAX_STAGES + 4));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + bar_off + 8 * (2 * SHRINK_MAX_STAGES + 4) + 8);
+    const uint32_t tfull_bar = bars + 8u * (2 * SHRINK_MAX_STAGES);
+    const uint32_t tempty_bar = bars + 8u * (2 * SHRINK_MAX_STAGES + 1);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + SHRINK_RING_BYTES + 8 * (2 * SHRINK_MAX_STAGES + 2));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SHRINK_RING_BYTES + 8 * (2 * SHRINK_MAX_STAGES + 2) + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = args.k_in / BK;
-    const bool stats = args.stats_out != nullptr;
-    // groups of slabs of a tile; in statistics mode a tile without slabs still makes one pass over x
-    auto n_groups = [&](int ns) { return stats && ns == 0 ? 1 : (ns + args.sg - 1) / args.sg; };
 
     if (threadIdx.x == 0) {
         // a stage is free again when its MMAs are done and, in statistics mode, the four epilogue warps
         // have read it too
         for (int s = 0; s < STG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), stats ? 5 : 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        mbar_init(tfull_bar, 1);
+        mbar_init(tempty_bar, 4);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {
-        tmem_alloc(smem_u32((const void*)tmem_slot), 2 * args.acc_cols);
+    if (warp == 1 && ns > 0) {
+        tmem_alloc(smem_u32((const void*)tmem_slot), acc_cols);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = ns > 0 ? *tmem_slot : 0u;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -799,25 +810,21 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
-                const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
-                const int ns = args.tile_nslabs[tile];
-                for (int g = 0; g < n_groups(ns) && ok; ++g) {
-                    const int g0 = g * args.sg;
-                    const int cnt = max(0, min(args.sg, ns - g0));
-                    for (int kb = 0; kb < num_kb && ok; ++kb) {
-                        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
-                        if (!ok) break;
-                        mbar_expect_tx(full_bar(stage), SHRINK_X_BYTES + cnt * SHRINK_A_SLAB_BYTES);
-                        const uint32_t sa = base + stage * stage_bytes;
-                        tma_load_2d(sa, &tm_x, kb * BK, tile * BM, full_bar(stage));
-                        for (int i = 0; i < cnt; ++i) {
-                            const int slab = args.tile_slab[tile * args.slab_cap + g0 + i];
-                            tma_load_2d(sa + SHRINK_X_BYTES + i * SHRINK_A_SLAB_BYTES, &tm_at, kb * BK,
-                                        slab * PM_SLAB, full_bar(stage));
-                        }
-                        if (++stage == STG) { stage = 0; phase ^= 1u; }
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int g0 = g * SHRINK_GROUP;
+                const int cnt = max(0, min(SHRINK_GROUP, ns - g0));
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    mbar_expect_tx(full_bar(stage), SHRINK_X_BYTES + cnt * SHRINK_A_SLAB_BYTES);
+                    const uint32_t sa = base + stage * stage_bytes;
+                    tma_load_2d(sa, &tm_x, kb * BK, tile * BM, full_bar(stage));
+                    for (int i = 0; i < cnt; ++i) {
+                        const int slab = args.tile_slab[tile * args.slab_cap + g0 + i];
+                        tma_load_2d(sa + SHRINK_X_BYTES + i * SHRINK_A_SLAB_BYTES, &tm_at, kb * BK,
+                                    slab * PM_SLAB, full_bar(stage));
                     }
+                    if (++stage == STG) { stage = 0; phase ^= 1u; }
                 }
             }
         }
@@ -825,144 +832,143 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         if (lane == 0) {
             // -------------------------------------------------------------- MMA issuer
             const uint64_t da0 = smem_desc(base, 128), db0 = smem_desc(base + SHRINK_X_BYTES, 128);
-            int stage = 0, acc = 0;
+            int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
-                const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
-                const int ns = args.tile_nslabs[tile];
-                for (int g = 0; g < n_groups(ns) && ok; ++g) {
-                    const int g0 = g * args.sg;
-                    const int cnt = max(0, min(args.sg, ns - g0));
-                    if (cnt == 0) {            // statistics only: hand the stages straight back
-                        for (int kb = 0; kb < num_kb && ok; ++kb) {
-                            ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
-                            if (!ok) break;
-                            mbar_arrive(empty_bar(stage));
-                            if (++stage == STG) { stage = 0; phase ^= 1u; }
-                        }
-                        continue;
-                    }
-                    const uint32_t idesc = instr_desc(cnt * PM_SLAB);
-                    ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, args.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)acc * args.acc_cols;
-                    uint32_t accumulate = 0;
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int g0 = g * SHRINK_GROUP;
+                const int cnt = max(0, min(SHRINK_GROUP, ns - g0));
+                if (cnt == 0) {            // statistics only: hand the stages straight back
                     for (int kb = 0; kb < num_kb && ok; ++kb) {
                         ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
                         if (!ok) break;
-                        tc_fence_after();
-                        const uint64_t so = (uint64_t)((stage * stage_bytes) >> 4);
-#pragma unroll
-                        for (int k = 0; k < BK / 16; ++k) {
-                            umma_bf16(d_tmem, da0 + so + 2 * k, db0 + so + 2 * k, idesc, accumulate);
-                            accumulate = 1;
-                        }
-                        umma_commit(empty_bar(stage));
+                        mbar_arrive(empty_bar(stage));
                         if (++stage == STG) { stage = 0; phase ^= 1u; }
                     }
-                    if (ok) umma_commit(tfull_bar(acc));
-                    if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                    continue;
                 }
+                const uint32_t idesc = instr_desc(cnt * PM_SLAB);
+                // the one accumulator: the epilogue warps have drained the previous group
+                ok = mbar_wait(tempty_bar, acc_phase ^ 1u, abort_flag, args.status);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t accumulate = 0;
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t so = (uint64_t)((stage * stage_bytes) >> 4);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        umma_bf16(tmem_base, da0 + so + 2 * k, db0 + so + 2 * k, idesc, accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit(empty_bar(stage));
+                    if (++stage == STG) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(tfull_bar);
+                acc_phase ^= 1u;
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;
         const int r = quarter * 32 + lane;
-        int acc = 0, stage = 0;
+        int stage = 0;
         uint32_t acc_phase = 0, phase = 0;
         bool ok = true;
-        for (int t_ = blockIdx.x; t_ < args.n_tiles && ok; t_ += gridDim.x) {
-            const int tile = args.reverse ? args.n_tiles - 1 - t_ : t_;
-            const int ns = args.tile_nslabs[tile];
-            float mean = 0.f, inv_rstd = 0.f;
-            for (int g = 0; g < n_groups(ns) && ok; ++g) {
-                const int g0 = g * args.sg;
-                const int cnt = max(0, min(args.sg, ns - g0));
-                if (stats) {
-                    // follow the ring: on the tile's first pass every thread sums its row of each x block
-                    // (shifted by the row's first element, which keeps the sum of squares well conditioned)
-                    float pivot = 0.f, s1 = 0.f, s2 = 0.f;
-                    for (int kb = 0; kb < num_kb && ok; ++kb) {
-                        ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
-                        ok = __all_sync(0xFFFFFFFFu, ok);
-                        if (!ok) break;
-                        if (g == 0) {
-                            const uint32_t row_addr = base + stage * stage_bytes + r * 128;
-#pragma unroll
-                            for (int c = 0; c < 8; ++c) {
-                                uint4 q;
-                                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                             : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w)
-                                             : "r"(row_addr + ((c ^ (r & 7)) << 4)));
-                                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-                                if (kb == 0 && c == 0) pivot = __uint_as_float(w[0] << 16);
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float a0 = __uint_as_float(w[e] << 16) - pivot;
-                                    const float a1 = __uint_as_float(w[e] & 0xFFFF0000u) - pivot;
-                                    s1 += a0 + a1;
-                                    s2 = fmaf(a0, a0, fmaf(a1, a1, s2));
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(empty_bar(stage));
-                        if (++stage == STG) { stage = 0; phase ^= 1u; }
-                    }
+        float mean = 0.f, inv_rstd = 0.f;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            const int g0 = g * SHRINK_GROUP;
+            const int cnt = max(0, min(SHRINK_GROUP, ns - g0));
+            if (stats) {
+                // follow the ring: on the tile's first pass every thread sums its row of each x block,
+                // shifted by the row's first element (which keeps the sum of squares well conditioned);
+                // the arithmetic runs on pairs (packed fp32): the two halves are added at the end
+                float pivot = 0.f;
+                uint64_t npivot2 = 0, s1p = pk2(0.f, 0.f), s2p = pk2(0.f, 0.f);
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = mbar_wait(full_bar(stage), phase, abort_flag, args.status);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     if (g == 0) {
-                        const float inv_d = 1.f / (float)args.k_in;
-                        const float m1 = s1 * inv_d;
-                        const float var = fmaxf(s2 * inv_d - m1 * m1, 0.f);
-                        const float rstd = rsqrtf(var + args.ln_eps);
-                        mean = pivot + m1;
-                        inv_rstd = 1.f / rstd;
-                        if (tile * BM + r < args.rows) args.stats_out[tile * BM + r] = make_float2(mean, rstd);
+                        const uint32_t row_addr = base + stage * stage_bytes + r * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint4 q;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w)
+                                         : "r"(row_addr + ((c ^ (r & 7)) << 4)));
+                            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+                            if (kb == 0 && c == 0) {
+                                pivot = __uint_as_float(w[0] << 16);
+                                npivot2 = pk2(-pivot, -pivot);
+                            }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const uint64_t a = add2(pk2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xFFFF0000u)), npivot2);
+                                s1p = add2(s1p, a);
+                                s2p = fma2(a, a, s2p);
+                            }
+                        }
                     }
-                    if (cnt == 0) continue;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar(stage));
+                    if (++stage == STG) { stage = 0; phase ^= 1u; }
                 }
-                ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, args.status);
-                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
-                tc_fence_after();
-                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * args.acc_cols;
-                if (args.ln_stats && tile * BM + r < args.rows) {
-                    const float2 st = args.ln_stats[tile * BM + r];
-                    mean = st.x;
-                    inv_rstd = 1.f / st.y;
+                if (g == 0) {
+                    float s1a, s1b, s2a, s2b;
+                    upk2(s1p, s1a, s1b);
+                    upk2(s2p, s2a, s2b);
+                    const float inv_d = 1.f / (float)args.k_in;
+                    const float m1 = (s1a + s1b) * inv_d;
+                    const float var = fmaxf((s2a + s2b) * inv_d - m1 * m1, 0.f);
+                    const float rstd = rsqrtf(var + args.ln_eps);
+                    mean = pivot + m1;
+                    inv_rstd = 1.f / rstd;
+                    if (tile * BM + r < args.rows) args.stats_out[tile * BM + r] = make_float2(mean, rstd);
                 }
-                for (int i = 0; i < cnt; ++i) {
-                    const int slot = tile * args.slab_cap + g0 + i;
-                    uint32_t v[16];
-                    tmem_ld16(t_row + (uint32_t)(i * PM_SLAB), v);
-                    tmem_ld_wait();
-                    const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
-                    const float sc = on ? args.tile_scale[slot] : 0.f;
-                    if (args.ln_stats || stats) {
-                        const float* c1 = args.ln_c1 + (size_t)args.tile_slab[slot] * PM_SLAB;
-                        const float* c2 = args.ln_c2 + (size_t)args.tile_slab[slot] * PM_SLAB;
-#pragma unroll
-                        for (int j = 0; j < PM_SLAB; ++j)
-                            v[j] = __float_as_uint(fmaf(-mean, __ldg(c1 + j), __uint_as_float(v[j])) +
-                                                   inv_rstd * __ldg(c2 + j));
-                    }
-                    uint4 o[2];
-                    uint32_t* ow = reinterpret_cast<uint32_t*>(o);
-#pragma unroll
-                    for (int j = 0; j < PM_SLAB; j += 2)
-                        ow[j >> 1] = pack_bf16(__uint_as_float(v[j]) * sc, __uint_as_float(v[j + 1]) * sc);
-                    uint4* dst = reinterpret_cast<uint4*>(args.tbuf + ((size_t)slot * BM + r) * PM_SLAB);
-                    dst[0] = o[0];
-                    dst[1] = o[1];
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(acc));
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                if (cnt == 0) continue;
             }
+            ok = mbar_wait(tfull_bar, acc_phase, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            if (args.ln_stats && tile * BM + r < args.rows) {
+                const float2 st = args.ln_stats[tile * BM + r];
+                mean = st.x;
+                inv_rstd = 1.f / st.y;
+            }
+            for (int i = 0; i < cnt; ++i) {
+                const int slot = tile * args.slab_cap + g0 + i;
+                uint32_t v[16];
+                tmem_ld16(t_row + (uint32_t)(i * PM_SLAB), v);
+                tmem_ld_wait();
+                const bool on = (args.tile_mask[(size_t)slot * 4 + quarter] >> lane) & 1u;
+                const float sc = on ? args.tile_scale[slot] : 0.f;
+                if (args.ln_stats || stats) {
+                    const float* c1 = args.ln_c1 + (size_t)args.tile_slab[slot] * PM_SLAB;
+                    const float* c2 = args.ln_c2 + (size_t)args.tile_slab[slot] * PM_SLAB;
+#pragma unroll
+                    for (int j = 0; j < PM_SLAB; ++j)
+                        v[j] = __float_as_uint(fmaf(-mean, __ldg(c1 + j), __uint_as_float(v[j])) +
+                                               inv_rstd * __ldg(c2 + j));
+                }
+                uint4 o[2];
+                uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+                for (int j = 0; j < PM_SLAB; j += 2)
+                    ow[j >> 1] = pack_bf16(__uint_as_float(v[j]) * sc, __uint_as_float(v[j + 1]) * sc);
+                uint4* dst = reinterpret_cast<uint4*>(args.tbuf + ((size_t)slot * BM + r) * PM_SLAB);
+                dst[0] = o[0];
+                dst[1] = o[1];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar);
+            acc_phase ^= 1u;
         }
     }
     __syncwarp();
@@ -971,9 +977,9 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 1 && ns > 0) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 2 * args.acc_cols);
+        tmem_dealloc(tmem_base, acc_cols);
     }
 }
 
@@ -1089,20 +1095,12 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 }
 
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int n_sms,
+                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int /*n_sms*/,
                           const float2* ln_stats, float2* stats_out, float ln_eps) {
     if (R.n_tiles <= 0) return cudaSuccess;
     if (R.slab_cap <= 0) return stats_out ? cudaErrorInvalidValue : cudaSuccess;   // nothing to shrink
     ShrinkArgs a;
     a.rows = rows; a.k_in = lin.k_in; a.slab_cap = R.slab_cap; a.n_tiles = R.n_tiles;
-    // groups of at most 8 slabs: two 128-column accumulators per CTA, so two CTAs share an SM's TMEM
-    a.sg = R.slab_cap < 8 ? R.slab_cap : 8;
-    uint32_t cols = 32;
-    while ((int)cols < a.sg * PM_SLAB) cols <<= 1;
-    a.acc_cols = cols;                                   // two buffers: at most 2 x 256 columns
-    const int stage_bytes = SHRINK_X_BYTES + a.sg * SHRINK_A_SLAB_BYTES;
-    // four stages while two CTAs still fit an SM (and their 2 x 2 accumulators fit its TMEM)
-    a.stages = (4 * stage_bytes + 256 <= 112 * 1024) ? 4 : 3;
     a.tile_nslabs = R.tile_nslabs; a.tile_slab = R.tile_slab; a.tile_scale = R.tile_scale;
     a.tile_mask = R.tile_mask; a.tbuf = tbuf; a.status = L.status;
     // a linear with LayerNorm folded in gets the row statistics either ready-made or computed here
@@ -1113,13 +1111,10 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     // is what the cache still holds: start there, and leave the front in the cache for the GEMM that
     // follows (which walks front to back)
     a.reverse = (size_t)rows * lin.k_in * sizeof(bf16) > ((size_t)96 << 20) ? 1 : 0;
-    const int smem = a.stages * stage_bytes + 256;
     static SmemGrant grant;
-    if (cudaError_t e = grant.ensure(shrink_tc_kernel, smem); e != cudaSuccess) return e;
-    const int per_sm = (2 * smem + 4096 <= 227 * 1024 && 4 * cols <= 512) ? 2 : 1;
-    const int grid = R.n_tiles < n_sms * per_sm ? R.n_tiles : n_sms * per_sm;
+    if (cudaError_t e = grant.ensure(shrink_tc_kernel, SHRINK_SMEM_BYTES); e != cudaSuccess) return e;
     ProfScope ps(L, KC_SHRINK);
-    shrink_tc_kernel<<<grid, SHRINK_THREADS, smem, L.st>>>(*tm_x, lin.tm_at, a);
+    shrink_tc_kernel<<<a.n_tiles, SHRINK_THREADS, SHRINK_SMEM_BYTES, L.st>>>(*tm_x, lin.tm_at, a);
     BUMP(L);
     return cudaGetLastError();
 }

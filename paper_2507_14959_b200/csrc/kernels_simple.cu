@@ -469,16 +469,24 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ z, const T* _
 
 __device__ __forceinline__ float sigmoidf_acc(float v) { return 1.f / (1.f + expf(-v)); }
 
-// grid (ceil(K/8), ceil(F/8)): a warp keeps the weight row of one class in registers and walks 8
-// slots (a longer walk is a longer chain of load latencies); base_out rows are in the caller's order.
-// NV = ceil(d / 32) values per lane.  All loads of a z row are issued before the first multiply-add
-// (the walk is bound by the latency of those loads), and the dot product runs in four chains.
+// grid (ceil(K/8), ceil(F/8)): a block owns 8 classes x 8 slots.  The 8 CLS features are staged once in
+// shared memory and shared by the block's 8 warps (read straight from global memory, every class of a
+// block would fetch them again: F x K x d x 4 bytes of cache traffic in all); each warp keeps the
+// weight row of its class in registers and walks the slots.  base_out rows are in the caller's order.
+// NV = ceil(d / 32) values per lane; the dot product runs in four chains.
 constexpr int BASE_HEAD_FRAMES = 8;
 template <typename T, int NV>
 __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict__ z, const T* __restrict__ wt,
                                                         const float* __restrict__ bias,
                                                         const int* __restrict__ perm, int d, int n_classes,
                                                         int n_frames, float* __restrict__ base_out) {
+    __shared__ float zs[BASE_HEAD_FRAMES][NV * 32];
+    const int s0 = blockIdx.y * BASE_HEAD_FRAMES, ns = min(n_frames - s0, BASE_HEAD_FRAMES);
+    for (int i = threadIdx.x; i < BASE_HEAD_FRAMES * NV * 32; i += 256) {
+        const int sl = i / (NV * 32), c = i % (NV * 32);
+        zs[sl][c] = (sl < ns && c < d) ? z[(size_t)(s0 + sl) * d + c] : 0.f;
+    }
+    __syncthreads();
     const int k = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (k >= n_classes) return;
@@ -489,20 +497,12 @@ __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict_
         w[i] = c < d ? to_f(wt[(size_t)k * d + c]) : 0.f;
     }
     const float bk = bias[k];
-    const int s0 = blockIdx.y * BASE_HEAD_FRAMES, s1 = min(n_frames, s0 + BASE_HEAD_FRAMES);
-    for (int slot = s0; slot < s1; ++slot) {
-        const float* zr = z + (size_t)slot * d;
-        float zv[NV];
-#pragma unroll
-        for (int i = 0; i < NV; ++i) {
-            const int c = lane + 32 * i;
-            zv[i] = c < d ? __ldg(zr + c) : 0.f;
-        }
+    for (int sl = 0; sl < ns; ++sl) {
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < NV; ++i) acc[i & 3] = fmaf(zv[i], w[i], acc[i & 3]);
+        for (int i = 0; i < NV; ++i) acc[i & 3] = fmaf(zs[sl][lane + 32 * i], w[i], acc[i & 3]);
         const float dot = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
-        if (lane == 0) base_out[(size_t)perm[slot] * n_classes + k] = sigmoidf_acc(dot + bk);
+        if (lane == 0) base_out[(size_t)perm[s0 + sl] * n_classes + k] = sigmoidf_acc(dot + bk);
     }
 }
 
@@ -705,19 +705,17 @@ __global__ void __launch_bounds__(SELECT_THREADS) select_kernel(const float* __r
         voff[g + 1] = run;
     }
     __syncthreads();
-    for (int g = warp; g < n_frames; g += nwarps) {
+    // emission: one thread per frame (all frames' loads are in flight at once; a frame has few ids)
+    for (int g = threadIdx.x; g < n_frames; g += SELECT_THREADS) {
         int pos = voff[g];
         for (int q = 0; q < AW; ++q) {
-            const uint64_t m = vmasks[(size_t)g * AW + q];
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const uint32_t bits = (uint32_t)(m >> (32 * half));
-                if ((bits >> lane) & 1u) {
-                    const int at = pos + __popc(bits & ((1u << lane) - 1u));
-                    if (at < ids_capacity) next_ids[at] = q * 64 + half * 32 + lane;
-                    else atomicCAS(status, 0, (int)PM_ERR_CAPACITY);
-                }
-                pos += __popc(bits);
+            uint64_t m = vmasks[(size_t)g * AW + q];
+            while (m) {
+                const int b = __ffsll((long long)m) - 1;
+                m &= m - 1;
+                if (pos < ids_capacity) next_ids[pos] = q * 64 + b;
+                else atomicCAS(status, 0, (int)PM_ERR_CAPACITY);
+                ++pos;
             }
         }
     }
