@@ -311,6 +311,17 @@ def run_streams(args, rank, world, dist, local_rank):
         stage.copy_(frames_dev[0])
         r.step(stage)
         r.capture(stage)
+    clip = clip_scores = None
+    if mode == "sequence":
+        # one eager clip, then all T steps of a clip are one recorded sequence reading a static clip buffer
+        args.steps = (args.steps + T - 1) // T * T
+        clip = frames_dev.clone()
+        clip_scores = torch.zeros((T, S, K), device="cuda")
+        clip_scores_host = torch.zeros((T, S, K)).pin_memory()
+        r.reset()
+        for t in range(T):
+            r.step(clip[t])
+        r.capture_sequence(clip, log_scores=clip_scores)
 
     def barrier():
         torch.cuda.synchronize()
@@ -319,6 +330,14 @@ def run_streams(args, rank, world, dist, local_rank):
         torch.cuda.synchronize()
 
     def loop(n, e2e, replay=True):
+        if mode == "sequence" and replay:
+            for _ in range(n // T):
+                if e2e:
+                    clip.copy_(frames_host, non_blocking=True)
+                r.run_sequence()
+                if e2e:
+                    clip_scores_host.copy_(clip_scores, non_blocking=True)
+            return
         for i in range(n):
             t = i % T
             if t == 0:
@@ -334,7 +353,7 @@ def run_streams(args, rank, world, dist, local_rank):
             if e2e:
                 scores_host.copy_(sc, non_blocking=True)
 
-    loop(max(args.warmup, 3), False)
+    loop(max(args.warmup, 3) if mode != "sequence" else T, False)
     assert m.status() == 0
     sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else 0)
     if rank == 0:
@@ -344,9 +363,9 @@ def run_streams(args, rank, world, dist, local_rank):
     walls = []
     for e2e in (False, True):
         if e2e:
-            loop(2, True)
+            loop(2 if mode != "sequence" else T, True)
         barrier()
-        count = lambda: m.launch_count() + (r.replayed_launches if mode == "graph" else 0)
+        count = lambda: m.launch_count() + (r.replayed_launches if mode in ("graph", "sequence") else 0)
         n0 = count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         walls.append(time.time())
@@ -405,7 +424,9 @@ def run_streams(args, rank, world, dist, local_rank):
                        "streams_per_gpu": S,
                        "loop": {"host": "routing plan on the host (a device-to-host copy and a stream synchronisation per step)",
                                 "device": "routing plan built on the device, no host synchronisation",
-                                "graph": "routing plan built on the device; steps after a stream's first are CUDA-graph replays"}[mode],
+                                "graph": "routing plan built on the device; steps after a stream's first are CUDA-graph replays",
+                                "sequence": "routing plan built on the device; a clip of 30 steps is one recorded sequence "
+                                            "(one CUDA-graph launch per clip)"}[mode],
                        "l2": "one step's activations fit the 126 MB L2; no flush" if args.workload == "latency"
                              else "one step touches ~0.2 GB of activations; no flush"},
             "latency_us_per_step": 1e3 * ms / args.steps,
@@ -454,9 +475,10 @@ def main():
                     help="batch: ViT-base 224x224, 256 frames (the headline); streams: ViT-base 384x384, 16 streams "
                          "in closed loop (forward -> Algorithm 2 -> next forward), one step = one frame per stream; "
                          "latency: DeiT-tiny, one stream in closed loop (the paper's embedded operating point)")
-    ap.add_argument("--loop", default="graph", choices=["host", "device", "graph"],
+    ap.add_argument("--loop", default="graph", choices=["host", "device", "graph", "sequence"],
                     help="streams / latency: where the routing plan of a step is built and whether steps are "
-                         "CUDA-graph replays")
+                         "CUDA-graph replays (graph: one replay per step; sequence: the whole 30-step clip is one "
+                         "recorded sequence, one graph launch per clip -- --steps is then rounded up to whole clips)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "polymorph" else args.warmup
 

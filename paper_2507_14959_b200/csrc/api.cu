@@ -647,7 +647,7 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, int n_slots, int
                                    : (void*)y == h->H.p ? &h->tm_y_h
                                    : (void*)y == h->X.p ? &h->tm_y_x : nullptr;
             return launch_lora_gemm(L, lo.dev, use_lora ? &R : nullptr, *tmx, &h->tm_t, tmy, nrows, epi,
-                                    (const bf16*)residual, pep, (bf16*)y, h->n_sms, st);
+                                    (const bf16*)residual, pep, (bf16*)y, h->n_sms, st, use_lora);
         } else {
             return launch_naive_linear<T>(L, lo.dev, R, h->meta, h->slabs_max, x, nrows, tokens_pf,
                                           lora ? h->t32.as<float>() : nullptr, epi, residual, pep, y);
@@ -1195,7 +1195,7 @@ int pm_linear_forward(pm_linear l, const void* x, int n_frames, const int32_t* s
         const bool lora = R.max_set > 0 && l->lin.dev.lora.At != nullptr;
         if (lora) CK(launch_shrink(L, l->lin.dev, R, &tm_x, (const bf16*)x, rows, l->tbuf.as<bf16>(), l->n_sms, nullptr, nullptr, 0.f));
         CK(launch_lora_gemm(L, l->lin.dev, lora ? &R : nullptr, tm_x, &l->tm_t, &tm_y, rows, l->epilogue,
-                            (const bf16*)residual, none, (bf16*)y, l->n_sms, nullptr));
+                            (const bf16*)residual, none, (bf16*)y, l->n_sms, nullptr, lora));
     } else {
         CK(launch_naive_linear<float>(L, l->lin.dev, R, l->meta, l->slabs_max, (const float*)x, rows, l->tokens,
                                       l->t32.as<float>(), l->epilogue, (const float*)residual, none, (float*)y));

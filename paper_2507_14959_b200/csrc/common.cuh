@@ -153,12 +153,14 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
                           const CUtensorMap* tm_x, const bf16* x, int rows, bf16* tbuf, int n_sms,
                           const float2* ln_stats, float2* stats_out, float ln_eps);
 cudaError_t launch_row_stats(const Launch& L, const bf16* x, float2* stats, int rows, int d, float eps);
+// after_shrink: the kernel enqueued just before on the stream is this linear's launch_shrink; the GEMM
+// may then start before it has finished (programmatic dependent launch) and awaits its results itself.
 // tm_y: [rows, n_out] output map with a (32 x 32) box and 64B swizzle for the TMA-store epilogue, or
 // null to store straight from registers (always the case for EPI_PATCH, whose rows are remapped)
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
                              const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
                              int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
-                             int n_sms, const float2* ln_stats);
+                             int n_sms, const float2* ln_stats, bool after_shrink = false);
 // x rows of slots [first_slot, n_slots) <- x rows of slot src_slot[slot] (a slot below first_slot)
 template <typename T>
 cudaError_t launch_fanout_rows(const Launch& L, T* x, const int* src_slot, int first_slot, int n_slots,

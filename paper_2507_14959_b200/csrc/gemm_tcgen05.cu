@@ -94,6 +94,8 @@ struct GemmArgs {
     const int* tile_slab;
     int slab_cap;
     int tma_store;             // 1: the epilogue stores through shared memory + TMA (tm_y valid)
+    int overlap_prev;          // host side only: launch with programmatic serialization (the kernel before it on
+                               // the stream is this linear's shrink, whose results are awaited with dep_wait())
     int* status;
     // LayerNorm folded into the linear (LNF kernels): y = rstd (acc - mean g) + bias, per row / column
     const float* ln_g;
@@ -353,7 +355,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            bool ok = true;
+            bool ok = true, dep_done = false;
             int it = 0;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
                 const int m = tile / args.n_tiles, n = tile % args.n_tiles;
@@ -367,6 +369,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 const int ns = tile_ns(it, m);
+                if (ns > 0 && !dep_done) { dep_wait(); dep_done = true; }     // t comes from the shrink kernel
                 for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
                     const int cnt = min(SLABS_PER_STAGE, ns - g0);
                     ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
@@ -443,6 +446,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
         const int half = (warp - 2) >> 2;             // which share of the tile's 32-column chunks
         const uint32_t staging = base + S::STAGING_OFFSET + (uint32_t)(warp - 2) * STAGING_BYTES_PER_WARP;
+        dep_wait();                                   // the row statistics come from the shrink kernel
         int acc = 0;
         uint32_t acc_phase = 0;
         uint32_t chunk_no = 0;                        // running chunk counter: picks the staging buffer
@@ -460,6 +464,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 
     // ---------------------------------------------------------------------- teardown
     __syncwarp();
+    dep_wait();               // never finish before the kernel this one was allowed to overtake
     if (*abort_flag) {
         // give copies and MMAs still in flight time to land before shared memory / TMEM go away
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
@@ -590,7 +595,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            bool ok = true;
+            bool ok = true, dep_done = false;
             int it = 0;
             for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++it) {
                 const int m2 = tile / args.n_tiles, n = tile % args.n_tiles;
@@ -606,6 +611,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
                 }
                 const int ns = tile_ns(it, m);
+                if (ns > 0 && !dep_done) { dep_wait(); dep_done = true; }     // t comes from the shrink kernel
                 for (int g0 = 0; g0 < ns && ok; g0 += SLABS_PER_STAGE) {
                     const int cnt = min(SLABS_PER_STAGE, ns - g0);
                     ok = mbar_wait_cluster(empty_bar(stage), phase ^ 1u, abort_flag, args.status);
@@ -680,6 +686,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
         const uint32_t staging = base + P_STAGING_OFFSET + (uint32_t)(warp - 2) * STAGING_BYTES_PER_WARP;
+        dep_wait();                                   // the row statistics come from the shrink kernel
         int acc = 0;
         uint32_t acc_phase = 0, res_phase = 0;
         uint32_t chunk_no = 0;
@@ -700,6 +707,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 
     // ---------------------------------------------------------------------- teardown
     __syncwarp();
+    dep_wait();               // never finish before the kernel this one was allowed to overtake
     if (*abort_flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);    // let copies / MMAs in flight land
     }
@@ -765,7 +773,8 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     const int tile = args.reverse ? args.n_tiles - 1 - (int)blockIdx.x : (int)blockIdx.x;
     const int ns = args.tile_nslabs[tile];
     const bool stats = args.stats_out != nullptr;
-    if (ns == 0 && !stats) return;            // nothing to do for this tile (the whole CTA leaves)
+    if (ns == 0 && !stats) return;            // nothing to do for this tile (the whole CTA leaves; an exited CTA
+                                              // counts as having released the kernel's dependents)
     const int sg = min(ns, SHRINK_GROUP);
     const int stage_bytes = SHRINK_X_BYTES + sg * SHRINK_A_SLAB_BYTES;
     const int STG = min(SHRINK_MAX_STAGES, SHRINK_RING_BYTES / stage_bytes);
@@ -803,6 +812,9 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ns > 0 ? *tmem_slot : 0u;
+    // The fused GEMM that follows needs t (and the row statistics) only when its first tile's base K loop
+    // is over: it may start on every SM this kernel's CTAs have left, while the slowest tiles finish.
+    dep_release();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -1133,10 +1145,20 @@ static cudaError_t launch_gemm_bn(const Launch& L, const CUtensorMap& tm_x, cons
     if (cudaError_t e = grant.ensure(lora_gemm_kernel<BN, EPI, EW, LNF>, Smem<BN, EW>::TOTAL); e != cudaSuccess) return e;
     const int total = a.m_tiles * a.n_tiles;
     const int grid = total < n_sms ? total : n_sms;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(64 + 32 * EW);
+    cfg.dynamicSmemBytes = Smem<BN, EW>::TOTAL;
+    cfg.stream = L.st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.overlap_prev ? 1 : 0;
     ProfScope ps(L, KC_GEMM);
-    lora_gemm_kernel<BN, EPI, EW, LNF><<<grid, 64 + 32 * EW, Smem<BN, EW>::TOTAL, L.st>>>(tm_x, tm_w, tm_t, tm_bt, tm_y, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_kernel<BN, EPI, EW, LNF>, tm_x, tm_w, tm_t, tm_bt, tm_y, a);
     BUMP(L);
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int BN>
@@ -1175,11 +1197,13 @@ static cudaError_t launch_gemm_pair(const Launch& L, const CUtensorMap& tm_x, co
     cfg.blockDim = dim3(P_THREADS);
     cfg.dynamicSmemBytes = P_SMEM_TOTAL;
     cfg.stream = L.st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = a.overlap_prev ? 2 : 1;
     ProfScope ps(L, KC_GEMM);
     cudaError_t e = cudaLaunchKernelEx(&cfg, lora_gemm_pair_kernel<EPI, LNF, RESS>, tm_x, tm_w, tm_t, tm_bt, tm_y, tm_res, a);
     BUMP(L);
@@ -1211,7 +1235,7 @@ int gemm_tile_n(int n_out) { return (n_out % 256 == 0) ? 256 : 128; }
 cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteDev* R,
                              const CUtensorMap& tm_x, const CUtensorMap* tm_t, const CUtensorMap* tm_y,
                              int rows, int epi, const bf16* residual, const PatchEpi& pe, bf16* y,
-                             int n_sms, const float2* ln_stats) {
+                             int n_sms, const float2* ln_stats, bool after_shrink) {
     if (rows <= 0) return cudaSuccess;
     if ((lin.ln_g != nullptr) != (ln_stats != nullptr)) return cudaErrorInvalidValue;
     const int bn = gemm_tile_n(lin.n_out);
@@ -1225,6 +1249,7 @@ cudaError_t launch_lora_gemm(const Launch& L, const LinearDev& lin, const RouteD
     a.tile_slab = lora ? R->tile_slab : nullptr;
     a.slab_cap = lora ? R->slab_cap : 0;
     a.status = L.status;
+    a.overlap_prev = (after_shrink && lora) ? 1 : 0;
     a.ln_g = lin.ln_g; a.ln_stats = ln_stats;
     a.tma_store = (tm_y != nullptr && epi != EPI_PATCH) ? 1 : 0;
     const CUtensorMap& tt = lora ? *tm_t : tm_x;      // placeholders are never dereferenced

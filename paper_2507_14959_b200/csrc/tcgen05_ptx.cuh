@@ -179,6 +179,13 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
 
 
 
+// ---- programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while the kernel before it on the stream is still running, once every CTA of that kernel has
+// released its dependents (or exited); what the earlier kernel writes may only be touched after dep_wait().
+// Without the attribute both are no-ops.
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- CTA pairs (thread-block clusters of two): the helpers of the two-SM tensor-core kernels ----
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;

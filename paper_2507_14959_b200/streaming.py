@@ -88,6 +88,39 @@ class StreamRunner:
         self.t += 1
         return self.scores, self.base
 
+    def capture_sequence(self, frames_seq, log_base=None, log_scores=None):
+        """Records the closed loop over a whole clip -- frames_seq: device tensor [T, n_streams, 3, img,
+        img], kept and re-read on every replay -- as ONE CUDA graph: empty sets for the first frame, then
+        T times forward -> select, each step reading the lists the step before wrote.  log_base /
+        log_scores ([T, n_streams, n_classes] device tensors, optional) receive every step's scores
+        inside the graph.  Needs device_plan and one eager pass over a clip before it.  Replay with
+        run_sequence(); to process another clip, copy its frames into frames_seq first."""
+        import torch
+        if not self.device_plan:
+            raise ValueError("capture_sequence needs device_plan (the host planner synchronises the stream)")
+        T = int(frames_seq.shape[0])
+        g = torch.cuda.CUDAGraph()
+        n0 = self.model.launch_count()
+        with torch.cuda.graph(g):
+            for off, _ in self.csr:
+                off.zero_()
+            for t in range(T):
+                self._enqueue(frames_seq[t], t % 2, t > 0)
+                if log_base is not None:
+                    log_base[t].copy_(self.base)
+                if log_scores is not None:
+                    log_scores[t].copy_(self.scores)
+        self.seq_graph, self.seq_steps = g, T
+        self.seq_launches = self.model.launch_count() - n0
+        self.replayed_launches = getattr(self, "replayed_launches", 0)
+
+    def run_sequence(self):
+        """Replays the recorded clip (capture_sequence): one graph launch for all its steps."""
+        self.seq_graph.replay()
+        self.replayed_launches += self.seq_launches
+        self.t = self.seq_steps
+        return self.scores, self.base
+
     def current_sets(self):
         """The sets the next step will use, as host lists (synchronises)."""
         off, ids = self.csr[self.t % 2]

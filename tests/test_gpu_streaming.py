@@ -108,6 +108,22 @@ def test_device_plan_and_graph_replay_match_host_plan():
         assert np.abs(outs[1]["base"][t, st] - bo[0]).max() < 1e-2
     for o in outs:
         check_device_metrics(o, S)
+    # the whole clip as ONE recorded sequence (T steps in a single graph launch): same bits, same counters
+    r = outs[1]["runner"]
+    clip = fd.transpose(0, 1).contiguous()                          # [T, S, 3, img, img]
+    log_b = torch.zeros((T, S, spec.n_classes), device="cuda")
+    log_s = torch.zeros_like(log_b)
+    r.capture_sequence(clip, log_b, log_s)
+    for _ in range(2):                                              # a replay leaves no state behind
+        log_b.fill_(-1.0)
+        m.metrics_reset()
+        r.run_sequence()
+        n, contexts, switches = m.metrics_read()
+        np.testing.assert_array_equal(log_b.cpu().numpy(), outs[1]["base"])
+        np.testing.assert_array_equal(log_s.cpu().numpy(), outs[1]["scores"])
+        assert r.current_sets() == outs[1]["chosen_sets"][-1]
+        assert n == S * T and contexts / n == pytest.approx(outs[1]["avg_coverage"])
+        assert switches == outs[1]["switch_penalty"]
     assert m.status() == 0
     m.close()
 
