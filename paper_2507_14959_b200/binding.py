@@ -21,7 +21,7 @@ ERROR_NAMES = {0: "PM_OK", -1: "PM_ERR_ARG", -2: "PM_ERR_STATE", -3: "PM_ERR_CAP
 
 EXPORTS = [
     "pm_create", "pm_register_adapter", "pm_set_cover", "pm_destroy", "pm_forward", "pm_forward_branched", "pm_forward_device_sets", "pm_select",
-    "pm_select_static", "pm_metrics_reset", "pm_metrics_read", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_profile_enable", "pm_profile_read", "pm_plan_stats", "pm_linear_create", "pm_linear_register",
+    "pm_select_static", "pm_metrics_reset", "pm_metrics_read", "pm_status", "pm_last_error", "pm_launch_count", "pm_set_graphs", "pm_set_small_batch_kernel", "pm_profile_enable", "pm_profile_read", "pm_plan_stats", "pm_linear_create", "pm_linear_register",
     "pm_linear_forward", "pm_linear_status", "pm_linear_last_error", "pm_linear_destroy",
     "pm_layernorm", "pm_attention", "pm_selftest_wait_timeout", "pm_cooccurrence", "pm_build_contexts", "pm_intra_coherence",
 ]
@@ -89,6 +89,7 @@ def load():
     lib.pm_build_contexts.argtypes = [_FP, ip, ip, ip, ip, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int)]
     lib.pm_intra_coherence.argtypes = [_FP, ip, C.POINTER(C.c_int32), C.POINTER(C.c_int32), ip, C.POINTER(C.c_double)]
     lib.pm_set_graphs.argtypes = [vp, ip]
+    lib.pm_set_small_batch_kernel.argtypes = [vp, ip]
     lib.pm_launch_count.restype = C.c_longlong
     lib.pm_profile_enable.argtypes = [vp, ip]
     lib.pm_profile_read.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
@@ -225,6 +226,10 @@ class Model:
     def set_graphs(self, on):
         """Switches the recording / replaying of the forward's launch sequence as CUDA graphs."""
         self._check(self.lib.pm_set_graphs(self.handle, int(on)), "pm_set_graphs")
+
+    def set_small_batch_kernel(self, on):
+        """Whether small batches of small models run as the one whole-network kernel (default on)."""
+        self._check(self.lib.pm_set_small_batch_kernel(self.handle, int(on)), "pm_set_small_batch_kernel")
 
     KERNEL_CLASSES = ("gemm", "shrink", "attention", "layernorm", "other", "heads", "select", "plan")
 

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpolymorph.so")
-SOURCES = ["api.cu", "kernels_simple.cu", "gemm_tcgen05.cu", "attention.cu", "plan_device.cu", "contexts.cu"]
+SOURCES = ["api.cu", "kernels_simple.cu", "gemm_tcgen05.cu", "attention.cu", "plan_device.cu", "contexts.cu", "latency_kernel.cu"]
 
 
 def nvcc_path() -> str:

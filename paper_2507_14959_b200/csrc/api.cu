@@ -464,6 +464,9 @@ struct pm_handle_s {
     long long launches = 0;
     Profiler prof;
     std::string err;
+    // whole-network kernel for a handful of frames (latency_kernel.cu)
+    DevBuf lat_lin, lat_kv, lat_bar;
+    bool lat_dirty = true, lat_on = true;
     // recorded launch sequences of the forward entry points (see run_graphed)
     struct GraphEntry {
         const void* key_ptr[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -699,6 +702,63 @@ int forward_t(pm_handle_s* h, const void* frames, int n_frames, int n_slots, int
     return PM_OK;
 }
 
+// ---- the whole-network kernel: small batches of small models in one launch --------------------------
+constexpr int LAT_ROWS = 16;
+int lat_tiles_per_frame(const pm_handle_s* h) { return (h->tokens + LAT_ROWS - 1) / LAT_ROWS; }
+
+bool latency_eligible(const pm_handle_s* h, int n_frames) {
+    const pm_config& c = h->cfg;
+    if (!h->lat_on || c.dtype != 0 || c.d > 384 || c.mlp > 1536 || h->patch_dim > 1536 || c.max_set > 8) return false;
+    if (h->slabs_max * PM_SLAB * c.max_set > 512) return false;
+    if ((long long)n_frames * lat_tiles_per_frame(h) > h->n_sms) return false;       // one CTA per SM, all resident
+    return latency_smem_bytes(c.d, c.mlp, h->patch_dim, h->slabs_max * PM_SLAB * c.max_set, h->tokens) <= 227 * 1024;
+}
+
+// slots: perm (slot -> frame) or null; set lists: device CSR over slots
+int forward_latency(pm_handle_s* h, const void* frames, int n_frames, const int* perm, const int* d_off, const int* d_ids,
+                    float* scores_out, float* base_out, cudaStream_t st) {
+    std::string& err = h->err;
+    const pm_config& c = h->cfg;
+    auto view = [](const LinearObj& lo) {
+        LatLinear v;
+        v.Wt = (const bf16*)lo.dev.Wt; v.bias = lo.dev.bias; v.ln_g = lo.dev.ln_g;
+        v.At = (const bf16*)lo.dev.lora.At; v.Bt = (const bf16*)lo.dev.lora.Bt; v.c1 = lo.dev.ln_c1; v.c2 = lo.dev.ln_c2;
+        for (int i = 0; i < 8; ++i) v.adapted[i] = 0u;
+        for (size_t a = 0; a < lo.adapted.size() && a < 256; ++a) if (lo.adapted[a]) v.adapted[a >> 5] |= 1u << (a & 31);
+        if (lo.n_adapted == 0) { v.At = nullptr; v.Bt = nullptr; }
+        v.k_in = lo.dev.k_in; v.n_out = lo.dev.n_out;
+        return v;
+    };
+    if (h->lat_dirty) {
+        std::vector<LatLinear> lv;
+        for (const LinearObj& lo : h->lin) lv.push_back(view(lo));
+        CK(h->lat_lin.alloc(lv.size() * sizeof(LatLinear)));
+        CK(cudaMemcpy(h->lat_lin.p, lv.data(), lv.size() * sizeof(LatLinear), cudaMemcpyHostToDevice));
+        if (!h->lat_kv.p) {
+            const int max_f = h->n_sms / lat_tiles_per_frame(h);
+            CK(h->lat_kv.alloc((size_t)2 * std::max(1, max_f) * h->tokens * 2 * c.d * sizeof(bf16)));
+            CK(h->lat_bar.alloc(sizeof(unsigned int) * std::max(1, max_f)));
+        }
+        h->lat_dirty = false;
+    }
+    LatArgs a;
+    a.frames = (const bf16*)frames; a.n_frames = n_frames; a.img = c.img; a.grid = c.img / c.patch; a.tokens = h->tokens;
+    a.tiles_pf = lat_tiles_per_frame(h); a.d = c.d; a.heads = c.heads; a.mlp = c.mlp; a.layers = c.layers;
+    a.n_classes = c.n_classes; a.patch_dim = h->patch_dim; a.eps = c.ln_eps;
+    a.patch = view(h->patch); a.lin = h->lat_lin.as<LatLinear>();
+    a.cls = h->cls.as<float>(); a.pos = h->pos.as<float>(); a.lnf_g = h->lnf_g.as<float>(); a.lnf_b = h->lnf_b.as<float>();
+    a.head_wt = h->head_wt.as<bf16>(); a.head_b = h->head_b.as<float>();
+    a.hcat = h->hcat.as<bf16>(); a.hbias = h->hbias.as<float>(); a.hcls = h->hcls.as<int>(); a.hoff = h->hoff.as<int>();
+    a.set_off = d_off; a.set_ids = d_ids; a.perm = perm;
+    a.max_set = c.max_set; a.max_adapters = c.max_adapters; a.slabs_max = h->slabs_max;
+    a.rank = h->meta.rank; a.scale = h->meta.scale;
+    a.kv = h->lat_kv.as<bf16>(); a.bar = h->lat_bar.as<unsigned int>();
+    a.scores_out = scores_out; a.base_out = base_out; a.status = nullptr;
+    Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
+    CK(launch_latency_forward(L, a));
+    return PM_OK;
+}
+
 template <typename T>
 int create_t(pm_handle_s* h, const pm_backbone* w) {
     std::string& err = h->err;
@@ -832,7 +892,7 @@ int pm_register_adapter(pm_handle h, int id, const pm_adapter* a) {
     h->head_b_host[id].assign(a->head_b, a->head_b + a->n_cls);
     if (a->acc) h->acc[id].assign(a->acc, a->acc + a->n_cls);
     else h->acc[id].assign(a->n_cls, 1.f);
-    h->heads_dirty = true; h->cover_ready = false;
+    h->heads_dirty = true; h->cover_ready = false; h->lat_dirty = true;
     h->router.invalidate();
     h->drop_graphs();                 // recorded launch sequences refer to the old adapters and heads
     return sync_meta(h->scale_dev, h->rank_dev, h->scales, h->ranks, err);
@@ -903,8 +963,14 @@ int pm_forward(pm_handle h, const void* frames, int n_frames, const int32_t* set
     // the kernels read the plan from device tables at fixed addresses; of its contents only the widest
     // set shapes the launch sequence, so a recorded sequence is replayed for any sets of the same width
     key.key_int[2] = h->router.dev.max_set;
+    const bool small = latency_eligible(h, n_frames);
+    key.key_int[3] = small ? 1 : 0;
     key.plan_version = 0; key.st = st;
     return run_graphed(h, key, [&]() {
+        if (small) {
+            const RouteDev& R = h->router.dev;
+            return forward_latency(h, frames, n_frames, R.perm, R.slot_off, R.slot_ids, scores_out, base_out, st);
+        }
         return h->cfg.dtype == 0 ? forward_t<bf16>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st)
                                  : forward_t<float>(h, frames, n_frames, n_frames, 0, scores_out, base_out, st);
     });
@@ -930,9 +996,13 @@ int pm_forward_device_sets(pm_handle h, const void* frames, int n_frames, const 
     key.key_ptr[0] = frames; key.key_ptr[1] = scores_out; key.key_ptr[2] = base_out;
     key.key_ptr[3] = set_offsets; key.key_ptr[4] = set_ids;
     key.key_int[0] = n_frames; key.key_int[1] = 1 /* entry point */;
+    const bool small = latency_eligible(h, n_frames);
+    key.key_int[3] = small ? 1 : 0;
     // the launch sequence of a device plan depends on the frame count only, not on the lists
     key.plan_version = 0; key.st = st;
     return run_graphed(h, key, [&]() {
+        // a handful of frames of a small model: the whole network in one launch, straight from the lists
+        if (small) return forward_latency(h, frames, n_frames, nullptr, set_offsets, set_ids, scores_out, base_out, st);
         Launch L; L.st = st; L.launches = &h->launches; L.status = h->status.as<int>(); L.prof = &h->prof;
         int rc = h->router.build_on_device(L, n_frames, set_offsets, set_ids, h->meta, err);
         if (rc) return rc;
@@ -1096,6 +1166,12 @@ int pm_plan_stats(pm_handle h, long long* plans_built, double* host_ms) {
     if (!h) return PM_ERR_ARG;
     if (plans_built) *plans_built = h->router.plans_built;
     if (host_ms) *host_ms = h->router.plan_host_ms;
+    return PM_OK;
+}
+
+int pm_set_small_batch_kernel(pm_handle h, int on) {
+    if (!h) return PM_ERR_ARG;
+    h->lat_on = on != 0;
     return PM_OK;
 }
 

@@ -204,6 +204,50 @@ struct SmemGrant {
     }
 };
 
+// ---- whole-network kernel for a handful of frames (latency_kernel.cu)
+// One linear as this kernel sees it (device pointers into the handle's weights and LoRA arenas).
+struct LatLinear {
+    const bf16* Wt;            // [n_out, k_in]
+    const float* bias;         // [n_out]
+    const float* ln_g;         // [n_out] or null (LayerNorm folded into W)
+    const bf16* At;            // [max_adapters * RS, k_in] or null
+    const bf16* Bt;            // [max_adapters * slabs_max][n_out][16]
+    const float* c1;           // [max_adapters * RS] (folded linears)
+    const float* c2;
+    uint32_t adapted[8];       // bit a: adapter a really touches this linear
+    int k_in, n_out;
+};
+
+struct LatArgs {
+    const bf16* frames;        // [F, 3, img, img]
+    int n_frames, img, grid, tokens, tiles_pf, d, heads, mlp, layers, n_classes, patch_dim;
+    float eps;
+    LatLinear patch;
+    const LatLinear* lin;      // [layers * 4]
+    const float *cls, *pos, *lnf_g, *lnf_b;
+    const bf16* head_wt;       // [n_classes, d]
+    const float* head_b;
+    const bf16* hcat;          // adapter head rows [sum n_cls, d]
+    const float* hbias;
+    const int *hcls, *hoff;
+    const int *set_off, *set_ids;          // device CSR over slots (slot s = CTA group s)
+    const int* perm;                       // [F] slot -> caller's frame index, or null (slot = frame)
+    int max_set, max_adapters, slabs_max;
+    const int* rank;
+    const float* scale;
+    bf16* kv;                  // [2][F * tokens][2 d]: keys and values of the blocks, two buffers used in turn
+    unsigned int* bar;         // [F] arrival counters of the frames' CTAs (cleared before every launch)
+    float *scores_out, *base_out;          // [F, n_classes]
+    int* status;
+};
+
+// bytes of dynamic shared memory the kernel needs for this geometry (rs_total = slabs_max * 16 * max_set)
+size_t latency_smem_bytes(int d, int mlp, int patch_dim, int rs_total, int tokens);
+// One launch for the whole forward of a.n_frames frames; a.status is taken from L.  The grid
+// (n_frames * tiles_pf CTAs, one per SM) must be resident at once: a cooperative launch, which fails
+// with an error instead of starting if it cannot be.
+cudaError_t launch_latency_forward(const Launch& L, const LatArgs& a);
+
 // tensor-map helpers (gemm_tcgen05.cu); return false if the driver entry point is unavailable
 bool tm_encode_2d(CUtensorMap* tm, const void* base, uint64_t inner, uint64_t outer,
                   uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, int swizzle);

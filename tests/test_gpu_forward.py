@@ -69,6 +69,50 @@ def test_deit_tiny_2frames(dtype):
     m.close()
 
 
+@pytest.mark.parametrize("which", ["all_linears_rank4", "query_value_last_blocks_rank16"])
+def test_small_batch_kernel_against_oracle_and_layer_kernels(which):
+    """A handful of frames of a small model run as one whole-network kernel (a CTA owns 16 token rows
+    from the patch embedding to the last block).  Same inputs through that kernel and through the
+    layer-by-layer kernels: both within the score tolerance of the oracle, and the one-kernel path
+    really is one kernel per forward."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    if which == "all_linears_rank4":
+        w = wl.deit_tiny_2frames()
+        frames, sets = w.frames, [[0], [1, 3]]
+    else:
+        w = wl.deit_tiny_stream(n_steps=3, n_streams=1)
+        frames = w.extra["stream_frames"][0, :3]                      # three frames of the stream as a batch
+        sets = [[], [2, 5, 9], [0]]
+    off, ids = wl.sets_to_csr(sets)
+    m = binding.model_from_workload(w, dtype=0, max_frames=len(sets), max_set=8)
+    so, bo = po.forward(w.backbone, w.adapters, frames, off, ids, w.spec.heads, w.spec.patch, w.spec.ln_eps,
+                        w.spec.n_classes)
+    got = {}
+    for on in (True, False):
+        m.set_small_batch_kernel(on)
+        n0 = m.launch_count()
+        got[on] = run_forward(m, w, 0, frames=frames, offsets=off, ids=ids)
+        launches = m.launch_count() - n0
+        assert (launches == 1) if on else (launches > 50)
+        assert np.abs(got[on][0] - so).max() < 1e-2 and np.abs(got[on][1] - bo).max() < 1e-2
+        # device-resident lists take the same path
+        fd = frames_to_dev(frames, 0)
+        s2 = torch.zeros((len(sets), w.spec.n_classes), device="cuda")
+        b2 = torch.zeros_like(s2)
+        m.forward_device_sets(fd, torch.from_numpy(off).cuda(), torch.from_numpy(ids if len(ids) else np.zeros(1, np.int32)).cuda(),
+                              s2, b2)
+        assert m.status() == 0
+        np.testing.assert_array_equal(s2.cpu().numpy(), got[on][0].astype(np.float32))
+        np.testing.assert_array_equal(b2.cpu().numpy(), got[on][1].astype(np.float32))
+    for f, st in enumerate(sets):                                    # exact zeros outside the active subsets
+        allowed = np.zeros(w.spec.n_classes, bool)
+        for a in st:
+            allowed[w.adapters[a].class_ids] = True
+        assert np.all(got[True][0][f][~allowed] == 0) and np.all(got[True][0][f][allowed] > 0)
+    m.close()
+
+
 def test_recorded_sequence_follows_changing_sets():
     """On a stream of its own the third identical call replays a recorded launch sequence.  When the
     sets then change (same widest set) the replay must use the newly uploaded routing plan: results
@@ -126,6 +170,7 @@ def test_paper_variant_query_value_last_blocks(dtype):
                               head_w=ad.head_w, head_b=ad.head_b, acc=ad.acc))
     w2 = wl.Workload(w.name, w.spec, w.backbone, ads, w.frames, w.set_offsets, w.set_ids)
     m = binding.model_from_workload(w2, dtype=dtype)
+    m.set_small_batch_kernel(False)                    # the launch counts below are about the layer-by-layer path
     n0 = m.launch_count()
     s, b = run_forward(m, w2, dtype)
     launches = m.launch_count() - n0
@@ -138,6 +183,7 @@ def test_paper_variant_query_value_last_blocks(dtype):
     assert np.abs(bo - bo_plain).max() > 1e-4
     if dtype == 0:
         m_all = binding.model_from_workload(w, dtype=0)
+        m_all.set_small_batch_kernel(False)
         n1 = m_all.launch_count()
         run_forward(m_all, w, 0)
         # 48 shrink launches against 2; a shrink in front of qkv or fc1 also yields the LayerNorm row
@@ -147,7 +193,8 @@ def test_paper_variant_query_value_last_blocks(dtype):
     m.close()
 
 
-def test_recorded_launch_sequence_replays_identically():
+@pytest.mark.parametrize("small_kernel", [False, True])
+def test_recorded_launch_sequence_replays_identically(small_kernel):
     """On a stream of its own the forward records its launch sequence the second time it sees the same
     call and replays it afterwards: same results, same launch count per call; a change of the sets makes
     a new plan and is honoured; the device-plan entry point replays with lists that change in place."""
@@ -155,6 +202,7 @@ def test_recorded_launch_sequence_replays_identically():
     from paper_2507_14959_b200 import binding
     w = wl.deit_tiny_2frames()
     m = binding.model_from_workload(w, dtype=0)
+    m.set_small_batch_kernel(small_kernel)                  # the layer-by-layer sequence, or the one whole-network kernel
     K = w.spec.n_classes
     fd = frames_to_dev(w.frames, 0)
     ref_s, ref_b = run_forward(m, w, 0)                     # legacy default stream: never recorded
