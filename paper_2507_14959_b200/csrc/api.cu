@@ -466,6 +466,7 @@ struct pm_handle_s {
     std::string err;
     // whole-network kernel for a handful of frames (latency_kernel.cu)
     DevBuf lat_lin, lat_kv, lat_bar;
+    CUtensorMap lat_tm_kv;
     bool lat_dirty = true, lat_on = true;
     // recorded launch sequences of the forward entry points (see run_graphed)
     struct GraphEntry {
@@ -709,6 +710,7 @@ int lat_tiles_per_frame(const pm_handle_s* h) { return (h->tokens + LAT_ROWS - 1
 bool latency_eligible(const pm_handle_s* h, int n_frames) {
     const pm_config& c = h->cfg;
     if (!h->lat_on || c.dtype != 0 || c.d > 384 || c.mlp > 1536 || h->patch_dim > 1536 || c.max_set > 8) return false;
+    if (h->tokens > 256) return false;               // a head's keys are one TMA box
     if (h->slabs_max * PM_SLAB * c.max_set > 512) return false;
     if ((long long)n_frames * lat_tiles_per_frame(h) > h->n_sms) return false;       // one CTA per SM, all resident
     return latency_smem_bytes(c.d, c.mlp, h->patch_dim, h->slabs_max * PM_SLAB * c.max_set, h->tokens) <= 227 * 1024;
@@ -721,6 +723,8 @@ int forward_latency(pm_handle_s* h, const void* frames, int n_frames, const int*
     const pm_config& c = h->cfg;
     auto view = [](const LinearObj& lo) {
         LatLinear v;
+        v.tm_w = lo.dev.has_tm_half ? lo.dev.tm_w_half : lo.dev.tm_w;      // both fetch [128 rows][64 columns]
+        v.tm_at = lo.dev.tm_at;
         v.Wt = (const bf16*)lo.dev.Wt; v.bias = lo.dev.bias; v.ln_g = lo.dev.ln_g;
         v.At = (const bf16*)lo.dev.lora.At; v.Bt = (const bf16*)lo.dev.lora.Bt; v.c1 = lo.dev.ln_c1; v.c2 = lo.dev.ln_c2;
         for (int i = 0; i < 8; ++i) v.adapted[i] = 0u;
@@ -732,12 +736,19 @@ int forward_latency(pm_handle_s* h, const void* frames, int n_frames, const int*
     if (h->lat_dirty) {
         std::vector<LatLinear> lv;
         for (const LinearObj& lo : h->lin) lv.push_back(view(lo));
+        lv.push_back(view(h->patch));
         CK(h->lat_lin.alloc(lv.size() * sizeof(LatLinear)));
         CK(cudaMemcpy(h->lat_lin.p, lv.data(), lv.size() * sizeof(LatLinear), cudaMemcpyHostToDevice));
         if (!h->lat_kv.p) {
             const int max_f = h->n_sms / lat_tiles_per_frame(h);
-            CK(h->lat_kv.alloc((size_t)2 * std::max(1, max_f) * h->tokens * 2 * c.d * sizeof(bf16)));
+            const size_t kv_rows = (size_t)2 * std::max(1, max_f) * h->tokens;
+            CK(h->lat_kv.alloc(kv_rows * 2 * c.d * sizeof(bf16)));
+            CK(cudaMemset(h->lat_kv.p, 0, h->lat_kv.bytes));
             CK(h->lat_bar.alloc(sizeof(unsigned int) * std::max(1, max_f)));
+            const int tpad = (h->tokens + 15) / 16 * 16;
+            if (tpad > 256 || !tm_encode_2d(&h->lat_tm_kv, h->lat_kv.p, (uint64_t)2 * c.d, kv_rows, (uint64_t)2 * c.d * 2, 64, tpad, 128)) {
+                err = "cuTensorMapEncodeTiled failed (key/value exchange buffer)"; return PM_ERR_CUDA;
+            }
         }
         h->lat_dirty = false;
     }
@@ -745,7 +756,7 @@ int forward_latency(pm_handle_s* h, const void* frames, int n_frames, const int*
     a.frames = (const bf16*)frames; a.n_frames = n_frames; a.img = c.img; a.grid = c.img / c.patch; a.tokens = h->tokens;
     a.tiles_pf = lat_tiles_per_frame(h); a.d = c.d; a.heads = c.heads; a.mlp = c.mlp; a.layers = c.layers;
     a.n_classes = c.n_classes; a.patch_dim = h->patch_dim; a.eps = c.ln_eps;
-    a.patch = view(h->patch); a.lin = h->lat_lin.as<LatLinear>();
+    a.lin = h->lat_lin.as<LatLinear>(); a.tm_kv = h->lat_tm_kv;
     a.cls = h->cls.as<float>(); a.pos = h->pos.as<float>(); a.lnf_g = h->lnf_g.as<float>(); a.lnf_b = h->lnf_b.as<float>();
     a.head_wt = h->head_wt.as<bf16>(); a.head_b = h->head_b.as<float>();
     a.hcat = h->hcat.as<bf16>(); a.hbias = h->hbias.as<float>(); a.hcls = h->hcls.as<int>(); a.hoff = h->hoff.as<int>();

@@ -207,6 +207,8 @@ struct SmemGrant {
 // ---- whole-network kernel for a handful of frames (latency_kernel.cu)
 // One linear as this kernel sees it (device pointers into the handle's weights and LoRA arenas).
 struct LatLinear {
+    CUtensorMap tm_w;          // W^T [n_out, k_in], boxes of [128 rows][64 columns], 128B swizzle
+    CUtensorMap tm_at;         // A^T arena [max_adapters * RS, k_in], boxes of [16 rows][64 columns]
     const bf16* Wt;            // [n_out, k_in]
     const float* bias;         // [n_out]
     const float* ln_g;         // [n_out] or null (LayerNorm folded into W)
@@ -222,8 +224,8 @@ struct LatArgs {
     const bf16* frames;        // [F, 3, img, img]
     int n_frames, img, grid, tokens, tiles_pf, d, heads, mlp, layers, n_classes, patch_dim;
     float eps;
-    LatLinear patch;
-    const LatLinear* lin;      // [layers * 4]
+    const LatLinear* lin;      // [layers * 4 + 1]: the blocks' linears, then the patch projection
+    CUtensorMap tm_kv;         // the exchange buffer as [2 * F * tokens, 2 d], boxes of [tpad rows][64 columns]
     const float *cls, *pos, *lnf_g, *lnf_b;
     const bf16* head_wt;       // [n_classes, d]
     const float* head_b;

@@ -4,7 +4,8 @@
 //
 // Everything in a ViT block except attention is local to a token row, so a CTA owns 16 token rows of one
 // frame from the first layer to the last and keeps their residual stream (fp32) and every intermediate in
-// shared memory; the weights stream through shared memory (cp.async, two stages) and are the only thing
+// shared memory; the weights stream through a ring of 16 KB shared-memory slots filled by TMA (one
+// [128 outputs x 64 inputs] box per slot, 128B swizzle, several boxes in flight) and are the only thing
 // read from L2 -- every CTA reads all of them, which is what bounds a frame's latency.  The one exchange
 // per block is attention: each CTA publishes the keys and values of its rows (two global buffers used in
 // turn), the CTAs of a frame meet at a counter (bounded wait), then each CTA attends from its 16 query rows
@@ -21,9 +22,9 @@ namespace {
 constexpr int LT_ROWS = 16;
 constexpr int LT_THREADS = 256;
 constexpr int LT_WARPS = 8;
-constexpr int LT_KB = 192;                 // K columns of a weight stage
-constexpr int LT_WSTRIDE = LT_KB + 8;      // bf16 per staged weight row (16-byte skew: conflict-free ldmatrix)
-constexpr int LT_NCHUNK = 64;              // output columns per stage: one n8 tile per warp
+constexpr int LT_GROUP = 3;                // K boxes multiplied between two CTA-wide barriers
+constexpr int LT_SLOTS = 2 * LT_GROUP;     // weight ring: two groups of boxes
+constexpr int LT_BOX_BYTES = 128 * 128;    // [128 output rows][64 bf16 inputs], 128B swizzle
 constexpr int LT_MAX_SET = 8;
 constexpr int LT_HD = 64;
 constexpr long long LT_WAIT_CYCLES = 4000000000ll;
@@ -56,33 +57,52 @@ __device__ __forceinline__ void cp16(uint32_t dst, const void* src) {
 }
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_expect(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t bar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
 
 }  // namespace
 
 namespace {
 
 struct LatSmem {               // offsets (bytes) into dynamic shared memory
-    int xres, abuf, hbuf, qbuf, tbuf, stats, region, part, misc, total;
+    int region, xres, abuf, hbuf, qbuf, tbuf, stats, part, misc, total;
     int lda, ldh, ldq, ldt;    // row strides in bf16 elements
+    int kv_head;               // bytes of one head's keys + values in the region
 };
 
 __host__ __device__ inline LatSmem lat_layout(int d, int mlp, int patch_dim, int rs_total, int tokens) {
     LatSmem s;
     auto up = [](int v) { return (v + 127) & ~127; };
     s.lda = d + 8; s.ldh = (mlp > patch_dim ? mlp : patch_dim) + 8; s.ldq = d + 8; s.ldt = rs_total + 8;
+    // first (1024-byte aligned, as the 128B swizzle wants): the weight ring, or two heads' keys and values
+    // (each [tpad rows][128 bytes]) -- the next head's land while this one is computed
+    const int tpad = (tokens + 15) / 16 * 16;
+    s.kv_head = 2 * ((tpad * 128 + 1023) & ~1023);
+    const int wbytes = LT_SLOTS * LT_BOX_BYTES, kvbytes = 2 * s.kv_head;
     int o = 0;
+    s.region = o; o = up(o + (wbytes > kvbytes ? wbytes : kvbytes));
     s.xres = o; o = up(o + LT_ROWS * d * 4);
     s.abuf = o; o = up(o + LT_ROWS * s.lda * 2);
     s.hbuf = o; o = up(o + LT_ROWS * s.ldh * 2);
     s.qbuf = o; o = up(o + LT_ROWS * s.ldq * 2);
     s.tbuf = o; o = up(o + LT_ROWS * s.ldt * 2);
     s.stats = o; o = up(o + LT_ROWS * 16);
-    // weight stages (2 x 64 rows) or one head's keys and values (2 x tpad rows of 128 bytes)
-    const int tpad = (tokens + 15) / 16 * 16;
-    const int wbytes = 2 * LT_NCHUNK * LT_WSTRIDE * 2, kvbytes = 2 * tpad * 128;
-    s.region = o; o = up(o + (wbytes > kvbytes ? wbytes : kvbytes));
     s.part = o; o = up(o + LT_WARPS * LT_ROWS * (LT_HD + 2) * 4);      // partial attention results of the warps
-    s.misc = o; o = up(o + 256);
+    s.misc = o; o = up(o + 512);     // the adapter set, abort flag, mbarriers
     s.total = o;
     return s;
 }
@@ -91,16 +111,27 @@ struct Ctx {
     uint8_t* sm;
     LatSmem L;
     int warp, lane, g, t;
+    uint32_t box_no;           // boxes that have gone through the weight ring so far (the same in every thread)
+    uint32_t kv_no;            // head buffers filled so far
+    int* status;
+    volatile int* abort_flag;
 };
 
-// Streams W^T rows [n0, n0 + 64) x columns [k0, k0 + len) into stage `buf` (rows past n_out are skipped:
-// their products are never used).
-__device__ __forceinline__ void stage_weights(const Ctx& cx, int buf, const bf16* Wt, int N, int K, int n0, int k0, int len) {
-    const int chunks = len >> 3;                     // 16-byte pieces per row
-    const uint32_t dst0 = s_u32(cx.sm + cx.L.region) + buf * (LT_NCHUNK * LT_WSTRIDE * 2);
-    for (int i = threadIdx.x; i < LT_NCHUNK * chunks; i += LT_THREADS) {
-        const int r = i / chunks, c = i % chunks;
-        if (n0 + r < N) cp16(dst0 + (r * LT_WSTRIDE + c * 8) * 2, Wt + (size_t)(n0 + r) * K + k0 + c * 8);
+__device__ __forceinline__ uint32_t ring_bar(const Ctx& cx, int slot) { return s_u32(cx.sm + cx.L.misc + 256) + 8u * slot; }
+__device__ __forceinline__ uint32_t kv_bar(const Ctx& cx, int buf) { return s_u32(cx.sm + cx.L.misc + 256) + 8u * (LT_SLOTS + buf); }
+
+// Bounded wait on a transaction barrier (every thread of the CTA may call it).  Once a wait has run out
+// the CTA is aborting: later waits return at once and the results are meaningless (the status word says so).
+__device__ __forceinline__ void bar_wait(const Ctx& cx, uint32_t bar, uint32_t parity) {
+    if (bar_try(bar, parity)) return;
+    const long long t0 = clock64();
+    while (!bar_try(bar, parity)) {
+        if (*cx.abort_flag) return;
+        if (clock64() - t0 > LT_WAIT_CYCLES) {
+            *cx.abort_flag = 1;
+            atomicCAS(cx.status, 0, (int)PM_ERR_TIMEOUT);
+            return;
+        }
     }
 }
 
@@ -112,66 +143,106 @@ struct LoraExp {               // LoRA expand of the current linear: t (shared m
 };
 
 // y[16, N] = A[16, K] W + LoRA expand, handed element-wise to epi(row, n, value).  A: bf16 in shared memory
-// with row stride lda.  All threads of the CTA call it.
+// with row stride lda; rows [row0, row0 + N) of the [*, K] matrix behind `tm` come through the ring as TMA
+// boxes of [box_rows outputs][64 inputs] (box_rows = 128 for the weights: two n8 tiles per warp; 16 for a
+// LoRA slab of A^T: warp 0 alone).  All threads of the CTA call it; thread 0 issues the copies.
+// col0 / col1: optional per-output-column vectors (bias; LayerNorm g or c1 ...); a thread's four values of
+// each are fetched while the last K box is still being multiplied and handed to epi, so that the epilogue's
+// stores never sit between a load and its use.
 template <typename Epi>
-__device__ void linear16(const Ctx& cx, const bf16* A, int lda, const bf16* Wt, int N, int K, const LoraExp* lx, Epi epi) {
-    const int n_chunks = (N + LT_NCHUNK - 1) / LT_NCHUNK, k_blocks = (K + LT_KB - 1) / LT_KB;
-    const int total = n_chunks * k_blocks;
-    const uint32_t a_base = s_u32(A), w_base = s_u32(cx.sm + cx.L.region), t_base = s_u32(cx.sm + cx.L.tbuf);
+__device__ void linear16(Ctx& cx, const bf16* A, int lda, const CUtensorMap* tm, int box_rows, int row0, int N, int K,
+                         const LoraExp* lx, const float* col0, const float* col1, Epi epi) {
+    const int n_chunks = (N + box_rows - 1) / box_rows, k_boxes = K >> 6;
+    // boxes go through the ring in groups of up to LT_GROUP consecutive K boxes of one chunk of outputs: one
+    // CTA-wide barrier per group, and while a group is multiplied the next one is on its way
+    const int gpc = (k_boxes + LT_GROUP - 1) / LT_GROUP, n_groups = n_chunks * gpc;
+    const uint32_t a_base = s_u32(A), ring = s_u32(cx.sm + cx.L.region), t_base = s_u32(cx.sm + cx.L.tbuf);
     const int lane = cx.lane, warp = cx.warp;
-    stage_weights(cx, 0, Wt, N, K, 0, 0, min(LT_KB, K));
-    cp_commit();
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int it = 0; it < total; ++it) {
-        const int nc = it / k_blocks, kb = it % k_blocks;
-        if (it + 1 < total) {
-            const int nc1 = (it + 1) / k_blocks, kb1 = (it + 1) % k_blocks;
-            stage_weights(cx, (it + 1) & 1, Wt, N, K, nc1 * LT_NCHUNK, kb1 * LT_KB, min(LT_KB, K - kb1 * LT_KB));
-            cp_commit();
-            cp_wait<1>();
-        } else {
-            cp_wait<0>();
+    uint32_t issued = cx.box_no;                      // number of the next box to issue (the same in every thread)
+    auto issue_group = [&](int g) {
+        const int nc = g / gpc, kb0 = (g % gpc) * LT_GROUP, nb = min(LT_GROUP, k_boxes - kb0);
+        if (lane == 0 && warp < nb) {                 // box j of the group: lane 0 of warp j
+            const int slot = (int)((issued + (uint32_t)warp) % LT_SLOTS);
+            bar_expect(ring_bar(cx, slot), (uint32_t)box_rows * 128u);
+            tma_box(ring + slot * LT_BOX_BYTES, tm, (kb0 + warp) * 64, row0 + nc * box_rows, ring_bar(cx, slot));
         }
-        __syncthreads();
-        const int n8 = nc * LT_NCHUNK + warp * 8;
-        const bool active = n8 < N;
-        if (kb == 0) { acc[0] = acc[1] = acc[2] = acc[3] = 0.f; }
-        if (active) {
-            const int k0 = kb * LT_KB, len = min(LT_KB, K - k0);
-            const uint32_t a_row = a_base + ((lane & 15) * lda + k0 + (lane >> 4) * 8) * 2;
-            const uint32_t w_row = w_base + (it & 1) * (LT_NCHUNK * LT_WSTRIDE * 2) +
-                                   ((warp * 8 + (lane & 7)) * LT_WSTRIDE + ((lane >> 3) & 1) * 8) * 2;
-            for (int kk = 0; kk < len; kk += 16) {
-                uint32_t a[4], b0, b1;
-                ldsm4(a_row + kk * 2, a[0], a[1], a[2], a[3]);
-                ldsm2(w_row + kk * 2, b0, b1);
-                mma16816(acc, a, b0, b1);
+        issued += (uint32_t)nb;
+    };
+    issue_group(0);
+    float acc[2][4];
+    const int row16 = warp * 16;                   // this warp's rows of a box
+    const int mi = lane >> 3;
+    const int r = row16 + (mi >> 1) * 8 + (lane & 7);
+    for (int g = 0; g < n_groups; ++g) {
+        // the slots freed by the previous group (everyone is past its closing barrier) take the next one
+        if (g + 1 < n_groups) issue_group(g + 1);
+        const int nc = g / gpc, kb0 = (g % gpc) * LT_GROUP, nb = min(LT_GROUP, k_boxes - kb0);
+        const bool last = kb0 + nb == k_boxes;
+        if (kb0 == 0) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
+        }
+        const int n16 = nc * box_rows + row16;
+        const bool active = row16 < box_rows && n16 < N;
+        float cv0[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, cv1[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        if (active && last) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int n = n16 + q * 8 + 2 * cx.t;
+                if (n16 + q * 8 < N) {
+                    if (col0) { const float2 v = __ldg(reinterpret_cast<const float2*>(col0 + n)); cv0[q][0] = v.x; cv0[q][1] = v.y; }
+                    if (col1) { const float2 v = __ldg(reinterpret_cast<const float2*>(col1 + n)); cv1[q][0] = v.x; cv1[q][1] = v.y; }
+                }
             }
-            if (kb == k_blocks - 1) {
+        }
+        for (int j = 0; j < nb; ++j) {
+            const uint32_t no = cx.box_no + (uint32_t)j;
+            const int slot = (int)(no % LT_SLOTS);
+            bar_wait(cx, ring_bar(cx, slot), (no / LT_SLOTS) & 1u);
+            if (active) {
+                const uint32_t a_row = a_base + ((lane & 15) * lda + (kb0 + j) * 64 + (lane >> 4) * 8) * 2;
+                const uint32_t box = ring + slot * LT_BOX_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    uint32_t a[4], b0, b1, b2, b3;
+                    ldsm4(a_row + ks * 32, a[0], a[1], a[2], a[3]);
+                    const int c = ks * 2 + (mi & 1);
+                    ldsm4(box + r * 128 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
+                    mma16816(acc[0], a, b0, b1);
+                    mma16816(acc[1], a, b2, b3);
+                }
+            }
+        }
+        cx.box_no += (uint32_t)nb;
+        if (active && last) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int n8 = n16 + q * 8;
+                if (n8 >= N) break;
                 if (lx) {
                     for (int p = 0; p < lx->n_act; ++p)
-                        for (int s = 0; s < lx->slabs[p]; ++s) {
+                        for (int sl = 0; sl < lx->slabs[p]; ++sl) {
                             uint32_t a[4];
-                            ldsm4(t_base + ((lane & 15) * cx.L.ldt + p * lx->rs + s * 16 + (lane >> 4) * 8) * 2, a[0], a[1], a[2], a[3]);
-                            const bf16* bp = lx->Bt + (((size_t)(lx->adapter[p] * lx->slabs_max + s) * N) + n8 + cx.g) * PM_SLAB;
+                            ldsm4(t_base + ((lane & 15) * cx.L.ldt + p * lx->rs + sl * 16 + (lane >> 4) * 8) * 2, a[0], a[1], a[2], a[3]);
+                            const bf16* bp = lx->Bt + (((size_t)(lx->adapter[p] * lx->slabs_max + sl) * N) + n8 + cx.g) * PM_SLAB;
                             const uint32_t b0 = __ldg(reinterpret_cast<const unsigned int*>(bp + 2 * cx.t));
                             const uint32_t b1 = __ldg(reinterpret_cast<const unsigned int*>(bp + 2 * cx.t + 8));
-                            mma16816(acc, a, b0, b1);
+                            mma16816(acc[q], a, b0, b1);
                         }
                 }
                 const int n = n8 + 2 * cx.t;
-                epi(cx.g, n, acc[0]); epi(cx.g, n + 1, acc[1]);
-                epi(cx.g + 8, n, acc[2]); epi(cx.g + 8, n + 1, acc[3]);
+                epi(cx.g, n, acc[q][0], cv0[q][0], cv1[q][0]); epi(cx.g, n + 1, acc[q][1], cv0[q][1], cv1[q][1]);
+                epi(cx.g + 8, n, acc[q][2], cv0[q][0], cv1[q][0]); epi(cx.g + 8, n + 1, acc[q][3], cv0[q][1], cv1[q][1]);
             }
         }
-        __syncthreads();          // the stage may be overwritten two iterations from now
+        __syncthreads();          // the group's slots are refilled by the next iteration's copies
     }
 }
 
 __device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
 
 // abuf <- bf16(xres); stats[r] = (mean, rstd, 1/rstd) of the rounded row (what the tensor cores multiply)
-__device__ void round_rows_and_stats(const Ctx& cx, int d, float eps) {
+__device__ void round_rows_and_stats(Ctx& cx, int d, float eps) {
     const float* x = reinterpret_cast<const float*>(cx.sm + cx.L.xres);
     bf16* a = reinterpret_cast<bf16*>(cx.sm + cx.L.abuf);
     float4* st = reinterpret_cast<float4*>(cx.sm + cx.L.stats);
@@ -207,7 +278,7 @@ struct ActiveSet { int n; int id[LT_MAX_SET]; int slabs[LT_MAX_SET]; float scale
 // LoRA shrink for the adapters of `as` that touch `lin`: t[r][p * rs + j] (bf16) = s_a (x A_a) (folded
 // linears: s_a ((x A' - mean c1) + c2 / rstd), the fused accumulator being scaled by rstd afterwards).
 // Returns the expand description (adapters in ascending id).
-__device__ void lora_shrink(const Ctx& cx, const LatLinear& lin, const ActiveSet& as, int slabs_max, const bf16* A, int lda,
+__device__ void lora_shrink(Ctx& cx, const LatLinear& lin, const ActiveSet& as, int slabs_max, const bf16* A, int lda,
                             LoraExp* lx) {
     lx->n_act = 0; lx->Bt = lin.Bt; lx->slabs_max = slabs_max; lx->rs = slabs_max * PM_SLAB;
     if (!lin.At) return;
@@ -224,17 +295,21 @@ __device__ void lora_shrink(const Ctx& cx, const LatLinear& lin, const ActiveSet
         const float* c2 = lin.c2 ? lin.c2 + (size_t)a * lx->rs : nullptr;
         const bool folded = lin.ln_g != nullptr;
         const int ldt = cx.L.ldt, col0 = p * lx->rs;
-        linear16(cx, A, lda, lin.At + (size_t)a * lx->rs * lin.k_in, rs_a, lin.k_in, nullptr,
-                 [&](int r, int j, float v) {
-                     if (folded) v = (v - st[r].x * c1[j]) + c2[j] * st[r].z;
+        linear16(cx, A, lda, &lin.tm_at, PM_SLAB, a * lx->rs, rs_a, lin.k_in, nullptr, folded ? c1 : nullptr, folded ? c2 : nullptr,
+                 [&](int r, int j, float v, float c1j, float c2j) {
+                     if (folded) v = (v - st[r].x * c1j) + c2j * st[r].z;
                      tb[r * ldt + col0 + j] = __float2bfloat16_rn(v * sc);
                  });
     }
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const LatArgs args) {
-    extern __shared__ __align__(128) uint8_t smem[];
+__global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __grid_constant__ LatArgs args) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if (s_u32(smem) & 1023u) {                 // swizzled boxes need a 1024-byte aligned window
+        if (threadIdx.x == 0) atomicCAS(args.status, 0, (int)PM_ERR_CUDA);
+        return;
+    }
     Ctx cx;
     cx.sm = smem;
     cx.L = lat_layout(args.d, args.mlp, args.patch_dim, args.slabs_max * PM_SLAB * args.max_set, args.tokens);
@@ -250,6 +325,12 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const La
     const float4* stats = reinterpret_cast<const float4*>(smem + cx.L.stats);
     ActiveSet* as = reinterpret_cast<ActiveSet*>(smem + cx.L.misc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + cx.L.misc + 192);
+    cx.box_no = 0; cx.kv_no = 0; cx.status = args.status; cx.abort_flag = abort_flag;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < LT_SLOTS + 2; ++i) bar_init(ring_bar(cx, i), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
 
     // ---- the frame's adapter set: valid, registered, distinct ids in ascending order
     if (threadIdx.x == 0) {
@@ -297,11 +378,13 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const La
     __syncthreads();
     const ActiveSet aset = *as;
     // ---- patch projection + positions; the CLS row
-    linear16(cx, hbuf, cx.L.ldh, args.patch.Wt, d, args.patch_dim, nullptr, [&](int r, int n, float v) {
+    const LatLinear* patch = args.lin + (size_t)args.layers * 4;
+    const float* patch_bias = patch->bias;
+    linear16(cx, hbuf, cx.L.ldh, &patch->tm_w, 128, 0, d, args.patch_dim, nullptr, patch_bias, nullptr, [&](int r, int n, float v, float b, float) {
         const int tok = r0 + r;
         float out = 0.f;
         if (tok == 0) out = args.cls[n] + args.pos[n];
-        else if (tok < T) out = v + args.patch.bias[n] + args.pos[(size_t)tok * d + n];
+        else if (tok < T) out = v + b + args.pos[(size_t)tok * d + n];
         xres[r * d + n] = out;                              // rows past the frame stay zero
     });
     __syncthreads();
@@ -317,13 +400,15 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const La
         lora_shrink(cx, lin[0], aset, args.slabs_max, abuf, cx.L.lda, &lx);
         {
             const float* lg = lin[0].ln_g; const float* bb = lin[0].bias;
-            linear16(cx, abuf, cx.L.lda, lin[0].Wt, 3 * d, d, lx.n_act ? &lx : nullptr, [&](int r, int n, float v) {
-                const float y = stats[r].y * (v - stats[r].x * lg[n]) + bb[n];
+            linear16(cx, abuf, cx.L.lda, &lin[0].tm_w, 128, 0, 3 * d, d, lx.n_act ? &lx : nullptr, bb, lg, [&](int r, int n, float v, float b, float gsum) {
+                const float y = stats[r].y * (v - stats[r].x * gsum) + b;
                 if (n < d) qbuf[r * cx.L.ldq + n] = __float2bfloat16_rn(y);
                 else if (r0 + r < T) kvb[(size_t)(r0 + r) * 2 * d + (n - d)] = __float2bfloat16_rn(y);
             });
         }
-        // ---- the CTAs of the frame meet: all keys and values of this block are in place
+        // ---- the CTAs of the frame meet: all keys and values of this block are in place (they were written
+        // with ordinary stores and are fetched by TMA on the other side: order the two proxies as well)
+        asm volatile("fence.proxy.async.global;" ::: "memory");
         __threadfence();
         __syncthreads();
         if (threadIdx.x == 0 && !*abort_flag) {
@@ -343,18 +428,29 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const La
         __syncthreads();
         if (*abort_flag) break;
         // ---- attention, head by head: the warps split the keys, then merge their partial results
+        // keys and values of a head arrive as two TMA boxes ([tpad rows][64 dims], 128B swizzle; rows past
+        // the frame hold a neighbour's rows or zeros and are masked below); the next head's are on their
+        // way while this one is computed
+        const int kv_row0 = ((l & 1) * args.n_frames + f) * T;
+        auto fetch_head = [&](int h) {
+            const int buf = (int)(cx.kv_no & 1u);
+            const uint32_t dst = s_u32(smem + cx.L.region) + buf * cx.L.kv_head;
+            bar_expect(kv_bar(cx, buf), 2u * (uint32_t)tpad * 128u);
+            tma_box(dst, &args.tm_kv, h * LT_HD, kv_row0, kv_bar(cx, buf));
+            tma_box(dst + cx.L.kv_head / 2, &args.tm_kv, d + h * LT_HD, kv_row0, kv_bar(cx, buf));
+        };
+        if (threadIdx.x == 0) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            fetch_head(0);
+        }
         for (int h = 0; h < args.heads; ++h) {
-            uint8_t* Ks = smem + cx.L.region;
-            uint8_t* Vs = Ks + tpad * 128;
-            for (int i = threadIdx.x; i < tpad * 16; i += LT_THREADS) {
-                const int r = i >> 4, c = i & 7, isv = (i >> 3) & 1;
-                uint8_t* dst = (isv ? Vs : Ks) + r * 128 + ((c ^ (r & 7)) << 4);
-                if (r < T) cp16(s_u32(dst), kvb + (size_t)r * 2 * d + isv * d + h * LT_HD + c * 8);
-                else *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-            }
-            cp_commit();
-            cp_wait<0>();
-            __syncthreads();
+            const int buf = (int)(cx.kv_no & 1u);
+            uint8_t* Ks = smem + cx.L.region + buf * cx.L.kv_head;
+            uint8_t* Vs = Ks + cx.L.kv_head / 2;
+            bar_wait(cx, kv_bar(cx, buf), (cx.kv_no >> 1) & 1u);
+            ++cx.kv_no;
+            // the other buffer was last read by head h - 1, and everyone is past that head's closing barrier
+            if (threadIdx.x == 0 && h + 1 < args.heads) fetch_head(h + 1);
             const int n_t8 = tpad / 8;
             const int t8_lo = (n_t8 * cx.warp) / LT_WARPS, t8_hi = (n_t8 * (cx.warp + 1)) / LT_WARPS;    // at most 4 tiles
             const uint32_t ks_addr = s_u32(Ks), vs_addr = s_u32(Vs);
@@ -467,8 +563,8 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const La
         lora_shrink(cx, lin[1], aset, args.slabs_max, abuf, cx.L.lda, &lx);
         {
             const float* bb = lin[1].bias;
-            linear16(cx, abuf, cx.L.lda, lin[1].Wt, d, d, lx.n_act ? &lx : nullptr,
-                     [&](int r, int n, float v) { if (r0 + r < T) xres[r * d + n] += v + bb[n]; });
+            linear16(cx, abuf, cx.L.lda, &lin[1].tm_w, 128, 0, d, d, lx.n_act ? &lx : nullptr, bb, nullptr,
+                     [&](int r, int n, float v, float b, float) { if (r0 + r < T) xres[r * d + n] += v + b; });
         }
         __syncthreads();
         // ---- fc1 (LayerNorm 2 folded, GELU) and fc2 (+ residual)
@@ -477,21 +573,25 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const La
         lora_shrink(cx, lin[2], aset, args.slabs_max, abuf, cx.L.lda, &lx);
         {
             const float* lg = lin[2].ln_g; const float* bb = lin[2].bias;
-            linear16(cx, abuf, cx.L.lda, lin[2].Wt, args.mlp, d, lx.n_act ? &lx : nullptr, [&](int r, int n, float v) {
-                hbuf[r * cx.L.ldh + n] = __float2bfloat16_rn(gelu_exact(stats[r].y * (v - stats[r].x * lg[n]) + bb[n]));
+            linear16(cx, abuf, cx.L.lda, &lin[2].tm_w, 128, 0, args.mlp, d, lx.n_act ? &lx : nullptr, bb, lg, [&](int r, int n, float v, float b, float gsum) {
+                hbuf[r * cx.L.ldh + n] = __float2bfloat16_rn(gelu_exact(stats[r].y * (v - stats[r].x * gsum) + b));
             });
         }
         __syncthreads();
         lora_shrink(cx, lin[3], aset, args.slabs_max, hbuf, cx.L.ldh, &lx);
         {
             const float* bb = lin[3].bias;
-            linear16(cx, hbuf, cx.L.ldh, lin[3].Wt, d, args.mlp, lx.n_act ? &lx : nullptr,
-                     [&](int r, int n, float v) { if (r0 + r < T) xres[r * d + n] += v + bb[n]; });
+            linear16(cx, hbuf, cx.L.ldh, &lin[3].tm_w, 128, 0, d, args.mlp, lx.n_act ? &lx : nullptr, bb, nullptr,
+                     [&](int r, int n, float v, float b, float) { if (r0 + r < T) xres[r * d + n] += v + b; });
         }
         __syncthreads();
     }
 
-    if (rt != 0 || *abort_flag) return;
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);     // copies still in flight land before shared memory goes away
+        return;
+    }
+    if (rt != 0) return;
 
     // ---- heads on the CLS row (row 0 of the frame's first CTA): final LayerNorm, base head, adapter heads
     float* z = reinterpret_cast<float*>(smem + cx.L.region);
