@@ -10,8 +10,10 @@
 // per block is attention: each CTA publishes the keys and values of its rows (two global buffers used in
 // turn), the CTAs of a frame meet at a counter (bounded wait), then each CTA attends from its 16 query rows
 // to all keys of its frame, head by head (the eight warps split the keys and merge their partial softmax
-// results).  Contractions run on mma.sync m16n8k16 (bf16 in, fp32 accumulate): with 16 rows per CTA there is
-// no 128-row tile to give to tcgen05, and the tensor work is a small part of the time anyway.
+// results).  Contractions run on mma.sync m16n8k16 (bf16 in, fp32 accumulate; measured 2048 FLOP per clock
+// per SM on B200, a quarter of the tcgen05 rate): with 16 rows per CTA there is no 128-row tile to give to
+// tcgen05, and the tensor work is a small part of the time anyway.  What bounds a frame is that each of the
+// 13 CTAs streams every weight through one SM's path to L2.
 // LayerNorm uses the folded form the other kernels use: y = rstd (x W' - mean g) + b'.
 #include "common.cuh"
 
@@ -145,7 +147,7 @@ struct LoraExp {               // LoRA expand of the current linear: t (shared m
 // y[16, N] = A[16, K] W + LoRA expand, handed element-wise to epi(row, n, value).  A: bf16 in shared memory
 // with row stride lda; rows [row0, row0 + N) of the [*, K] matrix behind `tm` come through the ring as TMA
 // boxes of [box_rows outputs][64 inputs] (box_rows = 128 for the weights: two n8 tiles per warp; 16 for a
-// LoRA slab of A^T: warp 0 alone).  All threads of the CTA call it; thread 0 issues the copies.
+// LoRA slab of A^T: warp 0 alone).  All threads of the CTA call it; lane 0 of warps 0..2 issues the copies.
 // col0 / col1: optional per-output-column vectors (bias; LayerNorm g or c1 ...); a thread's four values of
 // each are fetched while the last K box is still being multiplied and handed to epi, so that the epilogue's
 // stores never sit between a load and its use.
