@@ -191,8 +191,8 @@ def test_lora_linear_full_size_sampled(k_in, n_out, rank, clustered, epi):
 def test_gelu_epilogue_accuracy():
     """The GELU epilogue against the exact-erf definition: y = gelu(4 x) through an identity-like
     weight, x sweeping [-3, 3] (so the argument spans [-12, 12]); the bf16 result must be within one
-    bf16 step of the exact value plus 3e-5 (the kernel evaluates a fitted logistic form of x Phi(x)
-    whose absolute error stays below 2.6e-5)."""
+    bf16 step of the exact value plus 3e-5 (the kernel evaluates a fitted form x (1/2 + 1/2 tanh(x q(x^2)))
+    of x Phi(x) whose absolute error stays below 2.6e-5, with the hardware's approximate tanh)."""
     import torch
     from paper_2507_14959_b200 import binding
     n, rows = 64, 197 * 3
