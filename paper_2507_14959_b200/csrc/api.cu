@@ -710,10 +710,11 @@ int lat_tiles_per_frame(const pm_handle_s* h) { return (h->tokens + LAT_ROWS - 1
 bool latency_eligible(const pm_handle_s* h, int n_frames) {
     const pm_config& c = h->cfg;
     if (!h->lat_on || c.dtype != 0 || c.d > 384 || c.mlp > 1536 || h->patch_dim > 1536 || c.max_set > 8) return false;
+    if (c.d % 64 || c.mlp % 64 || h->patch_dim % 64 || c.d / c.heads != 64 || c.patch != 16) return false;
     if (h->tokens > 256) return false;               // a head's keys are one TMA box
-    if (h->slabs_max * PM_SLAB * c.max_set > 512) return false;
+    if (h->slabs_max * c.max_set > 8 || c.layers > 64) return false;                  // LoRA slabs of one linear: one ring step
     if ((long long)n_frames * lat_tiles_per_frame(h) > h->n_sms) return false;       // one CTA per SM, all resident
-    return latency_smem_bytes(c.d, c.mlp, h->patch_dim, h->slabs_max * PM_SLAB * c.max_set, h->tokens) <= 227 * 1024;
+    return latency_smem_bytes(c.d, c.mlp, h->patch_dim, h->tokens, c.layers) <= 227 * 1024;
 }
 
 // slots: perm (slot -> frame) or null; set lists: device CSR over slots
@@ -721,22 +722,30 @@ int forward_latency(pm_handle_s* h, const void* frames, int n_frames, const int*
                     float* scores_out, float* base_out, cudaStream_t st) {
     std::string& err = h->err;
     const pm_config& c = h->cfg;
-    auto view = [](const LinearObj& lo) {
+    bool maps_ok = true;
+    auto view = [&](const LinearObj& lo) {
         LatLinear v;
-        v.tm_w = lo.dev.has_tm_half ? lo.dev.tm_w_half : lo.dev.tm_w;      // both fetch [128 rows][64 columns]
-        v.tm_at = lo.dev.tm_at;
+        std::memset(&v, 0, sizeof(v));
         v.Wt = (const bf16*)lo.dev.Wt; v.bias = lo.dev.bias; v.ln_g = lo.dev.ln_g;
         v.At = (const bf16*)lo.dev.lora.At; v.Bt = (const bf16*)lo.dev.lora.Bt; v.c1 = lo.dev.ln_c1; v.c2 = lo.dev.ln_c2;
-        for (int i = 0; i < 8; ++i) v.adapted[i] = 0u;
         for (size_t a = 0; a < lo.adapted.size() && a < 256; ++a) if (lo.adapted[a]) v.adapted[a >> 5] |= 1u << (a & 31);
         if (lo.n_adapted == 0) { v.At = nullptr; v.Bt = nullptr; }
         v.k_in = lo.dev.k_in; v.n_out = lo.dev.n_out;
+        // the kernel's own boxes: half a chunk of outputs, one slab of A^T, a chunk's rows of one slab of B^T
+        maps_ok = maps_ok && tm_encode_2d(&v.tm_w, lo.dev.Wt, v.k_in, v.n_out, (uint64_t)v.k_in * 2, 64, 64, 128);
+        if (v.At) {
+            const uint64_t arena_slabs = (uint64_t)c.max_adapters * h->slabs_max;
+            maps_ok = maps_ok && tm_encode_2d(&v.tm_at, lo.dev.lora.At, v.k_in, arena_slabs * PM_SLAB, (uint64_t)v.k_in * 2, 64, PM_SLAB, 128);
+            maps_ok = maps_ok && tm_encode_2d(&v.tm_bt, lo.dev.lora.Bt, PM_SLAB, arena_slabs * v.n_out, PM_SLAB * 2, PM_SLAB, 128, 32);
+        }
         return v;
     };
     if (h->lat_dirty) {
         std::vector<LatLinear> lv;
         for (const LinearObj& lo : h->lin) lv.push_back(view(lo));
         lv.push_back(view(h->patch));
+        lv.back().At = nullptr; lv.back().Bt = nullptr;         // the patch projection carries no adapter
+        if (!maps_ok) { err = "cuTensorMapEncodeTiled failed (whole-network kernel)"; return PM_ERR_CUDA; }
         CK(h->lat_lin.alloc(lv.size() * sizeof(LatLinear)));
         CK(cudaMemcpy(h->lat_lin.p, lv.data(), lv.size() * sizeof(LatLinear), cudaMemcpyHostToDevice));
         if (!h->lat_kv.p) {

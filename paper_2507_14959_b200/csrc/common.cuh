@@ -207,8 +207,9 @@ struct SmemGrant {
 // ---- whole-network kernel for a handful of frames (latency_kernel.cu)
 // One linear as this kernel sees it (device pointers into the handle's weights and LoRA arenas).
 struct LatLinear {
-    CUtensorMap tm_w;          // W^T [n_out, k_in], boxes of [128 rows][64 columns], 128B swizzle
-    CUtensorMap tm_at;         // A^T arena [max_adapters * RS, k_in], boxes of [16 rows][64 columns]
+    CUtensorMap tm_w;          // W^T [n_out, k_in], boxes of [64 rows][64 columns], 128B swizzle
+    CUtensorMap tm_at;         // A^T arena [max_adapters * RS, k_in], boxes of [16 rows][64 columns], 128B swizzle
+    CUtensorMap tm_bt;         // B^T arena [max_adapters * slabs_max * n_out, 16], boxes of [128 rows][16 columns], 32B swizzle
     const bf16* Wt;            // [n_out, k_in]
     const float* bias;         // [n_out]
     const float* ln_g;         // [n_out] or null (LayerNorm folded into W)
@@ -223,6 +224,7 @@ struct LatLinear {
 struct LatArgs {
     const bf16* frames;        // [F, 3, img, img]
     int n_frames, img, grid, tokens, tiles_pf, d, heads, mlp, layers, n_classes, patch_dim;
+    int ring_slots;            // 16 KB slots of the weight ring (set by the launcher)
     float eps;
     const LatLinear* lin;      // [layers * 4 + 1]: the blocks' linears, then the patch projection
     CUtensorMap tm_kv;         // the exchange buffer as [2 * F * tokens, 2 d], boxes of [tpad rows][64 columns]
@@ -243,8 +245,8 @@ struct LatArgs {
     int* status;
 };
 
-// bytes of dynamic shared memory the kernel needs for this geometry (rs_total = slabs_max * 16 * max_set)
-size_t latency_smem_bytes(int d, int mlp, int patch_dim, int rs_total, int tokens);
+// bytes of dynamic shared memory the kernel takes for this geometry (more than any device has if it cannot run)
+size_t latency_smem_bytes(int d, int mlp, int patch_dim, int tokens, int layers);
 // One launch for the whole forward of a.n_frames frames; a.status is taken from L.  The grid
 // (n_frames * tiles_pf CTAs, one per SM) must be resident at once: a cooperative launch, which fails
 // with an error instead of starting if it cannot be.

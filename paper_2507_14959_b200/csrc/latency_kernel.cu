@@ -4,16 +4,19 @@
 //
 // Everything in a ViT block except attention is local to a token row, so a CTA owns 16 token rows of one
 // frame from the first layer to the last and keeps their residual stream (fp32) and every intermediate in
-// shared memory; the weights stream through a ring of 16 KB shared-memory slots filled by TMA (one
-// [128 outputs x 64 inputs] box per slot, 128B swizzle, several boxes in flight) and are the only thing
-// read from L2 -- every CTA reads all of them, which is what bounds a frame's latency.  The one exchange
-// per block is attention: each CTA publishes the keys and values of its rows (two global buffers used in
-// turn), the CTAs of a frame meet at a counter (bounded wait), then each CTA attends from its 16 query rows
-// to all keys of its frame, head by head (the eight warps split the keys and merge their partial softmax
-// results).  Contractions run on mma.sync m16n8k16 (bf16 in, fp32 accumulate; measured 2048 FLOP per clock
-// per SM on B200, a quarter of the tcgen05 rate): with 16 rows per CTA there is no 128-row tile to give to
-// tcgen05, and the tensor work is a small part of the time anyway.  What bounds a frame is that each of the
-// 13 CTAs streams every weight through one SM's path to L2.
+// shared memory.  What a CTA reads from L2 is static -- weights, LoRA slabs, bias vectors, in an order that
+// is known when the kernel starts -- so one producer thread walks that order and keeps a ring of 16 KB
+// shared-memory slots full by TMA, across the boundaries of linears and blocks, while the eight consumer
+// warps multiply what has landed (full / empty transaction barriers per slot, no CTA-wide barrier in the
+// stream).  Every CTA reads every weight, 13 CTAs per frame.
+// The one exchange per block is attention: each CTA publishes the keys and values of its rows (two global
+// buffers used in turn) as soon as those columns of the qkv product are done, counts itself in at the
+// frame's counter and goes on with the query columns; a second producer thread waits for the counter
+// (bounded) and fetches the heads' keys and values, the next head's while this one is computed.  Each CTA
+// attends from its 16 query rows to all keys of its frame: four warp pairs split the keys, the two warps
+// of a pair split the head dimension, partial softmax results are merged through shared memory.
+// Contractions run on mma.sync m16n8k16 (bf16 in, fp32 accumulate): with 16 rows per CTA there is no
+// 128-row tile to give to tcgen05.
 // LayerNorm uses the folded form the other kernels use: y = rstd (x W' - mean g) + b'.
 #include "common.cuh"
 
@@ -22,13 +25,16 @@
 namespace {
 
 constexpr int LT_ROWS = 16;
-constexpr int LT_THREADS = 256;
-constexpr int LT_WARPS = 8;
-constexpr int LT_GROUP = 3;                // K boxes multiplied between two CTA-wide barriers
-constexpr int LT_SLOTS = 2 * LT_GROUP;     // weight ring: two groups of boxes
-constexpr int LT_BOX_BYTES = 128 * 128;    // [128 output rows][64 bf16 inputs], 128B swizzle
+constexpr int LT_CWARPS = 8;                 // consumer warps
+constexpr int LT_CTHREADS = LT_CWARPS * 32;
+constexpr int LT_THREADS = LT_CTHREADS + 64; // + the weight producer's warp + the key/value producer's warp
+constexpr int LT_SLOT_BYTES = 128 * 128;     // [128 output rows][64 bf16 inputs], 128B swizzle
+constexpr int LT_MAX_SLOTS = 8;
 constexpr int LT_MAX_SET = 8;
+constexpr int LT_MAX_SLABS = 8;              // active LoRA slabs of one linear
 constexpr int LT_HD = 64;
+constexpr int LT_KSPLIT = 4;                 // key ranges of the attention warps
+constexpr int LT_ST = 8;                     // key tiles (8 keys) of one range, at most (256 tokens)
 constexpr long long LT_WAIT_CYCLES = 4000000000ll;
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -54,16 +60,14 @@ __device__ __forceinline__ uint32_t pk_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
 }
-__device__ __forceinline__ void cp16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void bar_expect(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t bar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -76,54 +80,79 @@ __device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* tm, int
                  ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+// untiled copy: both addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(LT_CTHREADS) : "memory"); }
+
 }  // namespace
 
 namespace {
 
 struct LatSmem {               // offsets (bytes) into dynamic shared memory
-    int region, xres, abuf, hbuf, qbuf, tbuf, stats, part, misc, total;
+    int ring, kbuf, vbuf, xres, abuf, qbuf, hbuf, tbuf, stats, colv, slabs, misc, total;
     int lda, ldh, ldq, ldt;    // row strides in bf16 elements
-    int kv_head;               // bytes of one head's keys + values in the region
+    int kv_bytes;              // one head's keys (or values): [tpad rows][128 bytes], and a kilobyte behind them
+    int cv_floats;             // one vector pack: bias[nmax], g[nmax], c1[128], c2[128]
 };
 
-__host__ __device__ inline LatSmem lat_layout(int d, int mlp, int patch_dim, int rs_total, int tokens) {
+__host__ __device__ inline LatSmem lat_layout(int d, int mlp, int patch_dim, int tokens, int layers, int slots) {
     LatSmem s;
     auto up = [](int v) { return (v + 127) & ~127; };
-    s.lda = d + 8; s.ldh = (mlp > patch_dim ? mlp : patch_dim) + 8; s.ldq = d + 8; s.ldt = rs_total + 8;
-    // first (1024-byte aligned, as the 128B swizzle wants): the weight ring, or two heads' keys and values
-    // (each [tpad rows][128 bytes]) -- the next head's land while this one is computed
+    const int wide = mlp > patch_dim ? mlp : patch_dim, nmax = 3 * d > mlp ? 3 * d : mlp;
+    s.lda = d + 8; s.ldh = wide + 8; s.ldq = d + 8; s.ldt = LT_MAX_SLABS * PM_SLAB + 8;
     const int tpad = (tokens + 15) / 16 * 16;
-    s.kv_head = 2 * ((tpad * 128 + 1023) & ~1023);
-    const int wbytes = LT_SLOTS * LT_BOX_BYTES, kvbytes = 2 * s.kv_head;
+    s.kv_bytes = ((tpad * 128 + 1023) & ~1023) + 1024;      // + 1 KB that stays zero behind the values (see the P V loop)
+    s.cv_floats = 2 * nmax + 2 * LT_MAX_SLABS * PM_SLAB;
     int o = 0;
-    s.region = o; o = up(o + (wbytes > kvbytes ? wbytes : kvbytes));
+    s.ring = o; o += slots * LT_SLOT_BYTES;                      // 1024-byte aligned, as the 128B swizzle wants
+    s.kbuf = o; o += s.kv_bytes;
+    s.vbuf = o; o += s.kv_bytes;
     s.xres = o; o = up(o + LT_ROWS * d * 4);
     s.abuf = o; o = up(o + LT_ROWS * s.lda * 2);
-    s.hbuf = o; o = up(o + LT_ROWS * s.ldh * 2);
     s.qbuf = o; o = up(o + LT_ROWS * s.ldq * 2);
+    // the MLP's hidden rows (and the gathered patches); between blocks' MLPs: the attention warps' partial results
+    const int hb = LT_ROWS * s.ldh * 2, pb = LT_KSPLIT * LT_ROWS * (LT_HD + 2) * 4;
+    s.hbuf = o; o = up(o + (hb > pb ? hb : pb));
     s.tbuf = o; o = up(o + LT_ROWS * s.ldt * 2);
     s.stats = o; o = up(o + LT_ROWS * 16);
-    s.part = o; o = up(o + LT_WARPS * LT_ROWS * (LT_HD + 2) * 4);      // partial attention results of the warps
+    s.colv = o; o = up(o + 2 * s.cv_floats * 4);
+    s.slabs = o; o = up(o + layers * 4 * 32);
     s.misc = o; o = up(o + 512);     // the adapter set, abort flag, mbarriers
     s.total = o;
     return s;
 }
 
+struct ActiveSet { int n; int id[LT_MAX_SET]; int slabs[LT_MAX_SET]; float scale[LT_MAX_SET]; };
+// the LoRA slabs one linear applies to this frame: slab i belongs to set member who[i] and is its slab sl[i]
+struct SlabTab { int n; uint8_t who[LT_MAX_SLABS]; uint8_t sl[LT_MAX_SLABS]; int pad[3]; };
+static_assert(sizeof(SlabTab) == 32, "one table entry is 32 bytes");
+static_assert(sizeof(ActiveSet) <= 128, "the adapter set sits in the first 128 bytes of the last region");
+
 struct Ctx {
     uint8_t* sm;
     LatSmem L;
-    int warp, lane, g, t;
-    uint32_t box_no;           // boxes that have gone through the weight ring so far (the same in every thread)
-    uint32_t kv_no;            // head buffers filled so far
+    int warp, lane, g, t, ns;
+    uint32_t slot, phase;      // ring position: the same in every consumer thread (and in the producer)
+    uint32_t li;               // linears done so far (their vector packs alternate between two buffers)
     int* status;
     volatile int* abort_flag;
 };
 
-__device__ __forceinline__ uint32_t ring_bar(const Ctx& cx, int slot) { return s_u32(cx.sm + cx.L.misc + 256) + 8u * slot; }
-__device__ __forceinline__ uint32_t kv_bar(const Ctx& cx, int buf) { return s_u32(cx.sm + cx.L.misc + 256) + 8u * (LT_SLOTS + buf); }
+__device__ __forceinline__ uint32_t bars(const Ctx& cx) { return s_u32(cx.sm + cx.L.misc + 256); }
+__device__ __forceinline__ uint32_t full_bar(const Ctx& cx, uint32_t i) { return bars(cx) + 8u * i; }
+__device__ __forceinline__ uint32_t empty_bar(const Ctx& cx, uint32_t i) { return bars(cx) + 64u + 8u * i; }
+__device__ __forceinline__ uint32_t kfull_bar(const Ctx& cx) { return bars(cx) + 128u; }
+__device__ __forceinline__ uint32_t kempty_bar(const Ctx& cx) { return bars(cx) + 136u; }
+__device__ __forceinline__ uint32_t vfull_bar(const Ctx& cx) { return bars(cx) + 144u; }
+__device__ __forceinline__ uint32_t vempty_bar(const Ctx& cx) { return bars(cx) + 152u; }
+__device__ __forceinline__ uint32_t cfull_bar(const Ctx& cx, uint32_t b) { return bars(cx) + 160u + 8u * b; }
+__device__ __forceinline__ uint32_t cempty_bar(const Ctx& cx, uint32_t b) { return bars(cx) + 176u + 8u * b; }
 
-// Bounded wait on a transaction barrier (every thread of the CTA may call it).  Once a wait has run out
-// the CTA is aborting: later waits return at once and the results are meaningless (the status word says so).
+// Bounded wait on a barrier.  Once a wait has run out the CTA is aborting: later waits return at once and
+// the results are meaningless (the status word says so).
 __device__ __forceinline__ void bar_wait(const Ctx& cx, uint32_t bar, uint32_t parity) {
     if (bar_try(bar, parity)) return;
     const long long t0 = clock64();
@@ -136,174 +165,232 @@ __device__ __forceinline__ void bar_wait(const Ctx& cx, uint32_t bar, uint32_t p
         }
     }
 }
+__device__ __forceinline__ void ring_advance(Ctx& cx) {
+    if (++cx.slot == (uint32_t)cx.ns) { cx.slot = 0; cx.phase ^= 1u; }
+}
+// consumer side of one ring step: wait until the slot's copies have landed / hand the slot back
+__device__ __forceinline__ uint32_t step_acquire(Ctx& cx) {
+    bar_wait(cx, full_bar(cx, cx.slot), cx.phase);
+    return s_u32(cx.sm + cx.L.ring) + cx.slot * LT_SLOT_BYTES;
+}
+__device__ __forceinline__ void step_release(Ctx& cx) {
+    __syncwarp();
+    if (cx.lane == 0) bar_arrive(empty_bar(cx, cx.slot));
+    ring_advance(cx);
+}
+// producer side: wait until the eight consumer warps have handed the slot back (first lap: at once)
+__device__ __forceinline__ uint32_t step_claim(Ctx& cx, uint32_t bytes) {
+    bar_wait(cx, empty_bar(cx, cx.slot), cx.phase ^ 1u);
+    bar_expect(full_bar(cx, cx.slot), bytes);
+    return s_u32(cx.sm + cx.L.ring) + cx.slot * LT_SLOT_BYTES;
+}
 
-struct LoraExp {               // LoRA expand of the current linear: t (shared memory) times B slabs (global)
-    int n_act;
-    int adapter[LT_MAX_SET], slabs[LT_MAX_SET];
-    const bf16* Bt;
-    int slabs_max, rs;         // rs: columns of t per adapter
-};
+// What the weight producer sends for one linear, in this order (the consumers take it in the same order):
+//   the vector pack (bias, g, c1, c2) into the linear's pack buffer;
+//   LoRA shrink, if any slab is active: K/64 steps, each the [16 rows][64] boxes of A^T of all active slabs;
+//   for each chunk of 128 outputs, starting at first_chunk and wrapping round: K/64 steps of W^T
+//   ([64 rows][64] boxes, two per full chunk), then the chunk's rows of the active slabs' B^T
+//   ([128 rows][16] boxes, four per step).
+__device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st, const ActiveSet& as, int rs, int slabs_max,
+                               int first_chunk) {
+    const int N = lin->n_out, K = lin->k_in, k_boxes = K >> 6, n_chunks = (N + 127) >> 7, n_sl = st.n;
+    const bool folded = lin->ln_g != nullptr;
+    {
+        const uint32_t b = cx.li & 1u, use = cx.li >> 1;
+        bar_wait(cx, cempty_bar(cx, b), (use & 1u) ^ 1u);
+        const uint32_t dst = s_u32(cx.sm + cx.L.colv) + b * (uint32_t)cx.L.cv_floats * 4u;
+        const uint32_t vb = (uint32_t)N * 4u;
+        const uint32_t bytes = vb + (folded ? vb : 0u) + (folded ? (uint32_t)n_sl * 128u : 0u);
+        bar_expect(cfull_bar(cx, b), bytes);
+        bulk_copy(dst, lin->bias, vb, cfull_bar(cx, b));
+        if (folded) {
+            bulk_copy(dst + vb, lin->ln_g, vb, cfull_bar(cx, b));
+            for (int i = 0; i < n_sl; ++i) {
+                const int arow = as.id[st.who[i]] * rs + st.sl[i] * PM_SLAB;
+                bulk_copy(dst + 2u * vb + i * 64u, lin->c1 + arow, 64u, cfull_bar(cx, b));
+                bulk_copy(dst + 2u * vb + LT_MAX_SLABS * 64u + i * 64u, lin->c2 + arow, 64u, cfull_bar(cx, b));
+            }
+        }
+        ++cx.li;
+    }
+    if (n_sl) {
+        for (int kb = 0; kb < k_boxes && !*cx.abort_flag; ++kb) {
+            const uint32_t dst = step_claim(cx, (uint32_t)n_sl * 2048u);
+            for (int i = 0; i < n_sl; ++i)
+                tma_box(dst + i * 2048u, &lin->tm_at, kb * 64, as.id[st.who[i]] * rs + st.sl[i] * PM_SLAB, full_bar(cx, cx.slot));
+            ring_advance(cx);
+        }
+    }
+    for (int ci = 0; ci < n_chunks; ++ci) {
+        int nc = first_chunk + ci;
+        if (nc >= n_chunks) nc -= n_chunks;
+        const int rows = min(128, N - nc * 128);
+        for (int kb = 0; kb < k_boxes && !*cx.abort_flag; ++kb) {
+            const uint32_t dst = step_claim(cx, (uint32_t)rows * 128u);
+            for (int hf = 0; hf * 64 < rows; ++hf)
+                tma_box(dst + hf * 8192u, &lin->tm_w, kb * 64, nc * 128 + hf * 64, full_bar(cx, cx.slot));
+            ring_advance(cx);
+        }
+        for (int s0 = 0; s0 < n_sl && !*cx.abort_flag; s0 += 4) {
+            const int cnt = min(4, n_sl - s0);
+            const uint32_t dst = step_claim(cx, (uint32_t)cnt * 4096u);
+            for (int j = 0; j < cnt; ++j) {
+                const int i = s0 + j;
+                tma_box(dst + j * 4096u, &lin->tm_bt, 0, (as.id[st.who[i]] * slabs_max + st.sl[i]) * N + nc * 128, full_bar(cx, cx.slot));
+            }
+            ring_advance(cx);
+        }
+    }
+}
 
-// y[16, N] = A[16, K] W + LoRA expand, handed element-wise to epi(row, n, value).  A: bf16 in shared memory
-// with row stride lda; rows [row0, row0 + N) of the [*, K] matrix behind `tm` come through the ring as TMA
-// boxes of [box_rows outputs][64 inputs] (box_rows = 128 for the weights: two n8 tiles per warp; 16 for a
-// LoRA slab of A^T: warp 0 alone).  All threads of the CTA call it; lane 0 of warps 0..2 issues the copies.
-// col0 / col1: optional per-output-column vectors (bias; LayerNorm g or c1 ...); a thread's four values of
-// each are fetched while the last K box is still being multiplied and handed to epi, so that the epilogue's
-// stores never sit between a load and its use.
+// one ring step of weights ([rows][64 inputs], this warp's 16 rows) against 64 columns of A (bf16, shared memory)
+__device__ __forceinline__ void mma_step(Ctx& cx, uint32_t a_row, bool active, float (&acc)[2][2][4]) {
+    const uint32_t box = step_acquire(cx);
+    if (active) {
+        const int mi = cx.lane >> 3;
+        const int r = cx.warp * 16 + (mi >> 1) * 8 + (cx.lane & 7);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            uint32_t a[4], b0, b1, b2, b3;
+            ldsm4(a_row + ks * 32, a[0], a[1], a[2], a[3]);
+            const int c = ks * 2 + (mi & 1);
+            ldsm4(box + r * 128 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
+            mma16816(acc[0][ks & 1], a, b0, b1);
+            mma16816(acc[1][ks & 1], a, b2, b3);
+        }
+    }
+    step_release(cx);
+}
+__device__ __forceinline__ void acc_zero(float (&acc)[2][2][4]) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) acc[q][h][0] = acc[q][h][1] = acc[q][h][2] = acc[q][h][3] = 0.f;
+}
+
+// The consumers' side of a linear's chunks: y[16, N] = A[16, K] W + t B, handed to epi(row, n, y[n], y[n + 1])
+// for even n.  After the chunk `publish_after` (if >= 0) the CTA counts itself in at `counter`: everything
+// its threads stored to global memory up to there is visible to whoever sees the count.
 template <typename Epi>
-__device__ void linear16(Ctx& cx, const bf16* A, int lda, const CUtensorMap* tm, int box_rows, int row0, int N, int K,
-                         const LoraExp* lx, const float* col0, const float* col1, Epi epi) {
-    const int n_chunks = (N + box_rows - 1) / box_rows, k_boxes = K >> 6;
-    // boxes go through the ring in groups of up to LT_GROUP consecutive K boxes of one chunk of outputs: one
-    // CTA-wide barrier per group, and while a group is multiplied the next one is on its way
-    const int gpc = (k_boxes + LT_GROUP - 1) / LT_GROUP, n_groups = n_chunks * gpc;
-    const uint32_t a_base = s_u32(A), ring = s_u32(cx.sm + cx.L.region), t_base = s_u32(cx.sm + cx.L.tbuf);
-    const int lane = cx.lane, warp = cx.warp;
-    uint32_t issued = cx.box_no;                      // number of the next box to issue (the same in every thread)
-    auto issue_group = [&](int g) {
-        const int nc = g / gpc, kb0 = (g % gpc) * LT_GROUP, nb = min(LT_GROUP, k_boxes - kb0);
-        if (lane == 0 && warp < nb) {                 // box j of the group: lane 0 of warp j
-            const int slot = (int)((issued + (uint32_t)warp) % LT_SLOTS);
-            bar_expect(ring_bar(cx, slot), (uint32_t)box_rows * 128u);
-            tma_box(ring + slot * LT_BOX_BYTES, tm, (kb0 + warp) * 64, row0 + nc * box_rows, ring_bar(cx, slot));
-        }
-        issued += (uint32_t)nb;
-    };
-    issue_group(0);
-    float acc[2][4];
-    const int row16 = warp * 16;                   // this warp's rows of a box
-    const int mi = lane >> 3;
-    const int r = row16 + (mi >> 1) * 8 + (lane & 7);
-    for (int g = 0; g < n_groups; ++g) {
-        // the slots freed by the previous group (everyone is past its closing barrier) take the next one
-        if (g + 1 < n_groups) issue_group(g + 1);
-        const int nc = g / gpc, kb0 = (g % gpc) * LT_GROUP, nb = min(LT_GROUP, k_boxes - kb0);
-        const bool last = kb0 + nb == k_boxes;
-        if (kb0 == 0) {
-#pragma unroll
-            for (int q = 0; q < 2; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
-        }
-        const int n16 = nc * box_rows + row16;
-        const bool active = row16 < box_rows && n16 < N;
-        float cv0[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, cv1[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-        if (active && last) {
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int n = n16 + q * 8 + 2 * cx.t;
-                if (n16 + q * 8 < N) {
-                    if (col0) { const float2 v = __ldg(reinterpret_cast<const float2*>(col0 + n)); cv0[q][0] = v.x; cv0[q][1] = v.y; }
-                    if (col1) { const float2 v = __ldg(reinterpret_cast<const float2*>(col1 + n)); cv1[q][0] = v.x; cv1[q][1] = v.y; }
-                }
-            }
-        }
-        for (int j = 0; j < nb; ++j) {
-            const uint32_t no = cx.box_no + (uint32_t)j;
-            const int slot = (int)(no % LT_SLOTS);
-            bar_wait(cx, ring_bar(cx, slot), (no / LT_SLOTS) & 1u);
+__device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl, int first_chunk, int publish_after,
+                         unsigned int* counter, Epi epi) {
+    const int k_boxes = K >> 6, n_chunks = (N + 127) >> 7;
+    const uint32_t a_base = s_u32(A) + ((cx.lane & 15) * lda + (cx.lane >> 4) * 8) * 2;
+    const uint32_t t_row = s_u32(cx.sm + cx.L.tbuf) + ((cx.lane & 15) * cx.L.ldt + (cx.lane >> 4) * 8) * 2;
+    for (int ci = 0; ci < n_chunks; ++ci) {
+        int nc = first_chunk + ci;
+        if (nc >= n_chunks) nc -= n_chunks;
+        const int rows = min(128, N - nc * 128);
+        const bool active = cx.warp * 16 < rows;
+        float acc[2][2][4];
+        acc_zero(acc);
+        for (int kb = 0; kb < k_boxes; ++kb) mma_step(cx, a_base + kb * 128, active, acc);
+        for (int s0 = 0; s0 < n_sl; s0 += 4) {
+            const uint32_t box = step_acquire(cx);
             if (active) {
-                const uint32_t a_row = a_base + ((lane & 15) * lda + (kb0 + j) * 64 + (lane >> 4) * 8) * 2;
-                const uint32_t box = ring + slot * LT_BOX_BYTES;
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
+                // B^T rows are 32 bytes (16 ranks), 32B swizzle: the 16-byte half c of row n sits at c ^ ((n >> 2) & 1)
+                const int n = cx.warp * 16 + ((cx.lane >> 4) & 1) * 8 + (cx.lane & 7), c = (cx.lane >> 3) & 1;
+                const uint32_t b_row = box + n * 32 + ((c ^ ((n >> 2) & 1)) << 4);
+                const int cnt = min(4, n_sl - s0);
+                for (int j = 0; j < cnt; ++j) {
                     uint32_t a[4], b0, b1, b2, b3;
-                    ldsm4(a_row + ks * 32, a[0], a[1], a[2], a[3]);
-                    const int c = ks * 2 + (mi & 1);
-                    ldsm4(box + r * 128 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
-                    mma16816(acc[0], a, b0, b1);
-                    mma16816(acc[1], a, b2, b3);
+                    ldsm4(t_row + (s0 + j) * 32, a[0], a[1], a[2], a[3]);
+                    ldsm4(b_row + j * 4096, b0, b1, b2, b3);
+                    mma16816(acc[0][j & 1], a, b0, b1);
+                    mma16816(acc[1][j & 1], a, b2, b3);
                 }
             }
+            step_release(cx);
         }
-        cx.box_no += (uint32_t)nb;
-        if (active && last) {
+        if (active) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                const int n8 = n16 + q * 8;
-                if (n8 >= N) break;
-                if (lx) {
-                    for (int p = 0; p < lx->n_act; ++p)
-                        for (int sl = 0; sl < lx->slabs[p]; ++sl) {
-                            uint32_t a[4];
-                            ldsm4(t_base + ((lane & 15) * cx.L.ldt + p * lx->rs + sl * 16 + (lane >> 4) * 8) * 2, a[0], a[1], a[2], a[3]);
-                            const bf16* bp = lx->Bt + (((size_t)(lx->adapter[p] * lx->slabs_max + sl) * N) + n8 + cx.g) * PM_SLAB;
-                            const uint32_t b0 = __ldg(reinterpret_cast<const unsigned int*>(bp + 2 * cx.t));
-                            const uint32_t b1 = __ldg(reinterpret_cast<const unsigned int*>(bp + 2 * cx.t + 8));
-                            mma16816(acc[q], a, b0, b1);
-                        }
-                }
-                const int n = n8 + 2 * cx.t;
-                epi(cx.g, n, acc[q][0], cv0[q][0], cv1[q][0]); epi(cx.g, n + 1, acc[q][1], cv0[q][1], cv1[q][1]);
-                epi(cx.g + 8, n, acc[q][2], cv0[q][0], cv1[q][0]); epi(cx.g + 8, n + 1, acc[q][3], cv0[q][1], cv1[q][1]);
+                const int n = nc * 128 + cx.warp * 16 + q * 8 + 2 * cx.t;
+                epi(cx.g, n, acc[q][0][0] + acc[q][1][0], acc[q][0][1] + acc[q][1][1]);
+                epi(cx.g + 8, n, acc[q][0][2] + acc[q][1][2], acc[q][0][3] + acc[q][1][3]);
             }
         }
-        __syncthreads();          // the group's slots are refilled by the next iteration's copies
+        if (nc == publish_after) {
+            consumer_sync();
+            if (threadIdx.x == 0) {
+                // the stores were ordinary ones and are fetched by TMA on the other side: order the two proxies as well
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                atomicAdd(counter, 1u);
+            }
+        }
+    }
+}
+
+// The consumers' side of a linear's shrink steps: warp i < n_sl multiplies the rows by slab i of A^T and
+// hands epi(row, i, j, v[j], v[j + 1]) its 16 x 16 result (even j).
+template <typename Epi>
+__device__ void shrink16(Ctx& cx, const bf16* A, int lda, int K, int n_sl, Epi epi) {
+    const int k_boxes = K >> 6;
+    const uint32_t a_base = s_u32(A) + ((cx.lane & 15) * lda + (cx.lane >> 4) * 8) * 2;
+    const bool active = cx.warp < n_sl;
+    float acc[2][2][4];
+    acc_zero(acc);
+    for (int kb = 0; kb < k_boxes; ++kb) mma_step(cx, a_base + kb * 128, active, acc);
+    if (active) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int j = q * 8 + 2 * cx.t;
+            epi(cx.g, cx.warp, j, acc[q][0][0] + acc[q][1][0], acc[q][0][1] + acc[q][1][1]);
+            epi(cx.g + 8, cx.warp, j, acc[q][0][2] + acc[q][1][2], acc[q][0][3] + acc[q][1][3]);
+        }
     }
 }
 
 __device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
 
-// abuf <- bf16(xres); stats[r] = (mean, rstd, 1/rstd) of the rounded row (what the tensor cores multiply)
+// abuf <- bf16(xres); stats[r] = (mean, rstd, 1/rstd) of the rounded row (what the tensor cores multiply).
+// A warp takes two rows at once (two independent reduction chains); d is a multiple of 64, at most 384.
 __device__ void round_rows_and_stats(Ctx& cx, int d, float eps) {
     const float* x = reinterpret_cast<const float*>(cx.sm + cx.L.xres);
     bf16* a = reinterpret_cast<bf16*>(cx.sm + cx.L.abuf);
     float4* st = reinterpret_cast<float4*>(cx.sm + cx.L.stats);
-    for (int r = cx.warp; r < LT_ROWS; r += LT_WARPS) {
-        float v[12];                                        // d <= 384
-        float sum = 0.f;
+    const int n2 = d >> 6;                                  // float2 per lane and row
+    for (int r = 2 * cx.warp; r < LT_ROWS; r += 2 * LT_CWARPS) {
+        float2 v[2][6];
+        float sum[2] = {0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < 12; ++i) {
-            const int c = cx.lane + 32 * i;
-            v[i] = 0.f;
-            if (c < d) {
-                const bf16 h = __float2bfloat16_rn(x[r * d + c]);
-                a[r * cx.L.lda + c] = h;
-                v[i] = __bfloat162float(h);
-                sum += v[i];
+        for (int q = 0; q < 2; ++q)
+#pragma unroll
+            for (int i = 0; i < 6; ++i) {
+                v[q][i] = make_float2(0.f, 0.f);
+                if (i < n2) {
+                    const int c = 2 * cx.lane + 64 * i;
+                    const float2 f = *reinterpret_cast<const float2*>(x + (r + q) * d + c);
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(f.x, f.y);
+                    *reinterpret_cast<__nv_bfloat162*>(a + (r + q) * cx.L.lda + c) = h;
+                    v[q][i] = __bfloat1622float2(h);
+                    sum[q] += v[q][i].x + v[q][i].y;
+                }
             }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            sum[0] += __shfl_xor_sync(0xFFFFFFFFu, sum[0], o);
+            sum[1] += __shfl_xor_sync(0xFFFFFFFFu, sum[1], o);
         }
+        const float inv_d = 1.f / (float)d;
+        const float mean[2] = {sum[0] * inv_d, sum[1] * inv_d};
+        float sq[2] = {0.f, 0.f};
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-        const float mean = sum / (float)d;
-        float sq = 0.f;
+        for (int q = 0; q < 2; ++q)
 #pragma unroll
-        for (int i = 0; i < 12; ++i) if (cx.lane + 32 * i < d) { const float t = v[i] - mean; sq += t * t; }
+            for (int i = 0; i < 6; ++i)
+                if (i < n2) { const float t0 = v[q][i].x - mean[q], t1 = v[q][i].y - mean[q]; sq[q] += t0 * t0 + t1 * t1; }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
-        const float rstd = rsqrtf(sq / (float)d + eps);
-        if (cx.lane == 0) st[r] = make_float4(mean, rstd, 1.f / rstd, 0.f);
+        for (int o = 16; o > 0; o >>= 1) {
+            sq[0] += __shfl_xor_sync(0xFFFFFFFFu, sq[0], o);
+            sq[1] += __shfl_xor_sync(0xFFFFFFFFu, sq[1], o);
+        }
+        if (cx.lane < 2) {
+            const float rstd = rsqrtf((cx.lane ? sq[1] : sq[0]) * inv_d + eps);
+            st[r + cx.lane] = make_float4(cx.lane ? mean[1] : mean[0], rstd, 1.f / rstd, 0.f);
+        }
     }
-}
-
-struct ActiveSet { int n; int id[LT_MAX_SET]; int slabs[LT_MAX_SET]; float scale[LT_MAX_SET]; };
-
-// LoRA shrink for the adapters of `as` that touch `lin`: t[r][p * rs + j] (bf16) = s_a (x A_a) (folded
-// linears: s_a ((x A' - mean c1) + c2 / rstd), the fused accumulator being scaled by rstd afterwards).
-// Returns the expand description (adapters in ascending id).
-__device__ void lora_shrink(Ctx& cx, const LatLinear& lin, const ActiveSet& as, int slabs_max, const bf16* A, int lda,
-                            LoraExp* lx) {
-    lx->n_act = 0; lx->Bt = lin.Bt; lx->slabs_max = slabs_max; lx->rs = slabs_max * PM_SLAB;
-    if (!lin.At) return;
-    const float4* st = reinterpret_cast<const float4*>(cx.sm + cx.L.stats);
-    bf16* tb = reinterpret_cast<bf16*>(cx.sm + cx.L.tbuf);
-    for (int i = 0; i < as.n; ++i) {
-        const int a = as.id[i];
-        if (!((lin.adapted[a >> 5] >> (a & 31)) & 1u)) continue;
-        const int p = lx->n_act++;
-        lx->adapter[p] = a; lx->slabs[p] = as.slabs[i];
-        const int rs_a = as.slabs[i] * PM_SLAB;
-        const float sc = as.scale[i];
-        const float* c1 = lin.c1 ? lin.c1 + (size_t)a * lx->rs : nullptr;
-        const float* c2 = lin.c2 ? lin.c2 + (size_t)a * lx->rs : nullptr;
-        const bool folded = lin.ln_g != nullptr;
-        const int ldt = cx.L.ldt, col0 = p * lx->rs;
-        linear16(cx, A, lda, &lin.tm_at, PM_SLAB, a * lx->rs, rs_a, lin.k_in, nullptr, folded ? c1 : nullptr, folded ? c2 : nullptr,
-                 [&](int r, int j, float v, float c1j, float c2j) {
-                     if (folded) v = (v - st[r].x * c1j) + c2j * st[r].z;
-                     tb[r * ldt + col0 + j] = __float2bfloat16_rn(v * sc);
-                 });
-    }
-    __syncthreads();
 }
 
 __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __grid_constant__ LatArgs args) {
@@ -314,22 +401,29 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
     }
     Ctx cx;
     cx.sm = smem;
-    cx.L = lat_layout(args.d, args.mlp, args.patch_dim, args.slabs_max * PM_SLAB * args.max_set, args.tokens);
+    cx.L = lat_layout(args.d, args.mlp, args.patch_dim, args.tokens, args.layers, args.ring_slots);
+    cx.ns = args.ring_slots;
     cx.warp = threadIdx.x >> 5; cx.lane = threadIdx.x & 31; cx.g = cx.lane >> 2; cx.t = cx.lane & 3;
     const int f = blockIdx.x / args.tiles_pf, rt = blockIdx.x % args.tiles_pf;     // slot, row tile
     const int frame = args.perm ? args.perm[f] : f;                                  // input / output row
     const int T = args.tokens, d = args.d, r0 = rt * LT_ROWS;
     const int tpad = (T + 15) / 16 * 16;
+    const int rs = args.slabs_max * PM_SLAB;
     float* xres = reinterpret_cast<float*>(smem + cx.L.xres);
     bf16* abuf = reinterpret_cast<bf16*>(smem + cx.L.abuf);
     bf16* hbuf = reinterpret_cast<bf16*>(smem + cx.L.hbuf);
     bf16* qbuf = reinterpret_cast<bf16*>(smem + cx.L.qbuf);
+    bf16* tbuf = reinterpret_cast<bf16*>(smem + cx.L.tbuf);
     const float4* stats = reinterpret_cast<const float4*>(smem + cx.L.stats);
     ActiveSet* as = reinterpret_cast<ActiveSet*>(smem + cx.L.misc);
+    SlabTab* slabtab = reinterpret_cast<SlabTab*>(smem + cx.L.slabs);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + cx.L.misc + 192);
-    cx.box_no = 0; cx.kv_no = 0; cx.status = args.status; cx.abort_flag = abort_flag;
+    cx.slot = 0; cx.phase = 0; cx.li = 0; cx.status = args.status; cx.abort_flag = abort_flag;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < LT_SLOTS + 2; ++i) bar_init(ring_bar(cx, i), 1);
+        for (int i = 0; i < LT_MAX_SLOTS; ++i) { bar_init(full_bar(cx, i), 1); bar_init(empty_bar(cx, i), LT_CWARPS); }
+        bar_init(kfull_bar(cx), 1); bar_init(kempty_bar(cx), LT_CWARPS);
+        bar_init(vfull_bar(cx), 1); bar_init(vempty_bar(cx), LT_CWARPS);
+        for (int b = 0; b < 2; ++b) { bar_init(cfull_bar(cx, b), 1); bar_init(cempty_bar(cx, b), LT_CWARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -362,11 +456,75 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             as->scale[i] = args.scale[as->id[i]];
         }
     }
+    __syncthreads();
+    // ---- per linear: the slabs of the set's adapters that touch it (adapters in ascending id; at most
+    // LT_MAX_SLABS slabs, which the host checks against max_set * slabs_max)
+    if ((int)threadIdx.x < args.layers * 4) {
+        const LatLinear& lin = args.lin[threadIdx.x];
+        SlabTab st;
+        st.n = 0;
+        if (lin.At) {
+            for (int i = 0; i < as->n; ++i) {
+                const int a = as->id[i];
+                if (!((lin.adapted[a >> 5] >> (a & 31)) & 1u)) continue;
+                for (int s = 0; s < as->slabs[i] && st.n < LT_MAX_SLABS; ++s) { st.who[st.n] = (uint8_t)i; st.sl[st.n] = (uint8_t)s; ++st.n; }
+            }
+        }
+        slabtab[threadIdx.x] = st;
+    }
+    __syncthreads();
+    // qkv: the chunks that hold key and value columns come first; after the last chunk the frame's other
+    // CTAs may fetch them, and the chunks of query columns alone follow
+    const int qkv_chunks = (3 * d + 127) >> 7;
+    const int qkv_first = qkv_chunks > 1 ? d >> 7 : 0, qkv_last = qkv_chunks - 1;
+
+    // ---- the weight producer: one thread, the whole network's static operands in consumption order
+    if (cx.warp == LT_CWARPS) {
+        if (cx.lane != 0) return;
+        SlabTab none;
+        none.n = 0;
+        produce_linear(cx, args.lin + (size_t)args.layers * 4, none, *as, rs, args.slabs_max, 0);
+        for (int l = 0; l < args.layers && !*abort_flag; ++l)
+            for (int j = 0; j < 4; ++j)
+                produce_linear(cx, args.lin + (size_t)l * 4 + j, slabtab[l * 4 + j], *as, rs, args.slabs_max, j == 0 ? qkv_first : 0);
+        return;
+    }
+    // ---- the key/value producer: per block, wait for the frame's CTAs, then one head after the other
+    if (cx.warp == LT_CWARPS + 1) {
+        if (cx.lane != 0) return;
+        uint32_t idx = 0;
+        for (int l = 0; l < args.layers && !*abort_flag; ++l) {
+            const unsigned int want = (unsigned int)args.tiles_pf * (unsigned int)(l + 1);
+            const long long t0 = clock64();
+            unsigned int seen;
+            do {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(args.bar + f) : "memory");
+                if (seen < want && (*abort_flag || clock64() - t0 > LT_WAIT_CYCLES)) {
+                    if (!*abort_flag) { *abort_flag = 1; atomicCAS(args.status, 0, (int)PM_ERR_TIMEOUT); }
+                    break;
+                }
+            } while (seen < want);
+            if (*abort_flag) break;
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            const int kv_row0 = ((l & 1) * args.n_frames + f) * T;
+            for (int h = 0; h < args.heads; ++h, ++idx) {
+                bar_wait(cx, kempty_bar(cx), (idx & 1u) ^ 1u);
+                bar_expect(kfull_bar(cx), (uint32_t)tpad * 128u);
+                tma_box(s_u32(smem + cx.L.kbuf), &args.tm_kv, h * LT_HD, kv_row0, kfull_bar(cx));
+                bar_wait(cx, vempty_bar(cx), (idx & 1u) ^ 1u);
+                bar_expect(vfull_bar(cx), (uint32_t)tpad * 128u);
+                tma_box(s_u32(smem + cx.L.vbuf), &args.tm_kv, d + h * LT_HD, kv_row0, vfull_bar(cx));
+            }
+        }
+        return;
+    }
+
+    // ================================ consumers (256 threads) ================================
     // ---- patch gather: hbuf[r][c*P*P + py*P + px] = frame[c][gy*P + py][gx*P + px] of token r0 + r (token 0 = CLS)
     {
         const int P = 16, per_row = args.patch_dim / 8;
         const bf16* fr = args.frames + (size_t)frame * 3 * args.img * args.img;
-        for (int i = threadIdx.x; i < LT_ROWS * per_row; i += LT_THREADS) {
+        for (int i = threadIdx.x; i < LT_ROWS * per_row; i += LT_CTHREADS) {
             const int r = i / per_row, ch = i % per_row, tok = r0 + r;
             uint4 v = make_uint4(0, 0, 0, 0);
             if (tok >= 1 && tok < T) {
@@ -377,216 +535,239 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             *reinterpret_cast<uint4*>(hbuf + r * cx.L.ldh + ch * 8) = v;
         }
     }
-    __syncthreads();
-    const ActiveSet aset = *as;
-    // ---- patch projection + positions; the CLS row
-    const LatLinear* patch = args.lin + (size_t)args.layers * 4;
-    const float* patch_bias = patch->bias;
-    linear16(cx, hbuf, cx.L.ldh, &patch->tm_w, 128, 0, d, args.patch_dim, nullptr, patch_bias, nullptr, [&](int r, int n, float v, float b, float) {
-        const int tok = r0 + r;
-        float out = 0.f;
-        if (tok == 0) out = args.cls[n] + args.pos[n];
-        else if (tok < T) out = v + b + args.pos[(size_t)tok * d + n];
-        xres[r * d + n] = out;                              // rows past the frame stay zero
-    });
-    __syncthreads();
+    // the kilobyte behind the values is read as keys whose probabilities are zero: it has to hold finite numbers
+    for (int i = threadIdx.x; i < 256; i += LT_CTHREADS)
+        reinterpret_cast<uint32_t*>(smem + cx.L.vbuf + cx.L.kv_bytes - 1024)[i] = 0u;
+    consumer_sync();
 
-    LoraExp lx;
+    // the vector pack of the linear the consumers are at: wait for it / hand its buffer back
+    auto pack_acquire = [&]() -> const float* {
+        bar_wait(cx, cfull_bar(cx, cx.li & 1u), (cx.li >> 1) & 1u);
+        return reinterpret_cast<const float*>(smem + cx.L.colv) + (cx.li & 1u) * cx.L.cv_floats;
+    };
+    auto pack_release = [&]() {
+        __syncwarp();
+        if (cx.lane == 0) bar_arrive(cempty_bar(cx, cx.li & 1u));
+        ++cx.li;
+    };
+    // ---- patch projection + positions; the CLS row
+    {
+        const float* cv = pack_acquire();
+        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, 0, -1, nullptr, [&](int r, int n, float v0, float v1) {
+            const int tok = r0 + r;
+            float2 out = make_float2(0.f, 0.f);                     // rows past the frame stay zero
+            if (tok < T) {
+                const float2 p = *reinterpret_cast<const float2*>(args.pos + (size_t)tok * d + n);
+                if (tok == 0) out = make_float2(args.cls[n] + p.x, args.cls[n + 1] + p.y);
+                else out = make_float2(v0 + cv[n] + p.x, v1 + cv[n + 1] + p.y);
+            }
+            *reinterpret_cast<float2*>(xres + r * d + n) = out;
+        });
+        pack_release();
+    }
+    consumer_sync();
+
+    // LoRA shrink of a linear with slab table `st` on the rows A: t[r][16 i + j] (bf16) = s_a (x A_a)
+    // (folded linears: s_a ((x A' - mean c1) + c2 / rstd), the fused accumulator being scaled by rstd afterwards)
+    auto shrink = [&](const SlabTab& st, const bf16* A, int lda, int K, int N, bool folded, const float* cv) {
+        if (!st.n) return;
+        shrink16(cx, A, lda, K, st.n, [&](int r, int i, int j, float v0, float v1) {
+            if (folded) {
+                const float* c1 = cv + 2 * N + i * PM_SLAB + j;
+                const float* c2 = c1 + LT_MAX_SLABS * PM_SLAB;
+                v0 = (v0 - stats[r].x * c1[0]) + c2[0] * stats[r].z;
+                v1 = (v1 - stats[r].x * c1[1]) + c2[1] * stats[r].z;
+            }
+            const float sc = as->scale[st.who[i]];
+            *reinterpret_cast<uint32_t*>(tbuf + r * cx.L.ldt + i * PM_SLAB + j) = pk_bf16(v0 * sc, v1 * sc);
+        });
+        consumer_sync();
+    };
+    auto residual = [&](const float* cv) {
+        return [=](int r, int n, float v0, float v1) {
+            if (r0 + r < T) {
+                float2* x = reinterpret_cast<float2*>(xres + r * d + n);
+                *x = make_float2(x->x + v0 + cv[n], x->y + v1 + cv[n + 1]);
+            }
+        };
+    };
+
     const float att_scale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
+    uint32_t head_no = 0;                                    // heads attended so far (all blocks)
     for (int l = 0; l < args.layers; ++l) {
-        const LatLinear* lin = args.lin + (size_t)l * 4;
+        const SlabTab* st = slabtab + l * 4;
         bf16* kvb = args.kv + (size_t)(l & 1) * args.n_frames * T * 2 * d + (size_t)f * T * 2 * d;
         // ---- qkv (LayerNorm 1 folded): q stays here, k and v go to the frame's exchange buffer
         round_rows_and_stats(cx, d, args.eps);
-        __syncthreads();
-        lora_shrink(cx, lin[0], aset, args.slabs_max, abuf, cx.L.lda, &lx);
+        consumer_sync();
         {
-            const float* lg = lin[0].ln_g; const float* bb = lin[0].bias;
-            linear16(cx, abuf, cx.L.lda, &lin[0].tm_w, 128, 0, 3 * d, d, lx.n_act ? &lx : nullptr, bb, lg, [&](int r, int n, float v, float b, float gsum) {
-                const float y = stats[r].y * (v - stats[r].x * gsum) + b;
-                if (n < d) qbuf[r * cx.L.ldq + n] = __float2bfloat16_rn(y);
-                else if (r0 + r < T) kvb[(size_t)(r0 + r) * 2 * d + (n - d)] = __float2bfloat16_rn(y);
+            const float* cv = pack_acquire();
+            shrink(st[0], abuf, cx.L.lda, d, 3 * d, true, cv);
+            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, qkv_first, qkv_last, args.bar + f, [&](int r, int n, float v0, float v1) {
+                const float y0 = stats[r].y * (v0 - stats[r].x * cv[3 * d + n]) + cv[n];
+                const float y1 = stats[r].y * (v1 - stats[r].x * cv[3 * d + n + 1]) + cv[n + 1];
+                if (n < d) *reinterpret_cast<uint32_t*>(qbuf + r * cx.L.ldq + n) = pk_bf16(y0, y1);
+                else if (r0 + r < T) *reinterpret_cast<uint32_t*>(kvb + (size_t)(r0 + r) * 2 * d + (n - d)) = pk_bf16(y0, y1);
             });
+            pack_release();
         }
-        // ---- the CTAs of the frame meet: all keys and values of this block are in place (they were written
-        // with ordinary stores and are fetched by TMA on the other side: order the two proxies as well)
-        asm volatile("fence.proxy.async.global;" ::: "memory");
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0 && !*abort_flag) {
-            atomicAdd(args.bar + f, 1u);
-            const unsigned int want = (unsigned int)args.tiles_pf * (unsigned int)(l + 1);
-            const long long t0 = clock64();
-            unsigned int seen;
-            do {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(args.bar + f) : "memory");
-                if (seen < want && clock64() - t0 > LT_WAIT_CYCLES) {
-                    *abort_flag = 1;
-                    atomicCAS(args.status, 0, (int)PM_ERR_TIMEOUT);
-                    break;
-                }
-            } while (seen < want);
-        }
-        __syncthreads();
-        if (*abort_flag) break;
-        // ---- attention, head by head: the warps split the keys, then merge their partial results
-        // keys and values of a head arrive as two TMA boxes ([tpad rows][64 dims], 128B swizzle; rows past
-        // the frame hold a neighbour's rows or zeros and are masked below); the next head's are on their
-        // way while this one is computed
-        const int kv_row0 = ((l & 1) * args.n_frames + f) * T;
-        auto fetch_head = [&](int h) {
-            const int buf = (int)(cx.kv_no & 1u);
-            const uint32_t dst = s_u32(smem + cx.L.region) + buf * cx.L.kv_head;
-            bar_expect(kv_bar(cx, buf), 2u * (uint32_t)tpad * 128u);
-            tma_box(dst, &args.tm_kv, h * LT_HD, kv_row0, kv_bar(cx, buf));
-            tma_box(dst + cx.L.kv_head / 2, &args.tm_kv, d + h * LT_HD, kv_row0, kv_bar(cx, buf));
-        };
-        if (threadIdx.x == 0) {
-            asm volatile("fence.proxy.async.global;" ::: "memory");
-            fetch_head(0);
-        }
-        for (int h = 0; h < args.heads; ++h) {
-            const int buf = (int)(cx.kv_no & 1u);
-            uint8_t* Ks = smem + cx.L.region + buf * cx.L.kv_head;
-            uint8_t* Vs = Ks + cx.L.kv_head / 2;
-            bar_wait(cx, kv_bar(cx, buf), (cx.kv_no >> 1) & 1u);
-            ++cx.kv_no;
-            // the other buffer was last read by head h - 1, and everyone is past that head's closing barrier
-            if (threadIdx.x == 0 && h + 1 < args.heads) fetch_head(h + 1);
+        consumer_sync();                                     // all of q is in place
+        // ---- attention, head by head.  Warp w: key range w / 2 of four, dims 32 (w % 2) .. + 31 of the head.
+        // Keys and values of a head are one TMA box each ([tpad rows][64 dims], 128B swizzle; rows past the
+        // frame hold a neighbour's rows or zeros and are masked below).
+        {
+            const int kr = cx.warp >> 1, dh = cx.warp & 1;
             const int n_t8 = tpad / 8;
-            const int t8_lo = (n_t8 * cx.warp) / LT_WARPS, t8_hi = (n_t8 * (cx.warp + 1)) / LT_WARPS;    // at most 4 tiles
-            const uint32_t ks_addr = s_u32(Ks), vs_addr = s_u32(Vs);
-            float s[4][4];
-            uint32_t qa[4][4];
+            const int t8_lo = (n_t8 * kr) / LT_KSPLIT, t8_hi = (n_t8 * (kr + 1)) / LT_KSPLIT, n_t = t8_hi - t8_lo;   // <= LT_ST tiles
+            // a key tile is 8 rows of 128 bytes, so a lane's row keeps its swizzle phase (lane & 7) from tile
+            // to tile: one address per k16 step (keys) or pair of dim tiles (values), plus a multiple of 1 KB
+            const int l7 = cx.lane & 7, mi = cx.lane >> 3;
+            uint32_t k_addr[4], v_addr[2];
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                ldsm4(s_u32(qbuf) + ((cx.lane & 15) * cx.L.ldq + h * LT_HD + ks * 16 + (cx.lane >> 4) * 8) * 2,
-                      qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
-            float m_lo = -INFINITY, m_hi = -INFINITY;
+                k_addr[ks] = s_u32(smem + cx.L.kbuf) + (t8_lo * 8 + l7) * 128 + (((ks * 2 + (mi & 1)) ^ l7) << 4);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
-                const int t8 = t8_lo + j;
-                if (t8 < t8_hi) {
+            for (int n = 0; n < 2; ++n)
+                v_addr[n] = s_u32(smem + cx.L.vbuf) + (t8_lo * 8 + (mi & 1) * 8 + l7) * 128 + (((dh * 4 + n * 2 + (mi >> 1)) ^ l7) << 4);
+            float* part = reinterpret_cast<float*>(smem + cx.L.hbuf);
+            for (int h = 0; h < args.heads; ++h, ++head_no) {
+                uint32_t qa[4][4];
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const int r = t8 * 8 + (cx.lane & 7), c = ks * 2 + ((cx.lane >> 3) & 1);
-                        uint32_t b0, b1;
-                        ldsm2(ks_addr + r * 128 + ((c ^ (r & 7)) << 4), b0, b1);
-                        mma16816(s[j], qa[ks], b0, b1);
+                for (int ks = 0; ks < 4; ++ks)
+                    ldsm4(s_u32(qbuf) + ((cx.lane & 15) * cx.L.ldq + h * LT_HD + ks * 16 + (cx.lane >> 4) * 8) * 2,
+                          qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
+                bar_wait(cx, kfull_bar(cx), head_no & 1u);
+                float s[LT_ST][4];
+                float m_lo = -INFINITY, m_hi = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < LT_ST; ++j) {
+                    s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+                    if (j < n_t) {
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            uint32_t b0, b1;
+                            ldsm2(k_addr[ks] + j * 1024, b0, b1);
+                            mma16816(s[j], qa[ks], b0, b1);
+                        }
+                    }
+                    const int key = (t8_lo + j) * 8 + 2 * cx.t;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const bool ok = j < n_t && key + (e & 1) < T;
+                        s[j][e] = ok ? s[j][e] * att_scale : -INFINITY;
+                    }
+                    m_lo = fmaxf(m_lo, fmaxf(s[j][0], s[j][1]));
+                    m_hi = fmaxf(m_hi, fmaxf(s[j][2], s[j][3]));
+                }
+                __syncwarp();
+                if (cx.lane == 0) bar_arrive(kempty_bar(cx));        // the next head's keys may land
+                m_lo = fmaxf(m_lo, __shfl_xor_sync(0xFFFFFFFFu, m_lo, 1));
+                m_lo = fmaxf(m_lo, __shfl_xor_sync(0xFFFFFFFFu, m_lo, 2));
+                m_hi = fmaxf(m_hi, __shfl_xor_sync(0xFFFFFFFFu, m_hi, 1));
+                m_hi = fmaxf(m_hi, __shfl_xor_sync(0xFFFFFFFFu, m_hi, 2));
+                // a warp whose keys are all beyond the frame contributes nothing (its maximum stays -inf)
+                const float ms_lo = m_lo == -INFINITY ? 0.f : m_lo, ms_hi = m_hi == -INFINITY ? 0.f : m_hi;
+                float l_lo = 0.f, l_hi = 0.f;
+                uint32_t pa[LT_ST / 2][4];
+#pragma unroll
+                for (int j = 0; j < LT_ST; ++j) {
+                    const float p0 = exp2f(s[j][0] - ms_lo), p1 = exp2f(s[j][1] - ms_lo);
+                    const float p2 = exp2f(s[j][2] - ms_hi), p3 = exp2f(s[j][3] - ms_hi);
+                    l_lo += p0 + p1;
+                    l_hi += p2 + p3;
+                    pa[j >> 1][(j & 1) * 2 + 0] = pk_bf16(p0, p1);
+                    pa[j >> 1][(j & 1) * 2 + 1] = pk_bf16(p2, p3);
+                }
+                l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 1);
+                l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 2);
+                l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 1);
+                l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 2);
+                float o[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+                bar_wait(cx, vfull_bar(cx), head_no & 1u);
+                // 16-key steps of this warp's keys.  The second tile of the last step may belong to the next
+                // range (its probabilities are 0 here) or lie behind the last key (the kilobyte of zeros)
+#pragma unroll
+                for (int kk = 0; kk < LT_ST / 2; ++kk) {
+                    if (2 * kk < n_t) {
+#pragma unroll
+                        for (int n = 0; n < 2; ++n) {            // pairs of 8-dim tiles
+                            uint32_t b0, b1, b2, b3;
+                            ldsm4t(v_addr[n] + kk * 2048, b0, b1, b2, b3);
+                            mma16816(o[2 * n], pa[kk], b0, b1);
+                            mma16816(o[2 * n + 1], pa[kk], b2, b3);
+                        }
                     }
                 }
-                const int key = t8 * 8 + 2 * cx.t;
+                __syncwarp();
+                if (cx.lane == 0) bar_arrive(vempty_bar(cx));
+                // partial results: part[range][row][0..63] = o, [64] = max, [65] = sum
+                float* pw = part + (size_t)kr * LT_ROWS * (LT_HD + 2);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const bool ok = t8 < t8_hi && key + (e & 1) < T;
-                    s[j][e] = ok ? s[j][e] * att_scale : -INFINITY;
+                for (int i = 0; i < 4; ++i) {
+                    const int c = dh * 32 + i * 8 + 2 * cx.t;
+                    *reinterpret_cast<float2*>(pw + cx.g * (LT_HD + 2) + c) = make_float2(o[i][0], o[i][1]);
+                    *reinterpret_cast<float2*>(pw + (cx.g + 8) * (LT_HD + 2) + c) = make_float2(o[i][2], o[i][3]);
                 }
-                m_lo = fmaxf(m_lo, fmaxf(s[j][0], s[j][1]));
-                m_hi = fmaxf(m_hi, fmaxf(s[j][2], s[j][3]));
-            }
-            m_lo = fmaxf(m_lo, __shfl_xor_sync(0xFFFFFFFFu, m_lo, 1));
-            m_lo = fmaxf(m_lo, __shfl_xor_sync(0xFFFFFFFFu, m_lo, 2));
-            m_hi = fmaxf(m_hi, __shfl_xor_sync(0xFFFFFFFFu, m_hi, 1));
-            m_hi = fmaxf(m_hi, __shfl_xor_sync(0xFFFFFFFFu, m_hi, 2));
-            // a warp whose keys are all beyond the frame contributes nothing (its maximum stays -inf)
-            const float ms_lo = m_lo == -INFINITY ? 0.f : m_lo, ms_hi = m_hi == -INFINITY ? 0.f : m_hi;
-            float l_lo = 0.f, l_hi = 0.f;
-            uint32_t pa[2][4];
+                if (dh == 0 && cx.t == 0) {
+                    pw[cx.g * (LT_HD + 2) + 64] = m_lo; pw[cx.g * (LT_HD + 2) + 65] = l_lo;
+                    pw[(cx.g + 8) * (LT_HD + 2) + 64] = m_hi; pw[(cx.g + 8) * (LT_HD + 2) + 65] = l_hi;
+                }
+                consumer_sync();
+                {   // merge: thread -> (row, four dims)
+                    const int r = threadIdx.x >> 4, c4 = (threadIdx.x & 15) * 4;
+                    float m = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float p0 = exp2f(s[j][0] - ms_lo), p1 = exp2f(s[j][1] - ms_lo);
-                const float p2 = exp2f(s[j][2] - ms_hi), p3 = exp2f(s[j][3] - ms_hi);
-                l_lo += p0 + p1;
-                l_hi += p2 + p3;
-                pa[j >> 1][(j & 1) * 2 + 0] = pk_bf16(p0, p1);
-                pa[j >> 1][(j & 1) * 2 + 1] = pk_bf16(p2, p3);
-            }
-            l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 1);
-            l_lo += __shfl_xor_sync(0xFFFFFFFFu, l_lo, 2);
-            l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 1);
-            l_hi += __shfl_xor_sync(0xFFFFFFFFu, l_hi, 2);
-            float o[8][4];
+                    for (int w = 0; w < LT_KSPLIT; ++w) m = fmaxf(m, part[(w * LT_ROWS + r) * (LT_HD + 2) + 64]);
+                    float den = 0.f, num[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+                    for (int w = 0; w < LT_KSPLIT; ++w) {
+                        const float* pr = part + (w * LT_ROWS + r) * (LT_HD + 2);
+                        const float e = pr[64] == -INFINITY ? 0.f : exp2f(pr[64] - m);
+                        den += e * pr[65];
 #pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {                 // 16-key steps of this warp's keys
-                if (t8_lo + 2 * kk < t8_hi) {
-#pragma unroll
-                    for (int n = 0; n < 4; ++n) {            // pairs of 8-dim tiles
-                        const int mi = cx.lane >> 3;
-                        // rows past the warp's range belong to a neighbour's keys: their probabilities are 0
-                        const int r = min((t8_lo + 2 * kk) * 8 + (mi & 1) * 8 + (cx.lane & 7), tpad - 1);
-                        const int c = n * 2 + (mi >> 1);
-                        uint32_t b0, b1, b2, b3;
-                        ldsm4t(vs_addr + r * 128 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
-                        mma16816(o[2 * n], pa[kk], b0, b1);
-                        mma16816(o[2 * n + 1], pa[kk], b2, b3);
+                        for (int q = 0; q < 4; ++q) num[q] += e * pr[c4 + q];
                     }
+                    const float inv = 1.f / den;                 // key 0 is always valid: den > 0
+                    uint2 pkd;
+                    pkd.x = pk_bf16(num[0] * inv, num[1] * inv);
+                    pkd.y = pk_bf16(num[2] * inv, num[3] * inv);
+                    *reinterpret_cast<uint2*>(abuf + r * cx.L.lda + h * LT_HD + c4) = pkd;
                 }
+                consumer_sync();
             }
-            // partial results: part[warp][row][0..63] = o, [64] = max, [65] = sum
-            float* part = reinterpret_cast<float*>(smem + cx.L.part) + (size_t)cx.warp * LT_ROWS * (LT_HD + 2);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int c = i * 8 + 2 * cx.t;
-                part[cx.g * (LT_HD + 2) + c] = o[i][0]; part[cx.g * (LT_HD + 2) + c + 1] = o[i][1];
-                part[(cx.g + 8) * (LT_HD + 2) + c] = o[i][2]; part[(cx.g + 8) * (LT_HD + 2) + c + 1] = o[i][3];
-            }
-            if (cx.t == 0) {
-                part[cx.g * (LT_HD + 2) + 64] = m_lo; part[cx.g * (LT_HD + 2) + 65] = l_lo;
-                part[(cx.g + 8) * (LT_HD + 2) + 64] = m_hi; part[(cx.g + 8) * (LT_HD + 2) + 65] = l_hi;
-            }
-            __syncthreads();
-            {   // merge: thread -> (row, four dims)
-                const float* pall = reinterpret_cast<const float*>(smem + cx.L.part);
-                const int r = threadIdx.x >> 4, c4 = (threadIdx.x & 15) * 4;
-                float m = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < LT_WARPS; ++w) m = fmaxf(m, pall[(w * LT_ROWS + r) * (LT_HD + 2) + 64]);
-                float den = 0.f, num[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int w = 0; w < LT_WARPS; ++w) {
-                    const float* pr = pall + (w * LT_ROWS + r) * (LT_HD + 2);
-                    const float e = pr[64] == -INFINITY ? 0.f : exp2f(pr[64] - m);
-                    den += e * pr[65];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) num[q] += e * pr[c4 + q];
-                }
-                const float inv = 1.f / den;                 // key 0 is always valid: den > 0
-                uint2 pkd;
-                pkd.x = pk_bf16(num[0] * inv, num[1] * inv);
-                pkd.y = pk_bf16(num[2] * inv, num[3] * inv);
-                *reinterpret_cast<uint2*>(abuf + r * cx.L.lda + h * LT_HD + c4) = pkd;
-            }
-            __syncthreads();
         }
         // ---- proj (+ residual)
-        lora_shrink(cx, lin[1], aset, args.slabs_max, abuf, cx.L.lda, &lx);
         {
-            const float* bb = lin[1].bias;
-            linear16(cx, abuf, cx.L.lda, &lin[1].tm_w, 128, 0, d, d, lx.n_act ? &lx : nullptr, bb, nullptr,
-                     [&](int r, int n, float v, float b, float) { if (r0 + r < T) xres[r * d + n] += v + b; });
+            const float* cv = pack_acquire();
+            shrink(st[1], abuf, cx.L.lda, d, d, false, cv);
+            linear16(cx, abuf, cx.L.lda, d, d, st[1].n, 0, -1, nullptr, residual(cv));
+            pack_release();
         }
-        __syncthreads();
+        consumer_sync();
         // ---- fc1 (LayerNorm 2 folded, GELU) and fc2 (+ residual)
         round_rows_and_stats(cx, d, args.eps);
-        __syncthreads();
-        lora_shrink(cx, lin[2], aset, args.slabs_max, abuf, cx.L.lda, &lx);
+        consumer_sync();
         {
-            const float* lg = lin[2].ln_g; const float* bb = lin[2].bias;
-            linear16(cx, abuf, cx.L.lda, &lin[2].tm_w, 128, 0, args.mlp, d, lx.n_act ? &lx : nullptr, bb, lg, [&](int r, int n, float v, float b, float gsum) {
-                hbuf[r * cx.L.ldh + n] = __float2bfloat16_rn(gelu_exact(stats[r].y * (v - stats[r].x * gsum) + b));
+            const float* cv = pack_acquire();
+            const int N = args.mlp;
+            shrink(st[2], abuf, cx.L.lda, d, N, true, cv);
+            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, 0, -1, nullptr, [&](int r, int n, float v0, float v1) {
+                const float y0 = gelu_exact(stats[r].y * (v0 - stats[r].x * cv[N + n]) + cv[n]);
+                const float y1 = gelu_exact(stats[r].y * (v1 - stats[r].x * cv[N + n + 1]) + cv[n + 1]);
+                *reinterpret_cast<uint32_t*>(hbuf + r * cx.L.ldh + n) = pk_bf16(y0, y1);
             });
+            pack_release();
         }
-        __syncthreads();
-        lora_shrink(cx, lin[3], aset, args.slabs_max, hbuf, cx.L.ldh, &lx);
+        consumer_sync();
         {
-            const float* bb = lin[3].bias;
-            linear16(cx, hbuf, cx.L.ldh, &lin[3].tm_w, 128, 0, d, args.mlp, lx.n_act ? &lx : nullptr, bb, nullptr,
-                     [&](int r, int n, float v, float b, float) { if (r0 + r < T) xres[r * d + n] += v + b; });
+            const float* cv = pack_acquire();
+            shrink(st[3], hbuf, cx.L.ldh, args.mlp, d, false, cv);
+            linear16(cx, hbuf, cx.L.ldh, args.mlp, d, st[3].n, 0, -1, nullptr, residual(cv));
+            pack_release();
         }
-        __syncthreads();
+        consumer_sync();
     }
 
     if (*abort_flag) {
@@ -596,7 +777,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
     if (rt != 0) return;
 
     // ---- heads on the CLS row (row 0 of the frame's first CTA): final LayerNorm, base head, adapter heads
-    float* z = reinterpret_cast<float*>(smem + cx.L.region);
+    float* z = reinterpret_cast<float*>(smem + cx.L.hbuf);
     if (cx.warp == 0) {
         float v[12], sum = 0.f;
 #pragma unroll
@@ -617,42 +798,58 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         }
     }
     float* srow = args.scores_out + (size_t)frame * args.n_classes;
-    for (int k = threadIdx.x; k < args.n_classes; k += LT_THREADS) srow[k] = 0.f;
-    __syncthreads();
+    for (int k = threadIdx.x; k < args.n_classes; k += LT_CTHREADS) srow[k] = 0.f;
+    consumer_sync();
+    // one thread per head row: its d weights are independent 16-byte loads, all in flight at once
     auto dot = [&](const bf16* w) {
-        float acc = 0.f;
-        for (int c = cx.lane * 2; c < d; c += 64) {
-            const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(w + c);
-            acc = fmaf(z[c], __bfloat162float(h2.x), fmaf(z[c + 1], __bfloat162float(h2.y), acc));
-        }
+        float acc0 = 0.f, acc1 = 0.f;
+        for (int c = 0; c < d; c += 8) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(w + c));
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-        return acc;
+            for (int q = 0; q < 4; ++q) {
+                acc0 = fmaf(z[c + 2 * q], __bfloat162float(h2[q].x), acc0);
+                acc1 = fmaf(z[c + 2 * q + 1], __bfloat162float(h2[q].y), acc1);
+            }
+        }
+        return acc0 + acc1;
     };
     if (args.base_out) {
-        for (int k = cx.warp; k < args.n_classes; k += LT_WARPS) {
+        for (int k = threadIdx.x; k < args.n_classes; k += LT_CTHREADS) {
             const float v = dot(args.head_wt + (size_t)k * d) + args.head_b[k];
-            if (cx.lane == 0) args.base_out[(size_t)frame * args.n_classes + k] = 1.f / (1.f + expf(-v));
+            args.base_out[(size_t)frame * args.n_classes + k] = 1.f / (1.f + expf(-v));
         }
     }
-    for (int i = 0; i < aset.n; ++i) {
-        const int a = aset.id[i];
-        for (int r = args.hoff[a] + cx.warp; r < args.hoff[a + 1]; r += LT_WARPS) {
+    for (int i = 0; i < as->n; ++i) {
+        const int a = as->id[i];
+        for (int r = args.hoff[a] + threadIdx.x; r < args.hoff[a + 1]; r += LT_CTHREADS) {
             const float v = dot(args.hcat + (size_t)r * d) + args.hbias[r];
             // scores are positive: the maximum over adapters is an integer maximum of the bit patterns
-            if (cx.lane == 0) atomicMax(reinterpret_cast<int*>(srow + args.hcls[r]), __float_as_int(1.f / (1.f + expf(-v))));
+            atomicMax(reinterpret_cast<int*>(srow + args.hcls[r]), __float_as_int(1.f / (1.f + expf(-v))));
         }
     }
+}
+
+// the most ring slots that fit beside everything else (0: the geometry does not fit at all)
+int lat_ring_slots(int d, int mlp, int patch_dim, int tokens, int layers) {
+    const int fixed = lat_layout(d, mlp, patch_dim, tokens, layers, 0).total;
+    const int room = 227 * 1024 - fixed;
+    if (room < 3 * LT_SLOT_BYTES) return 0;
+    return room / LT_SLOT_BYTES < LT_MAX_SLOTS ? room / LT_SLOT_BYTES : LT_MAX_SLOTS;
 }
 
 }  // namespace
 
-size_t latency_smem_bytes(int d, int mlp, int patch_dim, int rs_total, int tokens) {
-    return (size_t)lat_layout(d, mlp, patch_dim, rs_total, tokens).total;
+size_t latency_smem_bytes(int d, int mlp, int patch_dim, int tokens, int layers) {
+    const int slots = lat_ring_slots(d, mlp, patch_dim, tokens, layers);
+    if (!slots) return (size_t)1 << 30;
+    return (size_t)lat_layout(d, mlp, patch_dim, tokens, layers, slots).total;
 }
 
 cudaError_t launch_latency_forward(const Launch& L, const LatArgs& a) {
-    const size_t smem = latency_smem_bytes(a.d, a.mlp, a.patch_dim, a.slabs_max * PM_SLAB * a.max_set, a.tokens);
+    const int slots = lat_ring_slots(a.d, a.mlp, a.patch_dim, a.tokens, a.layers);
+    if (!slots || a.layers * 4 > LT_THREADS) return cudaErrorInvalidValue;
+    const size_t smem = (size_t)lat_layout(a.d, a.mlp, a.patch_dim, a.tokens, a.layers, slots).total;
     static SmemGrant grant;
     if (cudaError_t e = grant.ensure(latency_forward_kernel, (int)smem); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -669,6 +866,7 @@ cudaError_t launch_latency_forward(const Launch& L, const LatArgs& a) {
     ProfScope ps(L, KC_GEMM);
     LatArgs copy = a;
     copy.status = L.status;
+    copy.ring_slots = slots;
     // the frames' arrival counters start at zero (an aborted launch may have left them anywhere)
     cudaError_t e = cudaMemsetAsync(a.bar, 0, sizeof(unsigned int) * a.n_frames, L.st);
     if (e != cudaSuccess) return e;
