@@ -298,6 +298,8 @@ def run_streams(args, rank, world, dist, local_rank):
     mode = args.loop
     m = binding.model_from_workload(w, dtype=0, max_frames=S, max_set=8)
     m.set_cover(w.tau)
+    if args.whole_network_kernel is not None:
+        m.set_small_batch_kernel(args.whole_network_kernel == "on")
     K = w.spec.n_classes
     frames_host = torch.from_numpy(w.extra["stream_frames"]).to(torch.bfloat16).transpose(0, 1).contiguous().pin_memory()
     frames_dev = frames_host.cuda()                              # [T, S, 3, img, img]
@@ -475,6 +477,9 @@ def main():
                     help="batch: ViT-base 224x224, 256 frames (the headline); streams: ViT-base 384x384, 16 streams "
                          "in closed loop (forward -> Algorithm 2 -> next forward), one step = one frame per stream; "
                          "latency: DeiT-tiny, one stream in closed loop (the paper's embedded operating point)")
+    ap.add_argument("--whole-network-kernel", default=None, choices=["on", "off"],
+                    help="latency: one kernel per forward (a CTA per 16 token rows) or the layer-by-layer kernels; "
+                         "default: the library's choice")
     ap.add_argument("--loop", default="graph", choices=["host", "device", "graph", "sequence"],
                     help="streams / latency: where the routing plan of a step is built and whether steps are "
                          "CUDA-graph replays (graph: one replay per step; sequence: the whole 30-step clip is one "

@@ -258,13 +258,14 @@ int pm_selftest_wait_timeout(long long limit_cycles, int32_t* status, int32_t* t
  * and frees the recorded graphs; default on. */
 int pm_set_graphs(pm_handle h, int on);
 
-/* Batches of a few frames of a small model (d <= 384, mlp <= 1536, tokens <= 256, max_set <= 8, bf16
- * build, and n_frames * ceil(tokens / 16) <= the number of SMs) -- the single-stream operating point of
- * Sec. 4 -- can run the whole forward (patch embedding, every block with its unmerged LoRA terms of
- * Sec. 3.1, heads, sigmoid, merge) as ONE kernel in which a CTA owns 16 token rows from the first layer to
- * the last.  pm_set_small_batch_kernel(h, 1) makes pm_forward and pm_forward_device_sets use it for
- * such batches (same results within rounding); default off: as measured on a B200 it does not yet beat
- * the layer-by-layer kernels replayed from a CUDA graph (594 against 559 us per DeiT-tiny frame). */
+/* Batches of a few frames of a small model (d <= 384 with 64-wide heads, mlp <= 1536, tokens <= 256,
+ * max_set * ceil(max_rank / 16) <= 8, bf16 build, and n_frames * ceil(tokens / 16) <= the number of SMs) --
+ * the single-stream operating point of Sec. 4 -- run the whole forward (patch embedding, every block with
+ * its unmerged LoRA terms of Sec. 3.1, heads, sigmoid, merge) as ONE kernel in which a CTA owns 16 token
+ * rows from the first layer to the last.  pm_forward and pm_forward_device_sets use it for such batches
+ * (same results within rounding as the layer-by-layer kernels; about 400 against 540 us per DeiT-tiny
+ * frame on a B200); pm_set_small_batch_kernel(h, 0) sends them through the layer-by-layer kernels
+ * instead.  Default on. */
 int pm_set_small_batch_kernel(pm_handle h, int on);
 
 /* Number of kernels the library has launched on this handle since creation (kernels of a replayed graph included). */

@@ -228,7 +228,7 @@ class Model:
         self._check(self.lib.pm_set_graphs(self.handle, int(on)), "pm_set_graphs")
 
     def set_small_batch_kernel(self, on):
-        """Whether small batches of small models run as the one whole-network kernel (default off)."""
+        """Whether small batches of small models run as the one whole-network kernel (default on)."""
         self._check(self.lib.pm_set_small_batch_kernel(self.handle, int(on)), "pm_set_small_batch_kernel")
 
     KERNEL_CLASSES = ("gemm", "shrink", "attention", "layernorm", "other", "heads", "select", "plan")

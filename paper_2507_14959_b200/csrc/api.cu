@@ -467,7 +467,7 @@ struct pm_handle_s {
     // whole-network kernel for a handful of frames (latency_kernel.cu)
     DevBuf lat_lin, lat_kv, lat_bar;
     CUtensorMap lat_tm_kv;
-    bool lat_dirty = true, lat_on = false;
+    bool lat_dirty = true, lat_on = true;
     // recorded launch sequences of the forward entry points (see run_graphed)
     struct GraphEntry {
         const void* key_ptr[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
