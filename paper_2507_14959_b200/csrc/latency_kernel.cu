@@ -268,8 +268,9 @@ __device__ __forceinline__ void acc_zero(float (&acc)[2][2][4]) {
         for (int h = 0; h < 2; ++h) acc[q][h][0] = acc[q][h][1] = acc[q][h][2] = acc[q][h][3] = 0.f;
 }
 
-// The consumers' side of a linear's chunks: y[16, N] = A[16, K] W + t B, handed to epi(row, n, y[n], y[n + 1])
-// for even n.  After the chunk `publish_after` (if >= 0) the CTA counts itself in at `counter`: everything
+// The consumers' side of a linear's chunks: y[16, N] = A[16, K] W + t B.  A thread's eight values of a chunk
+// go to epi(n0, y) in one call -- y[q][0..1] = columns n0 + 8 q, n0 + 8 q + 1 of row g, y[q][2..3] the same
+// columns of row g + 8 -- so that the epilogue can fetch everything it needs before its first store.  After the chunk `publish_after` (if >= 0) the CTA counts itself in at `counter`: everything
 // its threads stored to global memory up to there is visible to whoever sees the count.
 template <typename Epi>
 __device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl, int first_chunk, int publish_after,
@@ -303,12 +304,12 @@ __device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl
             step_release(cx);
         }
         if (active) {
+            float y[2][4];
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int n = nc * 128 + cx.warp * 16 + q * 8 + 2 * cx.t;
-                epi(cx.g, n, acc[q][0][0] + acc[q][1][0], acc[q][0][1] + acc[q][1][1]);
-                epi(cx.g + 8, n, acc[q][0][2] + acc[q][1][2], acc[q][0][3] + acc[q][1][3]);
-            }
+            for (int q = 0; q < 2; ++q)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) y[q][e] = acc[q][0][e] + acc[q][1][e];
+            epi(nc * 128 + cx.warp * 16 + 2 * cx.t, y);
         }
         if (nc == publish_after) {
             consumer_sync();
@@ -342,7 +343,16 @@ __device__ void shrink16(Ctx& cx, const bf16* A, int lda, int K, int n_sl, Epi e
     }
 }
 
-__device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f)); }
+// GELU as the layer-by-layer GEMM epilogue computes it: x (1/2 + 1/2 tanh(x q(x^2))), q a quadratic fitted so that
+// the result stays within 3e-5 of x Phi(x); one special-function instruction per element
+__device__ __forceinline__ float gelu_fit(float v) {
+    const float t = fminf(v * v, 50.f);                     // Phi has long saturated where the fitted q would turn over
+    float q = fmaf(t, -3.5151945e-04f, 3.7005664e-02f);
+    q = fmaf(q, t, 0.79750784f);
+    float h;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(h) : "f"(v * q));
+    return v * fmaf(h, 0.5f, 0.5f);
+}
 
 // abuf <- bf16(xres); stats[r] = (mean, rstd, 1/rstd) of the rounded row (what the tensor cores multiply).
 // A warp takes two rows at once (two independent reduction chains); d is a multiple of 64, at most 384.
@@ -553,15 +563,24 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
     // ---- patch projection + positions; the CLS row
     {
         const float* cv = pack_acquire();
-        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, 0, -1, nullptr, [&](int r, int n, float v0, float v1) {
-            const int tok = r0 + r;
-            float2 out = make_float2(0.f, 0.f);                     // rows past the frame stay zero
-            if (tok < T) {
-                const float2 p = *reinterpret_cast<const float2*>(args.pos + (size_t)tok * d + n);
-                if (tok == 0) out = make_float2(args.cls[n] + p.x, args.cls[n + 1] + p.y);
-                else out = make_float2(v0 + cv[n] + p.x, v1 + cv[n + 1] + p.y);
+        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, 0, -1, nullptr, [&](int n0, float (&y)[2][4]) {
+#pragma unroll
+            for (int hi = 0; hi < 2; ++hi) {
+                const int r = cx.g + 8 * hi, tok = r0 + r;
+                float2 p[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                if (tok < T) {
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) p[q] = *reinterpret_cast<const float2*>(args.pos + (size_t)tok * d + n0 + 8 * q);
+                }
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int n = n0 + 8 * q;
+                    float2 out = make_float2(0.f, 0.f);             // rows past the frame stay zero
+                    if (tok == 0) out = make_float2(args.cls[n] + p[q].x, args.cls[n + 1] + p[q].y);
+                    else if (tok < T) out = make_float2(y[q][2 * hi] + cv[n] + p[q].x, y[q][2 * hi + 1] + cv[n + 1] + p[q].y);
+                    *reinterpret_cast<float2*>(xres + r * d + n) = out;
+                }
             }
-            *reinterpret_cast<float2*>(xres + r * d + n) = out;
         });
         pack_release();
     }
@@ -584,11 +603,21 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         consumer_sync();
     };
     auto residual = [&](const float* cv) {
-        return [=](int r, int n, float v0, float v1) {
-            if (r0 + r < T) {
-                float2* x = reinterpret_cast<float2*>(xres + r * d + n);
-                *x = make_float2(x->x + v0 + cv[n], x->y + v1 + cv[n + 1]);
+        return [=](int n0, float (&y)[2][4]) {
+            float2 x[2][2], b[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                b[q] = *reinterpret_cast<const float2*>(cv + n0 + 8 * q);
+                x[q][0] = *reinterpret_cast<const float2*>(xres + cx.g * d + n0 + 8 * q);
+                x[q][1] = *reinterpret_cast<const float2*>(xres + (cx.g + 8) * d + n0 + 8 * q);
             }
+#pragma unroll
+            for (int q = 0; q < 2; ++q)
+#pragma unroll
+                for (int hi = 0; hi < 2; ++hi)
+                    if (r0 + cx.g + 8 * hi < T)
+                        *reinterpret_cast<float2*>(xres + (cx.g + 8 * hi) * d + n0 + 8 * q) =
+                            make_float2(x[q][hi].x + y[q][2 * hi] + b[q].x, x[q][hi].y + y[q][2 * hi + 1] + b[q].y);
         };
     };
 
@@ -603,11 +632,27 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         {
             const float* cv = pack_acquire();
             shrink(st[0], abuf, cx.L.lda, d, 3 * d, true, cv);
-            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, qkv_first, qkv_last, args.bar + f, [&](int r, int n, float v0, float v1) {
-                const float y0 = stats[r].y * (v0 - stats[r].x * cv[3 * d + n]) + cv[n];
-                const float y1 = stats[r].y * (v1 - stats[r].x * cv[3 * d + n + 1]) + cv[n + 1];
-                if (n < d) *reinterpret_cast<uint32_t*>(qbuf + r * cx.L.ldq + n) = pk_bf16(y0, y1);
-                else if (r0 + r < T) *reinterpret_cast<uint32_t*>(kvb + (size_t)(r0 + r) * 2 * d + (n - d)) = pk_bf16(y0, y1);
+            const float4 s_lo = stats[cx.g], s_hi = stats[cx.g + 8];
+            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, qkv_first, qkv_last, args.bar + f, [&](int n0, float (&y)[2][4]) {
+                float2 b[2], gs[2];
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    b[q] = *reinterpret_cast<const float2*>(cv + n0 + 8 * q);
+                    gs[q] = *reinterpret_cast<const float2*>(cv + 3 * d + n0 + 8 * q);
+                }
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int n = n0 + 8 * q;
+                    const uint32_t lo = pk_bf16(s_lo.y * (y[q][0] - s_lo.x * gs[q].x) + b[q].x, s_lo.y * (y[q][1] - s_lo.x * gs[q].y) + b[q].y);
+                    const uint32_t hi = pk_bf16(s_hi.y * (y[q][2] - s_hi.x * gs[q].x) + b[q].x, s_hi.y * (y[q][3] - s_hi.x * gs[q].y) + b[q].y);
+                    if (n < d) {
+                        *reinterpret_cast<uint32_t*>(qbuf + cx.g * cx.L.ldq + n) = lo;
+                        *reinterpret_cast<uint32_t*>(qbuf + (cx.g + 8) * cx.L.ldq + n) = hi;
+                    } else {
+                        if (r0 + cx.g < T) *reinterpret_cast<uint32_t*>(kvb + (size_t)(r0 + cx.g) * 2 * d + (n - d)) = lo;
+                        if (r0 + cx.g + 8 < T) *reinterpret_cast<uint32_t*>(kvb + (size_t)(r0 + cx.g + 8) * 2 * d + (n - d)) = hi;
+                    }
+                }
             });
             pack_release();
         }
@@ -753,10 +798,22 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             const float* cv = pack_acquire();
             const int N = args.mlp;
             shrink(st[2], abuf, cx.L.lda, d, N, true, cv);
-            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, 0, -1, nullptr, [&](int r, int n, float v0, float v1) {
-                const float y0 = gelu_exact(stats[r].y * (v0 - stats[r].x * cv[N + n]) + cv[n]);
-                const float y1 = gelu_exact(stats[r].y * (v1 - stats[r].x * cv[N + n + 1]) + cv[n + 1]);
-                *reinterpret_cast<uint32_t*>(hbuf + r * cx.L.ldh + n) = pk_bf16(y0, y1);
+            const float4 s_lo = stats[cx.g], s_hi = stats[cx.g + 8];
+            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, 0, -1, nullptr, [&](int n0, float (&y)[2][4]) {
+                float2 b[2], gs[2];
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    b[q] = *reinterpret_cast<const float2*>(cv + n0 + 8 * q);
+                    gs[q] = *reinterpret_cast<const float2*>(cv + N + n0 + 8 * q);
+                }
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int n = n0 + 8 * q;
+                    *reinterpret_cast<uint32_t*>(hbuf + cx.g * cx.L.ldh + n) =
+                        pk_bf16(gelu_fit(s_lo.y * (y[q][0] - s_lo.x * gs[q].x) + b[q].x), gelu_fit(s_lo.y * (y[q][1] - s_lo.x * gs[q].y) + b[q].y));
+                    *reinterpret_cast<uint32_t*>(hbuf + (cx.g + 8) * cx.L.ldh + n) =
+                        pk_bf16(gelu_fit(s_hi.y * (y[q][2] - s_hi.x * gs[q].x) + b[q].x), gelu_fit(s_hi.y * (y[q][3] - s_hi.x * gs[q].y) + b[q].y));
+                }
             });
             pack_release();
         }
