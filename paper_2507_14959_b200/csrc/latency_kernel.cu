@@ -42,9 +42,6 @@ __device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t& r0, uint32_t& r1,
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-__device__ __forceinline__ void ldsm2(uint32_t addr, uint32_t& r0, uint32_t& r1) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
-}
 __device__ __forceinline__ void ldsm4t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -55,6 +52,11 @@ __device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b
         "{%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {            // 2^x, one special-function instruction; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pk_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -667,10 +669,10 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             // a key tile is 8 rows of 128 bytes, so a lane's row keeps its swizzle phase (lane & 7) from tile
             // to tile: one address per k16 step (keys) or pair of dim tiles (values), plus a multiple of 1 KB
             const int l7 = cx.lane & 7, mi = cx.lane >> 3;
-            uint32_t k_addr[4], v_addr[2];
+            uint32_t k_addr[2], v_addr[2];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                k_addr[ks] = s_u32(smem + cx.L.kbuf) + (t8_lo * 8 + l7) * 128 + (((ks * 2 + (mi & 1)) ^ l7) << 4);
+            for (int kp = 0; kp < 2; ++kp)                   // one fetch brings a tile's keys for two k16 steps (32 dims)
+                k_addr[kp] = s_u32(smem + cx.L.kbuf) + (t8_lo * 8 + l7) * 128 + (((kp * 4 + mi) ^ l7) << 4);
 #pragma unroll
             for (int n = 0; n < 2; ++n)
                 v_addr[n] = s_u32(smem + cx.L.vbuf) + (t8_lo * 8 + (mi & 1) * 8 + l7) * 128 + (((dh * 4 + n * 2 + (mi >> 1)) ^ l7) << 4);
@@ -683,41 +685,48 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
                           qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
                 bar_wait(cx, kfull_bar(cx), head_no & 1u);
                 float s[LT_ST][4];
-                float m_lo = -INFINITY, m_hi = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < LT_ST; ++j) {
-                    s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
-                    if (j < n_t) {
+                for (int j = 0; j < LT_ST; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+                // tile by tile inside each k16 step: consecutive multiplications go to different accumulators
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            uint32_t b0, b1;
-                            ldsm2(k_addr[ks] + j * 1024, b0, b1);
-                            mma16816(s[j], qa[ks], b0, b1);
-                        }
-                    }
-                    const int key = (t8_lo + j) * 8 + 2 * cx.t;
+                for (int kp = 0; kp < 2; ++kp) {
+                    uint32_t kf[LT_ST][4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const bool ok = j < n_t && key + (e & 1) < T;
-                        s[j][e] = ok ? s[j][e] * att_scale : -INFINITY;
-                    }
-                    m_lo = fmaxf(m_lo, fmaxf(s[j][0], s[j][1]));
-                    m_hi = fmaxf(m_hi, fmaxf(s[j][2], s[j][3]));
+                    for (int j = 0; j < LT_ST; ++j)
+                        if (j < n_t) ldsm4(k_addr[kp] + j * 1024, kf[j][0], kf[j][1], kf[j][2], kf[j][3]);
+#pragma unroll
+                    for (int j = 0; j < LT_ST; ++j)
+                        if (j < n_t) mma16816(s[j], qa[2 * kp], kf[j][0], kf[j][1]);
+#pragma unroll
+                    for (int j = 0; j < LT_ST; ++j)
+                        if (j < n_t) mma16816(s[j], qa[2 * kp + 1], kf[j][2], kf[j][3]);
                 }
                 __syncwarp();
                 if (cx.lane == 0) bar_arrive(kempty_bar(cx));        // the next head's keys may land
+                float m_lo = -INFINITY, m_hi = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < LT_ST; ++j) {
+                    const int key = (t8_lo + j) * 8 + 2 * cx.t;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (!(j < n_t && key + (e & 1) < T)) s[j][e] = -INFINITY;
+                    m_lo = fmaxf(m_lo, fmaxf(s[j][0], s[j][1]));
+                    m_hi = fmaxf(m_hi, fmaxf(s[j][2], s[j][3]));
+                }
                 m_lo = fmaxf(m_lo, __shfl_xor_sync(0xFFFFFFFFu, m_lo, 1));
                 m_lo = fmaxf(m_lo, __shfl_xor_sync(0xFFFFFFFFu, m_lo, 2));
                 m_hi = fmaxf(m_hi, __shfl_xor_sync(0xFFFFFFFFu, m_hi, 1));
                 m_hi = fmaxf(m_hi, __shfl_xor_sync(0xFFFFFFFFu, m_hi, 2));
-                // a warp whose keys are all beyond the frame contributes nothing (its maximum stays -inf)
+                // the maxima in the exponent's units (1/sqrt(64) log2 e); a warp whose keys are all beyond the
+                // frame contributes nothing (its maximum stays -inf)
+                m_lo *= att_scale; m_hi *= att_scale;
                 const float ms_lo = m_lo == -INFINITY ? 0.f : m_lo, ms_hi = m_hi == -INFINITY ? 0.f : m_hi;
                 float l_lo = 0.f, l_hi = 0.f;
                 uint32_t pa[LT_ST / 2][4];
 #pragma unroll
                 for (int j = 0; j < LT_ST; ++j) {
-                    const float p0 = exp2f(s[j][0] - ms_lo), p1 = exp2f(s[j][1] - ms_lo);
-                    const float p2 = exp2f(s[j][2] - ms_hi), p3 = exp2f(s[j][3] - ms_hi);
+                    const float p0 = ex2(fmaf(s[j][0], att_scale, -ms_lo)), p1 = ex2(fmaf(s[j][1], att_scale, -ms_lo));
+                    const float p2 = ex2(fmaf(s[j][2], att_scale, -ms_hi)), p3 = ex2(fmaf(s[j][3], att_scale, -ms_hi));
                     l_lo += p0 + p1;
                     l_hi += p2 + p3;
                     pa[j >> 1][(j & 1) * 2 + 0] = pk_bf16(p0, p1);
@@ -769,7 +778,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
 #pragma unroll
                     for (int w = 0; w < LT_KSPLIT; ++w) {
                         const float* pr = part + (w * LT_ROWS + r) * (LT_HD + 2);
-                        const float e = pr[64] == -INFINITY ? 0.f : exp2f(pr[64] - m);
+                        const float e = pr[64] == -INFINITY ? 0.f : ex2(pr[64] - m);
                         den += e * pr[65];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) num[q] += e * pr[c4 + q];
