@@ -5,7 +5,7 @@
 // Everything in a ViT block except attention is local to a token row, so a CTA owns 16 token rows of one
 // frame from the first layer to the last and keeps their residual stream (fp32) and every intermediate in
 // shared memory.  What a CTA reads from L2 is static -- weights, LoRA slabs, bias vectors, in an order that
-// is known when the kernel starts -- so one producer thread walks that order and keeps a ring of 16 KB
+// is known when the kernel starts -- so one producer thread walks that order and keeps a ring of 32 KB
 // shared-memory slots full by TMA, across the boundaries of linears and blocks, while the eight consumer
 // warps multiply what has landed (full / empty transaction barriers per slot, no CTA-wide barrier in the
 // stream).  Every CTA reads every weight, 13 CTAs per frame.
@@ -28,7 +28,8 @@ constexpr int LT_ROWS = 16;
 constexpr int LT_CWARPS = 8;                 // consumer warps
 constexpr int LT_CTHREADS = LT_CWARPS * 32;
 constexpr int LT_THREADS = LT_CTHREADS + 64; // + the weight producer's warp + the key/value producer's warp
-constexpr int LT_SLOT_BYTES = 128 * 128;     // [128 output rows][64 bf16 inputs], 128B swizzle
+constexpr int LT_BOX_BYTES = 128 * 128;      // [128 output rows][64 bf16 inputs], 128B swizzle
+constexpr int LT_SLOT_BYTES = 2 * LT_BOX_BYTES;  // a ring step: two K boxes of a chunk of outputs
 constexpr int LT_MAX_SLOTS = 8;
 constexpr int LT_MAX_SET = 8;
 constexpr int LT_MAX_SLABS = 8;              // active LoRA slabs of one linear
@@ -216,10 +217,13 @@ __device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st,
         ++cx.li;
     }
     if (n_sl) {
-        for (int kb = 0; kb < k_boxes && !*cx.abort_flag; ++kb) {
-            const uint32_t dst = step_claim(cx, (uint32_t)n_sl * 2048u);
-            for (int i = 0; i < n_sl; ++i)
-                tma_box(dst + i * 2048u, &lin->tm_at, kb * 64, as.id[st.who[i]] * rs + st.sl[i] * PM_SLAB, full_bar(cx, cx.slot));
+        for (int kb0 = 0; kb0 < k_boxes && !*cx.abort_flag; kb0 += 2) {
+            const int nb = min(2, k_boxes - kb0);
+            const uint32_t dst = step_claim(cx, (uint32_t)(nb * n_sl) * 2048u);
+            for (int b = 0; b < nb; ++b)
+                for (int i = 0; i < n_sl; ++i)
+                    tma_box(dst + b * LT_BOX_BYTES + i * 2048u, &lin->tm_at, (kb0 + b) * 64, as.id[st.who[i]] * rs + st.sl[i] * PM_SLAB,
+                            full_bar(cx, cx.slot));
             ring_advance(cx);
         }
     }
@@ -227,10 +231,12 @@ __device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st,
         int nc = first_chunk + ci;
         if (nc >= n_chunks) nc -= n_chunks;
         const int rows = min(128, N - nc * 128);
-        for (int kb = 0; kb < k_boxes && !*cx.abort_flag; ++kb) {
-            const uint32_t dst = step_claim(cx, (uint32_t)rows * 128u);
-            for (int hf = 0; hf * 64 < rows; ++hf)
-                tma_box(dst + hf * 8192u, &lin->tm_w, kb * 64, nc * 128 + hf * 64, full_bar(cx, cx.slot));
+        for (int kb0 = 0; kb0 < k_boxes && !*cx.abort_flag; kb0 += 2) {
+            const int nb = min(2, k_boxes - kb0);
+            const uint32_t dst = step_claim(cx, (uint32_t)(nb * rows) * 128u);
+            for (int b = 0; b < nb; ++b)
+                for (int hf = 0; hf * 64 < rows; ++hf)
+                    tma_box(dst + b * LT_BOX_BYTES + hf * 8192u, &lin->tm_w, (kb0 + b) * 64, nc * 128 + hf * 64, full_bar(cx, cx.slot));
             ring_advance(cx);
         }
         for (int s0 = 0; s0 < n_sl && !*cx.abort_flag; s0 += 4) {
@@ -246,19 +252,26 @@ __device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st,
 }
 
 // one ring step of weights ([rows][64 inputs], this warp's 16 rows) against 64 columns of A (bf16, shared memory)
-__device__ __forceinline__ void mma_step(Ctx& cx, uint32_t a_row, bool active, float (&acc)[2][2][4]) {
-    const uint32_t box = step_acquire(cx);
+__device__ __forceinline__ void mma_step(Ctx& cx, uint32_t a_row0, int nb, bool active, float (&acc)[2][2][4]) {
+    const uint32_t box0 = step_acquire(cx);
     if (active) {
         const int mi = cx.lane >> 3;
         const int r = cx.warp * 16 + (mi >> 1) * 8 + (cx.lane & 7);
+        for (int bx = 0; bx < nb; ++bx) {
+        const uint32_t box = box0 + bx * LT_BOX_BYTES, a_row = a_row0 + bx * 128;
+        // all eight fetches first, then the eight multiplications (four independent accumulators in turn)
+        uint32_t a[4][4], b[4][4];
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {
-            uint32_t a[4], b0, b1, b2, b3;
-            ldsm4(a_row + ks * 32, a[0], a[1], a[2], a[3]);
+            ldsm4(a_row + ks * 32, a[ks][0], a[ks][1], a[ks][2], a[ks][3]);
             const int c = ks * 2 + (mi & 1);
-            ldsm4(box + r * 128 + ((c ^ (r & 7)) << 4), b0, b1, b2, b3);
-            mma16816(acc[0][ks & 1], a, b0, b1);
-            mma16816(acc[1][ks & 1], a, b2, b3);
+            ldsm4(box + r * 128 + ((c ^ (r & 7)) << 4), b[ks][0], b[ks][1], b[ks][2], b[ks][3]);
+        }
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            mma16816(acc[0][ks & 1], a[ks], b[ks][0], b[ks][1]);
+            mma16816(acc[1][ks & 1], a[ks], b[ks][2], b[ks][3]);
+        }
         }
     }
     step_release(cx);
@@ -287,7 +300,7 @@ __device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl
         const bool active = cx.warp * 16 < rows;
         float acc[2][2][4];
         acc_zero(acc);
-        for (int kb = 0; kb < k_boxes; ++kb) mma_step(cx, a_base + kb * 128, active, acc);
+        for (int kb0 = 0; kb0 < k_boxes; kb0 += 2) mma_step(cx, a_base + kb0 * 128, min(2, k_boxes - kb0), active, acc);
         for (int s0 = 0; s0 < n_sl; s0 += 4) {
             const uint32_t box = step_acquire(cx);
             if (active) {
@@ -334,7 +347,7 @@ __device__ void shrink16(Ctx& cx, const bf16* A, int lda, int K, int n_sl, Epi e
     const bool active = cx.warp < n_sl;
     float acc[2][2][4];
     acc_zero(acc);
-    for (int kb = 0; kb < k_boxes; ++kb) mma_step(cx, a_base + kb * 128, active, acc);
+    for (int kb0 = 0; kb0 < k_boxes; kb0 += 2) mma_step(cx, a_base + kb0 * 128, min(2, k_boxes - kb0), active, acc);
     if (active) {
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
@@ -900,7 +913,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
 int lat_ring_slots(int d, int mlp, int patch_dim, int tokens, int layers) {
     const int fixed = lat_layout(d, mlp, patch_dim, tokens, layers, 0).total;
     const int room = 227 * 1024 - fixed;
-    if (room < 3 * LT_SLOT_BYTES) return 0;
+    if (room < 2 * LT_SLOT_BYTES) return 0;
     return room / LT_SLOT_BYTES < LT_MAX_SLOTS ? room / LT_SLOT_BYTES : LT_MAX_SLOTS;
 }
 
