@@ -153,6 +153,7 @@ __device__ __forceinline__ uint32_t vfull_bar(const Ctx& cx) { return bars(cx) +
 __device__ __forceinline__ uint32_t vempty_bar(const Ctx& cx) { return bars(cx) + 152u; }
 __device__ __forceinline__ uint32_t cfull_bar(const Ctx& cx, uint32_t b) { return bars(cx) + 160u + 8u * b; }
 __device__ __forceinline__ uint32_t cempty_bar(const Ctx& cx, uint32_t b) { return bars(cx) + 176u + 8u * b; }
+__device__ __forceinline__ uint32_t kvdone_bar(const Ctx& cx) { return bars(cx) + 192u; }
 
 // Bounded wait on a barrier.  Once a wait has run out the CTA is aborting: later waits return at once and
 // the results are meaningless (the status word says so).
@@ -285,11 +286,12 @@ __device__ __forceinline__ void acc_zero(float (&acc)[2][2][4]) {
 
 // The consumers' side of a linear's chunks: y[16, N] = A[16, K] W + t B.  A thread's eight values of a chunk
 // go to epi(n0, y) in one call -- y[q][0..1] = columns n0 + 8 q, n0 + 8 q + 1 of row g, y[q][2..3] the same
-// columns of row g + 8 -- so that the epilogue can fetch everything it needs before its first store.  After the chunk `publish_after` (if >= 0) the CTA counts itself in at `counter`: everything
-// its threads stored to global memory up to there is visible to whoever sees the count.
+// columns of row g + 8 -- so that the epilogue can fetch everything it needs before its first store.
+// After the chunk `publish_after` (if >= 0) each warp reports at the barrier on which the key/value producer
+// waits before it counts the CTA in at the frame's counter.
 template <typename Epi>
 __device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl, int first_chunk, int publish_after,
-                         unsigned int* counter, Epi epi) {
+                         Epi epi) {
     const int k_boxes = K >> 6, n_chunks = (N + 127) >> 7;
     const uint32_t a_base = s_u32(A) + ((cx.lane & 15) * lda + (cx.lane >> 4) * 8) * 2;
     const uint32_t t_row = s_u32(cx.sm + cx.L.tbuf) + ((cx.lane & 15) * cx.L.ldt + (cx.lane >> 4) * 8) * 2;
@@ -326,14 +328,9 @@ __device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl
                 for (int e = 0; e < 4; ++e) y[q][e] = acc[q][0][e] + acc[q][1][e];
             epi(nc * 128 + cx.warp * 16 + 2 * cx.t, y);
         }
-        if (nc == publish_after) {
-            consumer_sync();
-            if (threadIdx.x == 0) {
-                // the stores were ordinary ones and are fetched by TMA on the other side: order the two proxies as well
-                asm volatile("fence.proxy.async.global;" ::: "memory");
-                __threadfence();
-                atomicAdd(counter, 1u);
-            }
+        if (nc == publish_after) {       // this warp's keys and values of the block are stored: tell the key/value producer
+            __syncwarp();
+            if (cx.lane == 0) bar_arrive(kvdone_bar(cx));
         }
     }
 }
@@ -449,6 +446,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         bar_init(kfull_bar(cx), 1); bar_init(kempty_bar(cx), LT_CWARPS);
         bar_init(vfull_bar(cx), 1); bar_init(vempty_bar(cx), LT_CWARPS);
         for (int b = 0; b < 2; ++b) { bar_init(cfull_bar(cx, b), 1); bar_init(cempty_bar(cx, b), LT_CWARPS); }
+        bar_init(kvdone_bar(cx), LT_CWARPS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -519,6 +517,14 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         if (cx.lane != 0) return;
         uint32_t idx = 0;
         for (int l = 0; l < args.layers && !*abort_flag; ++l) {
+            // the consumer warps have stored this CTA's keys and values of block l (ordinary stores, fetched by
+            // TMA on the other side: order the two proxies as well as the scopes), so the CTA counts itself in:
+            // everything its threads stored up to there is visible to whoever sees the count
+            bar_wait(cx, kvdone_bar(cx), (uint32_t)l & 1u);
+            if (*abort_flag) break;
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            __threadfence();
+            atomicAdd(args.bar + f, 1u);
             const unsigned int want = (unsigned int)args.tiles_pf * (unsigned int)(l + 1);
             const long long t0 = clock64();
             unsigned int seen;
@@ -578,7 +584,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
     // ---- patch projection + positions; the CLS row
     {
         const float* cv = pack_acquire();
-        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, 0, -1, nullptr, [&](int n0, float (&y)[2][4]) {
+        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, 0, -1, [&](int n0, float (&y)[2][4]) {
 #pragma unroll
             for (int hi = 0; hi < 2; ++hi) {
                 const int r = cx.g + 8 * hi, tok = r0 + r;
@@ -648,7 +654,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             const float* cv = pack_acquire();
             shrink(st[0], abuf, cx.L.lda, d, 3 * d, true, cv);
             const float4 s_lo = stats[cx.g], s_hi = stats[cx.g + 8];
-            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, qkv_first, qkv_last, args.bar + f, [&](int n0, float (&y)[2][4]) {
+            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, qkv_first, qkv_last, [&](int n0, float (&y)[2][4]) {
                 float2 b[2], gs[2];
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
@@ -720,9 +726,11 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
 #pragma unroll
                 for (int j = 0; j < LT_ST; ++j) {
                     const int key = (t8_lo + j) * 8 + 2 * cx.t;
+                    if (j >= n_t || (t8_lo + j) * 8 + 8 > T) {       // only the frame's last tile has keys to mask
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (!(j < n_t && key + (e & 1) < T)) s[j][e] = -INFINITY;
+                        for (int e = 0; e < 4; ++e)
+                            if (!(j < n_t && key + (e & 1) < T)) s[j][e] = -INFINITY;
+                    }
                     m_lo = fmaxf(m_lo, fmaxf(s[j][0], s[j][1]));
                     m_hi = fmaxf(m_hi, fmaxf(s[j][2], s[j][3]));
                 }
@@ -809,7 +817,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         {
             const float* cv = pack_acquire();
             shrink(st[1], abuf, cx.L.lda, d, d, false, cv);
-            linear16(cx, abuf, cx.L.lda, d, d, st[1].n, 0, -1, nullptr, residual(cv));
+            linear16(cx, abuf, cx.L.lda, d, d, st[1].n, 0, -1, residual(cv));
             pack_release();
         }
         consumer_sync();
@@ -821,7 +829,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             const int N = args.mlp;
             shrink(st[2], abuf, cx.L.lda, d, N, true, cv);
             const float4 s_lo = stats[cx.g], s_hi = stats[cx.g + 8];
-            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, 0, -1, nullptr, [&](int n0, float (&y)[2][4]) {
+            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, 0, -1, [&](int n0, float (&y)[2][4]) {
                 float2 b[2], gs[2];
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
@@ -843,7 +851,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         {
             const float* cv = pack_acquire();
             shrink(st[3], hbuf, cx.L.ldh, args.mlp, d, false, cv);
-            linear16(cx, hbuf, cx.L.ldh, args.mlp, d, st[3].n, 0, -1, nullptr, residual(cv));
+            linear16(cx, hbuf, cx.L.ldh, args.mlp, d, st[3].n, 0, -1, residual(cv));
             pack_release();
         }
         consumer_sync();
