@@ -469,12 +469,14 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ z, const T* _
 
 __device__ __forceinline__ float sigmoidf_acc(float v) { return 1.f / (1.f + expf(-v)); }
 
-// grid (ceil(K/8), ceil(F/8)): a block owns 8 classes x 8 slots.  The 8 CLS features are staged once in
+// grid (ceil(K/32), ceil(F/8)): a block owns 32 classes x 8 slots.  The 8 CLS features are staged once in
 // shared memory and shared by the block's 8 warps (read straight from global memory, every class of a
-// block would fetch them again: F x K x d x 4 bytes of cache traffic in all); each warp keeps the
-// weight row of its class in registers and walks the slots.  base_out rows are in the caller's order.
+// block would fetch them again: F x K x d x 4 bytes of cache traffic in all); each warp takes four of the
+// classes in turn, keeps the weight row of the class in registers and walks the slots (the next class's
+// row is fetched while this one is multiplied).  base_out rows are in the caller's order.
 // NV = ceil(d / 32) values per lane; the dot product runs in four chains.
 constexpr int BASE_HEAD_FRAMES = 8;
+constexpr int BASE_HEAD_CLASSES = 32;
 template <typename T, int NV>
 __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict__ z, const T* __restrict__ wt,
                                                         const float* __restrict__ bias,
@@ -487,22 +489,29 @@ __global__ void __launch_bounds__(256) base_head_kernel(const float* __restrict_
         zs[sl][c] = (sl < ns && c < d) ? z[(size_t)(s0 + sl) * d + c] : 0.f;
     }
     __syncthreads();
-    const int k = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (k >= n_classes) return;
-    float w[NV];
+    auto fetch = [&](int k, float (&w)[NV]) {
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-        const int c = lane + 32 * i;
-        w[i] = c < d ? to_f(wt[(size_t)k * d + c]) : 0.f;
-    }
-    const float bk = bias[k];
-    for (int sl = 0; sl < ns; ++sl) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int i = 0; i < NV; ++i) {
+            const int c = lane + 32 * i;
+            w[i] = (k < n_classes && c < d) ? to_f(wt[(size_t)k * d + c]) : 0.f;
+        }
+    };
+    const int k0 = blockIdx.x * BASE_HEAD_CLASSES + (threadIdx.x >> 5);
+    float w[NV], wn[NV];
+    fetch(k0, w);
+    for (int k = k0; k < n_classes && k < (int)(blockIdx.x + 1) * BASE_HEAD_CLASSES; k += 8) {
+        fetch(k + 8 < (int)(blockIdx.x + 1) * BASE_HEAD_CLASSES ? k + 8 : n_classes, wn);
+        const float bk = bias[k];
+        for (int sl = 0; sl < ns; ++sl) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < NV; ++i) acc[i & 3] = fmaf(zs[sl][lane + 32 * i], w[i], acc[i & 3]);
-        const float dot = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
-        if (lane == 0) base_out[(size_t)perm[s0 + sl] * n_classes + k] = sigmoidf_acc(dot + bk);
+            for (int i = 0; i < NV; ++i) acc[i & 3] = fmaf(zs[sl][lane + 32 * i], w[i], acc[i & 3]);
+            const float dot = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
+            if (lane == 0) base_out[(size_t)perm[s0 + sl] * n_classes + k] = sigmoidf_acc(dot + bk);
+        }
+#pragma unroll
+        for (int i = 0; i < NV; ++i) w[i] = wn[i];
     }
 }
 
@@ -542,7 +551,7 @@ cudaError_t launch_heads(const Launch& L, const T* x, int n_slots, int n_out_fra
     final_ln_kernel<T><<<(n_slots + 7) / 8, 256, 0, L.st>>>(x, lnf_g, lnf_b, z, n_slots, tokens, d, eps);
     BUMP(L);
     if (base_out && n_base_slots > 0) {
-        dim3 grid((n_classes + 7) / 8, (n_base_slots + BASE_HEAD_FRAMES - 1) / BASE_HEAD_FRAMES);
+        dim3 grid((n_classes + BASE_HEAD_CLASSES - 1) / BASE_HEAD_CLASSES, (n_base_slots + BASE_HEAD_FRAMES - 1) / BASE_HEAD_FRAMES);
         const int nv = (d + 31) / 32;                  // d <= 1024
         auto kern = nv <= 6 ? base_head_kernel<T, 6> : nv <= 12 ? base_head_kernel<T, 12>
                   : nv <= 24 ? base_head_kernel<T, 24> : base_head_kernel<T, 32>;
