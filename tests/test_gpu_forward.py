@@ -69,6 +69,39 @@ def test_deit_tiny_2frames(dtype):
     m.close()
 
 
+def test_small_batch_kernel_largest_batch_and_first_batch_beyond_it():
+    """The whole-network kernel takes as many frames as there are SMs for their 16-row tiles (13 tiles per
+    197-token frame: 11 frames on 148 SMs), frames with different sets (empty, one, three adapters) side
+    by side; every frame is compared with the oracle.  One frame more and the same call goes through the
+    layer-by-layer kernels, with the same results within the tolerance."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    w = wl.deit_tiny_stream(n_steps=13, n_streams=1)
+    n_sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n_fit = n_sms // 13
+    if not 2 <= n_fit < 13:
+        pytest.skip("needs a GPU whose SM count fits 2..12 frames of 13 tiles")
+    pool = [[], [2, 5, 9], [0], [1, 10], [3], [4, 6, 7], [8], [], [0, 5], [9], [2], [6, 10], [1]]
+    for n_frames, one_launch in ((n_fit, True), (n_fit + 1, False)):
+        frames = w.extra["stream_frames"][0, :n_frames]
+        sets = pool[:n_frames]
+        off, ids = wl.sets_to_csr(sets)
+        m = binding.model_from_workload(w, dtype=0, max_frames=n_frames, max_set=8)
+        n0 = m.launch_count()
+        s, b = run_forward(m, w, 0, frames=frames, offsets=off, ids=ids)
+        launches = m.launch_count() - n0
+        assert (launches == 1) if one_launch else (launches > 50)
+        so, bo = po.forward(w.backbone, w.adapters, frames, off, ids, w.spec.heads, w.spec.patch, w.spec.ln_eps,
+                            w.spec.n_classes)
+        assert np.abs(s - so).max() < 1e-2 and np.abs(b - bo).max() < 1e-2
+        for f, st in enumerate(sets):                                # exact zeros outside the active subsets
+            allowed = np.zeros(w.spec.n_classes, bool)
+            for a in st:
+                allowed[w.adapters[a].class_ids] = True
+            assert np.all(s[f][~allowed] == 0) and np.all(s[f][allowed] > 0)
+        m.close()
+
+
 @pytest.mark.parametrize("which", ["all_linears_rank4", "query_value_last_blocks_rank16"])
 def test_small_batch_kernel_against_oracle_and_layer_kernels(which):
     """A handful of frames of a small model run as one whole-network kernel (a CTA owns 16 token rows
