@@ -224,7 +224,7 @@ struct LatLinear {
 struct LatArgs {
     const bf16* frames;        // [F, 3, img, img]
     int n_frames, img, grid, tokens, tiles_pf, d, heads, mlp, layers, n_classes, patch_dim;
-    int ring_slots;            // 16 KB slots of the weight ring (set by the launcher)
+    int ring_slots;            // 32 KB slots of the weight ring (set by the launcher)
     float eps;
     const LatLinear* lin;      // [layers * 4 + 1]: the blocks' linears, then the patch projection
     CUtensorMap tm_kv;         // the exchange buffer as [2 * F * tokens, 2 d], boxes of [tpad rows][64 columns]

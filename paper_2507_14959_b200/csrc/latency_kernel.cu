@@ -191,10 +191,11 @@ __device__ __forceinline__ uint32_t step_claim(Ctx& cx, uint32_t bytes) {
 
 // What the weight producer sends for one linear, in this order (the consumers take it in the same order):
 //   the vector pack (bias, g, c1, c2) into the linear's pack buffer;
-//   LoRA shrink, if any slab is active: K/64 steps, each the [16 rows][64] boxes of A^T of all active slabs;
-//   for each chunk of 128 outputs, starting at first_chunk and wrapping round: K/64 steps of W^T
-//   ([64 rows][64] boxes, two per full chunk), then the chunk's rows of the active slabs' B^T
-//   ([128 rows][16] boxes, four per step).
+//   LoRA shrink, if any slab is active: K/128 steps, each the [16 rows][64] boxes of A^T of all active slabs
+//   for two K boxes (the second K box's slabs 16 KB into the slot);
+//   for each chunk of 128 outputs, starting at first_chunk and wrapping round: K/128 steps of W^T, each two
+//   K boxes of the chunk ([64 rows][64] boxes, two per K box of a full chunk), then the chunk's rows of
+//   the active slabs' B^T ([128 rows][16] boxes, four per step).
 __device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st, const ActiveSet& as, int rs, int slabs_max,
                                int first_chunk) {
     const int N = lin->n_out, K = lin->k_in, k_boxes = K >> 6, n_chunks = (N + 127) >> 7, n_sl = st.n;
