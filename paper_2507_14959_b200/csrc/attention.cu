@@ -190,10 +190,12 @@ __global__ void __launch_bounds__(512) attention_mma_kernel(const bf16* __restri
 // comes from the same scores.  With several blocks the scores are formed twice: a first sweep
 // yields each row's maximum over all keys, the second forms P against that final maximum and
 // accumulates O over the blocks, so no rescaling of O is ever needed.
-// The issuing thread and the softmax warps alternate through two mbarriers (scores / O ready,
-// rows done).  ATT_SHARES softmax warps per lane quarter split the key columns of a block; they
-// exchange row maxima and row sums through shared memory.  (One key block goes to the pipelined
-// kernel further down.)
+// Tensor memory holds two regions of scores (208 columns each) and O behind them; the issuing thread
+// forms the scores of the next step in the other region while the softmax warps sweep this one
+// (per region: one mbarrier "scores formed", one "scores consumed"), and issues a block's P V
+// product as soon as its probabilities are written.  ATT_SHARES softmax warps per lane quarter
+// split the key columns of a block; they exchange row maxima and row sums through shared memory.
+// (One key block goes to the pipelined kernel further down.)
 // ---------------------------------------------------------------------------------------
 constexpr int AQ = 128;                    // query rows per tile
 constexpr int AKB = 208;                   // keys per score block
@@ -307,24 +309,34 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t k_s = q_s + AQ_BYTES;
     const uint32_t v_s = k_s + n_blocks * AKB_BYTES;
     const uint32_t bars = v_s + n_blocks * AKB_BYTES;
-    const uint32_t kv_bar = bars, s_bar = bars + 8, r_bar = bars + 16, q_bar = bars + 24;
-    const uint32_t max_bar = bars + 48, sum_bar = bars + 56;
+    // barriers: operands landed (kv, q); scores of a step formed, per score region (s_bar[2]); a step's scores
+    // consumed by all softmax warps -- maxima taken, or probabilities written (c_bar[2]); O complete (o_bar);
+    // O read out (ofree_bar); the shares' row maxima / row sums exchanged (max_bar, sum_bar)
+    const uint32_t kv_bar = bars, q_bar = bars + 8, o_bar = bars + 48, ofree_bar = bars + 56;
+    const uint32_t max_bar = bars + 64, sum_bar = bars + 72;
+    auto s_bar = [&](uint32_t r) { return bars + 16u + 8u * r; };
+    auto c_bar = [&](uint32_t r) { return bars + 32u + 8u * r; };
     uint8_t* bar_ptr = smem_raw + (bars - base);
-    float* xchg = reinterpret_cast<float*>(bar_ptr + 64);        // [max | sum][share][row]
+    float* xchg = reinterpret_cast<float*>(bar_ptr + 128);       // [max | sum][share][row]
     constexpr int shares = SHARES;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 32);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 40);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 80);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 88);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // score steps of one query tile: with several key blocks the scores are formed twice (all of a row's
+    // maxima must be known before its first exponential, and tensor memory holds two blocks of scores
+    // beside O, not three): steps 0 .. n_blocks-1 for the maxima, n_blocks .. 2 n_blocks-1 for the
+    // probabilities.  Step s of the CTA (all tiles) uses score region s % 2.
+    const int n_steps = n_blocks > 1 ? 2 * n_blocks : 1;
 
     if (threadIdx.x == 0) {
-        mbar_init(kv_bar, 1); mbar_init(q_bar, 1); mbar_init(s_bar, 1); mbar_init(r_bar, 4 * shares);
+        mbar_init(kv_bar, 1); mbar_init(q_bar, 1);
+        for (uint32_t r = 0; r < 2; ++r) { mbar_init(s_bar(r), 1); mbar_init(c_bar(r), 4 * shares); }
+        mbar_init(o_bar, 1); mbar_init(ofree_bar, 4 * shares);
         mbar_init(max_bar, 4 * shares); mbar_init(sum_bar, 4 * shares);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        // All operand loads of the head go out before tensor memory is requested: with three CTAs
-        // resident per SM but tensor memory for two, the third one's loads land while it waits for
-        // its columns.
+        // all operand loads of the head go out before tensor memory is requested
         mbar_expect_tx(kv_bar, (uint32_t)(n_blocks * 2 * AKB_BYTES));
         for (int b = 0; b < n_blocks; ++b) {
             tma_load_2d(k_s + b * AKB_BYTES, &tm_kv, d + h * HD, f * T + b * AKB, kv_bar);
@@ -347,52 +359,69 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (warp == 0) {
         if (lane == 0) {
             // ------------------------------------------------------ TMA + MMA issue
+            // The scores of step s + 1 are formed in the other region while the softmax warps are at step s;
+            // products issued by this thread run in issue order, so a region's P V product is through
+            // before the scores that are issued after it overwrite the region.
             const uint32_t idesc_pv = instr_desc_b_mn(HD);
             // descriptors built once; a K step adds 2 (32 B) for Q / K and 128 (2048 B) for V
             const uint64_t dq0 = smem_desc(q_s, 128), dk0 = smem_desc(k_s, 128), dv0 = smem_desc(v_s, 128);
-            uint32_t step = 0;
+            uint32_t s = 0;                                      // score steps issued so far
             bool ok = true;
+            auto issue_scores = [&](int i) {                     // step i of the tile: key block i % n_blocks
+                const int b = i % n_blocks;
+                const uint32_t r = s & 1u;
+                // the region's previous scores (step s - 2) must have been consumed
+                ok = mbar_wait(c_bar(r), ((s >> 1) & 1u) ^ 1u, abort_flag, args.status);
+                if (!ok) return;
+                tc_fence_after();
+                const int nb = min(AKB, args.tpad - b * AKB);
+                const uint32_t idesc_s = instr_desc(nb);
+                const uint64_t bo = (uint64_t)((b * AKB_BYTES) >> 4);
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k)
+                    umma_bf16(tmem_base + r * (uint32_t)AKB, dq0 + 2 * k, dk0 + bo + 2 * k, idesc_s, k > 0);
+                umma_commit(s_bar(r));
+                ++s;
+            };
             for (int qt = qt0; qt < qt1 && ok; ++qt) {
                 if (qt == qt0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
                 ok = ok && mbar_wait(q_bar, (qt - qt0) & 1, abort_flag, args.status);
                 if (!ok) break;
                 tc_fence_after();
-                for (int pass = (n_blocks > 1 ? 0 : 1); pass < 2 && ok; ++pass) {
-                    for (int b = 0; b < n_blocks && ok; ++b) {
-                        const int nb = min(AKB, args.tpad - b * AKB);
-                        const uint32_t idesc_s = instr_desc(nb);
-#pragma unroll
-                        const uint64_t bo = (uint64_t)((b * AKB_BYTES) >> 4);
-#pragma unroll
-                        for (int k = 0; k < HD / 16; ++k)
-                            umma_bf16(tmem_base, dq0 + 2 * k, dk0 + bo + 2 * k, idesc_s, k > 0);
-                        umma_commit(s_bar);
-                        ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
-                        ++step;
+                const uint32_t s0 = s;                           // the tile's first step
+                issue_scores(0);
+                for (int i = 0; i < n_steps && ok; ++i) {
+                    if (i + 1 < n_steps) issue_scores(i + 1);
+                    if (!ok) break;
+                    if (n_blocks > 1 && i < n_blocks) continue;  // a step for the maxima: nothing to multiply
+                    const int b = i % n_blocks;
+                    const uint32_t si = s0 + (uint32_t)i, r = si & 1u;
+                    // the step's probabilities are written (so its scores, the tile's last ones included, exist)
+                    ok = mbar_wait(c_bar(r), (si >> 1) & 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (b == n_blocks - 1 && qt + 1 < qt1) {
+                        // the query rows are no longer needed: fetch the next tile's behind the P V products
+                        mbar_expect_tx(q_bar, AQ_BYTES);
+                        tma_load_2d(q_s, &tm_q, h * HD, f * T + (qt + 1) * AQ, q_bar);
+                    }
+                    if (b == 0 && qt > qt0) {
+                        // the first product of a tile overwrites O: the previous tile's must have been read out
+                        ok = mbar_wait(ofree_bar, (uint32_t)(qt - qt0 - 1) & 1u, abort_flag, args.status);
                         if (!ok) break;
                         tc_fence_after();
-                        if (pass == 1) {
-                            if (b == n_blocks - 1 && qt + 1 < qt1) {
-                                // the last scores of this tile exist, so its query rows are no longer
-                                // needed: fetch the next tile's behind the P V products
-                                mbar_expect_tx(q_bar, AQ_BYTES);
-                                tma_load_2d(q_s, &tm_q, h * HD, f * T + (qt + 1) * AQ, q_bar);
-                            }
-                            // P of piece kk sits where its share left it: at the start of that share's columns
-                            uint32_t p_col = 0;
-                            for (int kk = 0; kk < nb / 16; ++kk) {
-                                if (kk == att_first(shares, 1) || kk == att_first(shares, 2)) p_col = (uint32_t)(kk * 16);
-                                umma_bf16_ts(o_tmem, tmem_base + p_col, dv0 + bo + 128 * kk, idesc_pv,
-                                             (b > 0 || kk > 0) ? 1u : 0u);
-                                p_col += 8;
-                            }
-                            umma_commit(s_bar);
-                            ok = mbar_wait(r_bar, step & 1u, abort_flag, args.status);
-                            ++step;
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
                     }
+                    const int nb = min(AKB, args.tpad - b * AKB);
+                    const uint64_t bo = (uint64_t)((b * AKB_BYTES) >> 4);
+                    // P of piece kk sits where its share left it: at the start of that share's columns
+                    uint32_t p_col = 0;
+                    for (int kk = 0; kk < nb / 16; ++kk) {
+                        if (kk == att_first(shares, 1) || kk == att_first(shares, 2)) p_col = (uint32_t)(kk * 16);
+                        umma_bf16_ts(o_tmem, tmem_base + r * (uint32_t)AKB + p_col, dv0 + bo + 128 * kk, idesc_pv,
+                                     (b > 0 || kk > 0) ? 1u : 0u);
+                        p_col += 8;
+                    }
+                    if (b == n_blocks - 1) umma_commit(o_bar);
                 }
             }
         }
@@ -405,20 +434,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const float c = 0.125f * 1.4426950408889634f;            // 1/sqrt(64) * log2(e)
         float* maxes = xchg;                                     // [share][row]
         float* sums = xchg + ATT_MAX_SHARES * AQ;
-        uint32_t step = 0, tile_no = 0;
+        uint32_t s = 0, tile_no = 0;
         bool ok = true;
-        auto begin_step = [&]() {
-            ok = mbar_wait(s_bar, step & 1u, abort_flag, args.status);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (ok) tc_fence_after();
-            return ok;
-        };
-        auto end_step = [&]() {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(r_bar);
-            ++step;
-        };
         // this warp's columns of key block b: [col0, col0 + ncols), `valid` of them real
         auto my_cols = [&](int b, int& col0, int& ncols, int& valid) {
             const int np = min(AKB, args.tpad - b * AKB) / 16;
@@ -430,23 +447,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const bool warp_active = qt * AQ + quarter * 32 < T;      // else: no row of this warp exists
             float m = -INFINITY, l = 0.f;
             int col0, ncols, valid;
-            if (n_blocks > 1) {
-                for (int b = 0; b < n_blocks; ++b) {
-                    if (!begin_step()) break;
-                    my_cols(b, col0, ncols, valid);
-                    if (warp_active && ncols > 0)
-                        m = score_range_sweep<false>(t_lane + (uint32_t)col0, 0u, ncols, valid, 0.f, 0.f, m);
-                    end_step();
-                }
+            for (int i = 0; i < n_steps; ++i, ++s) {
+                const int b = i % n_blocks;
+                const bool probs = n_blocks == 1 || i >= n_blocks;
+                const uint32_t r = s & 1u;
+                ok = mbar_wait(s_bar(r), (s >> 1) & 1u, abort_flag, args.status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
-            }
-            for (int b = 0; b < n_blocks; ++b) {
-                if (!begin_step()) break;
+                tc_fence_after();
+                const uint32_t t_s = t_lane + r * (uint32_t)AKB;
                 my_cols(b, col0, ncols, valid);
-                if (b == 0) {
-                    if (n_blocks == 1 && warp_active && ncols > 0)
-                        m = score_range_sweep<false>(t_lane + (uint32_t)col0, 0u, ncols, valid, 0.f, 0.f, m);
-                    if (shares > 1) {
+                if (!probs || n_blocks == 1) {
+                    if (warp_active && ncols > 0)
+                        m = score_range_sweep<false>(t_s + (uint32_t)col0, 0u, ncols, valid, 0.f, 0.f, m);
+                }
+                if (probs) {
+                    if (b == 0 && shares > 1) {
                         // the row maximum over all keys: every share's part, through shared memory
                         maxes[share * AQ + row] = m;
                         __syncwarp();
@@ -457,57 +473,65 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int k = 0; k < shares; ++k) m = fmaxf(m, maxes[k * AQ + row]);
                     }
-                }
-                if (warp_active && ncols > 0) {
-                    l = score_range_sweep<true>(t_lane + (uint32_t)col0, t_lane + (uint32_t)col0, ncols, valid, c, m * c, l);
-                    tmem_st_wait();
-                }
-                if (shares > 1 && b == n_blocks - 1) {
-                    sums[share * AQ + row] = l;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(sum_bar);
-                }
-                end_step();
-                // O (+)= P V_b is issued now; after the last block the finished rows are written out
-                if (!begin_step()) break;
-                if (b == n_blocks - 1) {
-                    if (shares > 1) {
-                        ok = mbar_wait(sum_bar, tile_no & 1u, abort_flag, args.status);
-                        ok = __all_sync(0xFFFFFFFFu, ok);
-                        if (!ok) break;
-                        l = 0.f;
-#pragma unroll
-                        for (int k = 0; k < shares; ++k) l += sums[k * AQ + row];
+                    if (warp_active && ncols > 0) {
+                        l = score_range_sweep<true>(t_s + (uint32_t)col0, t_s + (uint32_t)col0, ncols, valid, c, m * c, l);
+                        tmem_st_wait();
                     }
-                    // the output columns are split between the first two shares (all 64 to the only one)
-                    const int ocols = shares == 1 ? 64 : 32;
-                    if (warp_active && share * ocols < 64) {
-                        const float inv = 1.f / l;
-                        bf16* orow = args.out + ((size_t)f * T + q_row) * d + h * HD + share * ocols;
-                        for (int part = 0; part < ocols / 32; ++part) {
-                            uint32_t v[32];
-                            tmem_ld32((t_lane + args.o_col) + (uint32_t)(share * ocols + part * 32), v);
-                            tmem_ld_wait();
-                            if (q_row < T) {
-                                // 32-byte stores: one full sector per row per instruction
+                    if (shares > 1 && b == n_blocks - 1) {
+                        sums[share * AQ + row] = l;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(sum_bar);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(c_bar(r));
+            }
+            if (!ok) break;
+            if (shares > 1) {
+                ok = mbar_wait(sum_bar, tile_no & 1u, abort_flag, args.status);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                l = 0.f;
 #pragma unroll
-                                for (int q = 0; q < 2; ++q) {
-                                    uint32_t o[8];
+                for (int k = 0; k < shares; ++k) l += sums[k * AQ + row];
+            }
+            // O = sum over the key blocks of P V is complete: the finished rows are written out
+            ok = mbar_wait(o_bar, tile_no & 1u, abort_flag, args.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            {
+                // the output columns are split between the first two shares (all 64 to the only one)
+                const int ocols = shares == 1 ? 64 : 32;
+                if (warp_active && share * ocols < 64) {
+                    const float inv = 1.f / l;
+                    bf16* orow = args.out + ((size_t)f * T + q_row) * d + h * HD + share * ocols;
+                    for (int part = 0; part < ocols / 32; ++part) {
+                        uint32_t v[32];
+                        tmem_ld32((t_lane + args.o_col) + (uint32_t)(share * ocols + part * 32), v);
+                        tmem_ld_wait();
+                        if (q_row < T) {
+                            // 32-byte stores: one full sector per row per instruction
 #pragma unroll
-                                    for (int e = 0; e < 8; ++e)
-                                        o[e] = pack2(__uint_as_float(v[q * 16 + 2 * e]) * inv,
-                                                     __uint_as_float(v[q * 16 + 2 * e + 1]) * inv);
-                                    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                                                 ::"l"(orow + part * 32 + q * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]),
-                                                   "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
-                                                 : "memory");
-                                }
+                            for (int q = 0; q < 2; ++q) {
+                                uint32_t o[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    o[e] = pack2(__uint_as_float(v[q * 16 + 2 * e]) * inv,
+                                                 __uint_as_float(v[q * 16 + 2 * e + 1]) * inv);
+                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                             ::"l"(orow + part * 32 + q * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]),
+                                               "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                                             : "memory");
                             }
                         }
                     }
                 }
-                end_step();
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ofree_bar);
         }
     }
 
@@ -776,10 +800,9 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
     // one key block: a CTA per head (three fit an SM).  Several key blocks: one CTA per SM, so each
     // head's query tiles are spread over several CTAs when there are too few heads to fill the GPU.
     a.q_split = (a.n_blocks > 1 && n_frames * heads < 4 * 148) ? a.n_qtiles : 1;
-    // one block: P (104 columns) replaces S (208) and O takes columns 128..191 of the same 256;
-    // several blocks: O must outlive the score blocks and sits in a second group of 256 columns
-    a.tmem_cols = a.n_blocks == 1 ? 256u : 512u;
-    a.o_col = a.n_blocks == 1 ? 128u : 256u;
+    // two regions of scores (208 columns each), O behind them
+    a.tmem_cols = 512u;
+    a.o_col = 2u * AKB;
     a.out = out; a.status = L.status;
     if (a.n_blocks == 1 && a.n_qtiles <= 2 && n_sms > 0) {
         // one key block: the pipelined persistent kernel
@@ -794,8 +817,8 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
         BUMP(L);
         return cudaGetLastError();
     }
-    // one block: 68 KB, three CTAs per SM (two computing, the third loading while it waits for TMEM)
-    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 64 + 2 * ATT_MAX_SHARES * AQ * sizeof(float);
+    // all of tensor memory and most of the shared memory: one CTA per SM
+    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 128 + 2 * ATT_MAX_SHARES * AQ * sizeof(float);
     static SmemGrant grant;
     if (cudaError_t e = grant.ensure(attention_tc_kernel<ATT_SHARES>, (int)smem); e != cudaSuccess) return e;
     ProfScope ps(L, KC_ATTENTION);

@@ -63,6 +63,27 @@ def test_attention(dtype, frames, tokens, heads):
         np.testing.assert_allclose(got[f * tokens:(f + 1) * tokens], want, **TOL[dtype])
 
 
+def test_attention_many_heads_several_query_tiles_per_cta():
+    """With enough (frame, head) pairs to fill the GPU several times over, the kernel for 209..624 tokens
+    gives each CTA all query tiles of its pair (instead of one tile per CTA): two key blocks and three
+    query tiles here, the second and third tile reusing the score regions and O of the first.  Three
+    frames of the batch are compared with the oracle."""
+    import torch
+    from paper_2507_14959_b200 import binding
+    frames, tokens, heads = 50, 300, 12
+    d = heads * 64
+    qkv = wl.normal((frames * tokens, 3 * d), 1.0, "attn_gpu_many", frames, tokens, heads).astype(np.float32)
+    qd = to_dev(qkv, 0)
+    od = torch.full((frames * tokens, d), float("nan"), device="cuda", dtype=tdtype(0))
+    binding.attention(qd, od, frames, tokens, heads, 0)
+    torch.cuda.synchronize()
+    got = to_np(od)
+    assert np.isfinite(got).all()
+    for f in (0, 17, 49):
+        want = po.attention(to_np(qd[f * tokens:(f + 1) * tokens]).astype(np.float64), heads)
+        np.testing.assert_allclose(got[f * tokens:(f + 1) * tokens], want, **TOL[0])
+
+
 def oracle_linear(cell_x, w, b, A, B, scale, tokens, offsets, ids, epilogue, residual):
     out = np.empty((cell_x.shape[0], w.shape[1]))
     w64, b64 = w.astype(np.float64), b.astype(np.float64)
