@@ -312,12 +312,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // barriers: operands landed (kv, q); scores of a step formed, per score region (s_bar[2]); a step's scores
     // consumed by all softmax warps -- maxima taken, or probabilities written (c_bar[2]); O complete (o_bar);
     // O read out (ofree_bar); the shares' row maxima / row sums exchanged (max_bar, sum_bar)
-    const uint32_t kv_bar = bars, q_bar = bars + 8, o_bar = bars + 48, ofree_bar = bars + 56;
+    const uint32_t q_bar = bars + 8, o_bar = bars + 48, ofree_bar = bars + 56;
+    auto k_bar = [&](int b) { return bars + 96u + 8u * (uint32_t)b; };       // key block b landed
+    auto v_bar = [&](int b) { return bars + 120u + 8u * (uint32_t)b; };      // value block b landed
     const uint32_t max_bar = bars + 64, sum_bar = bars + 72;
     auto s_bar = [&](uint32_t r) { return bars + 16u + 8u * r; };
     auto c_bar = [&](uint32_t r) { return bars + 32u + 8u * r; };
     uint8_t* bar_ptr = smem_raw + (bars - base);
-    float* xchg = reinterpret_cast<float*>(bar_ptr + 128);       // [max | sum][share][row]
+    float* xchg = reinterpret_cast<float*>(bar_ptr + 160);       // [max | sum][share][row]
     constexpr int shares = SHARES;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_ptr + 80);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 88);
@@ -329,21 +331,27 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int n_steps = n_blocks > 1 ? 2 * n_blocks : 1;
 
     if (threadIdx.x == 0) {
-        mbar_init(kv_bar, 1); mbar_init(q_bar, 1);
+        mbar_init(q_bar, 1);
+        for (int b = 0; b < ATT_MAX_BLOCKS; ++b) { mbar_init(k_bar(b), 1); mbar_init(v_bar(b), 1); }
         for (uint32_t r = 0; r < 2; ++r) { mbar_init(s_bar(r), 1); mbar_init(c_bar(r), 4 * shares); }
         mbar_init(o_bar, 1); mbar_init(ofree_bar, 4 * shares);
         mbar_init(max_bar, 4 * shares); mbar_init(sum_bar, 4 * shares);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        // all operand loads of the head go out before tensor memory is requested
-        mbar_expect_tx(kv_bar, (uint32_t)(n_blocks * 2 * AKB_BYTES));
-        for (int b = 0; b < n_blocks; ++b) {
-            tma_load_2d(k_s + b * AKB_BYTES, &tm_kv, d + h * HD, f * T + b * AKB, kv_bar);
-            tma_load_2d(v_s + b * AKB_BYTES, &tm_kv, 2 * d + h * HD, f * T + b * AKB, kv_bar);
-        }
+        // all operand loads of the head go out before tensor memory is requested, in the order of their
+        // first use and each block on a barrier of its own: the first scores need the query tile and the
+        // first key block only
         mbar_expect_tx(q_bar, AQ_BYTES);
         tma_load_2d(q_s, &tm_q, h * HD, f * T + qt0 * AQ, q_bar);
+        for (int b = 0; b < n_blocks; ++b) {
+            mbar_expect_tx(k_bar(b), (uint32_t)AKB_BYTES);
+            tma_load_2d(k_s + b * AKB_BYTES, &tm_kv, d + h * HD, f * T + b * AKB, k_bar(b));
+        }
+        for (int b = 0; b < n_blocks; ++b) {
+            mbar_expect_tx(v_bar(b), (uint32_t)AKB_BYTES);
+            tma_load_2d(v_s + b * AKB_BYTES, &tm_kv, 2 * d + h * HD, f * T + b * AKB, v_bar(b));
+        }
     }
     __syncwarp();
     if (warp == 0) {
@@ -372,6 +380,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t r = s & 1u;
                 // the region's previous scores (step s - 2) must have been consumed
                 ok = mbar_wait(c_bar(r), ((s >> 1) & 1u) ^ 1u, abort_flag, args.status);
+                if (ok && s < (uint32_t)n_blocks) ok = mbar_wait(k_bar(b), 0, abort_flag, args.status);   // a block's first use
                 if (!ok) return;
                 tc_fence_after();
                 const int nb = min(AKB, args.tpad - b * AKB);
@@ -384,8 +393,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 ++s;
             };
             for (int qt = qt0; qt < qt1 && ok; ++qt) {
-                if (qt == qt0) ok = mbar_wait(kv_bar, 0, abort_flag, args.status);
-                ok = ok && mbar_wait(q_bar, (qt - qt0) & 1, abort_flag, args.status);
+                ok = mbar_wait(q_bar, (qt - qt0) & 1, abort_flag, args.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s0 = s;                           // the tile's first step
@@ -398,6 +406,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const uint32_t si = s0 + (uint32_t)i, r = si & 1u;
                     // the step's probabilities are written (so its scores, the tile's last ones included, exist)
                     ok = mbar_wait(c_bar(r), (si >> 1) & 1u, abort_flag, args.status);
+                    if (ok && qt == qt0) ok = mbar_wait(v_bar(b), 0, abort_flag, args.status);          // a block's first use
                     if (!ok) break;
                     tc_fence_after();
                     if (b == n_blocks - 1 && qt + 1 < qt1) {
@@ -818,7 +827,7 @@ cudaError_t launch_attention_tc(const Launch& L, const CUtensorMap& tm_q, const 
         return cudaGetLastError();
     }
     // all of tensor memory and most of the shared memory: one CTA per SM
-    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 128 + 2 * ATT_MAX_SHARES * AQ * sizeof(float);
+    size_t smem = (size_t)AQ_BYTES + (size_t)a.n_blocks * 2 * AKB_BYTES + 160 + 2 * ATT_MAX_SHARES * AQ * sizeof(float);
     static SmemGrant grant;
     if (cudaError_t e = grant.ensure(attention_tc_kernel<ATT_SHARES>, (int)smem); e != cudaSuccess) return e;
     ProfScope ps(L, KC_ATTENTION);
