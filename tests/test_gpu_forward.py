@@ -69,6 +69,34 @@ def test_deit_tiny_2frames(dtype):
     m.close()
 
 
+def test_small_batch_kernel_odd_geometry():
+    """The whole-network kernel on a geometry that exercises its ragged ends: width 128 (two K boxes: one
+    ring step), an MLP of 320 (a last chunk of 64 outputs; five K boxes: a last step of one box), 26
+    tokens (a second row tile with 10 rows, four one-tile key ranges, two of them partly or wholly beyond
+    the frame), adapters of rank 4, 8, 16 and 24 (one and two slabs; five slabs on one frame: two steps of
+    B^T rows).  Against the oracle, and against the layer-by-layer kernels."""
+    from paper_2507_14959_b200 import binding
+    name = "odd_small_model"
+    spec = wl.ModelSpec(img=80, d=128, heads=2, mlp=320, n_classes=24, layers=3)
+    bb = wl.make_backbone(name, spec)
+    ads = [wl.make_adapter(name, spec, a, r, np.arange(6 * a, 6 * a + 6)) for a, r in enumerate((8, 24, 16, 4))]
+    sets = [[0, 1, 2, 3], [1], [], [3, 0]]
+    off, ids = wl.sets_to_csr(sets)
+    w = wl.Workload(name, spec, bb, ads, wl.make_frames(name, spec, len(sets)), off, ids)
+    so, bo = po.forward(w.backbone, w.adapters, w.frames, off, ids, spec.heads, spec.patch, spec.ln_eps, spec.n_classes)
+    m = binding.model_from_workload(w, dtype=0, max_frames=len(sets), max_set=4)
+    got = {}
+    for on in (True, False):
+        m.set_small_batch_kernel(on)
+        n0 = m.launch_count()
+        got[on] = run_forward(m, w, 0)
+        launches = m.launch_count() - n0
+        assert (launches == 1) if on else (launches > 10)
+        assert np.abs(got[on][0] - so).max() < 1e-2 and np.abs(got[on][1] - bo).max() < 1e-2
+    assert np.abs(got[True][0] - got[False][0]).max() < 5e-3
+    m.close()
+
+
 def test_small_batch_kernel_largest_batch_and_first_batch_beyond_it():
     """The whole-network kernel takes as many frames as there are SMs for their 16-row tiles (13 tiles per
     197-token frame: 11 frames on 148 SMs), frames with different sets (empty, one, three adapters) side
