@@ -153,7 +153,35 @@ __device__ __forceinline__ uint32_t vfull_bar(const Ctx& cx) { return bars(cx) +
 __device__ __forceinline__ uint32_t vempty_bar(const Ctx& cx) { return bars(cx) + 152u; }
 __device__ __forceinline__ uint32_t cfull_bar(const Ctx& cx, uint32_t b) { return bars(cx) + 160u + 8u * b; }
 __device__ __forceinline__ uint32_t cempty_bar(const Ctx& cx, uint32_t b) { return bars(cx) + 176u + 8u * b; }
-__device__ __forceinline__ uint32_t kvdone_bar(const Ctx& cx) { return bars(cx) + 192u; }
+__device__ __forceinline__ uint32_t kvdone_bar(const Ctx& cx, uint32_t part) { return bars(cx) + 192u + 8u * part; }
+
+// The order in which a linear's chunks of 128 outputs are taken (producer and consumers alike).  qkv (width d):
+// the chunk with the first head's keys, the chunk with its values, the other chunks with key or value
+// columns, then the chunks of query columns alone -- the frame's other CTAs can fetch the first head's keys
+// and values, and then the others', while this CTA is still multiplying.  Every other linear: as they come.
+struct ChunkOrder { int n_chunks, ck, cv, n_kv; bool qkv, reorder; };
+__device__ __forceinline__ ChunkOrder chunk_order(int N, int d, bool qkv) {
+    ChunkOrder o;
+    o.n_chunks = (N + 127) >> 7; o.qkv = qkv; o.reorder = qkv && o.n_chunks > 2;
+    o.ck = d >> 7; o.cv = (2 * d) >> 7; o.n_kv = o.n_chunks - o.ck;
+    return o;
+}
+__device__ __forceinline__ int chunk_at(const ChunkOrder& o, int i) {
+    if (!o.reorder) return i;
+    if (i == 0) return o.ck;
+    if (i == 1) return o.cv;
+    const int j = i - 2, rest = o.n_kv - 2;              // chunks with key / value columns besides ck and cv
+    if (j >= rest) return j - rest;                      // query columns alone: chunks 0 .. ck - 1
+    const int c = o.ck + 1 + j;
+    return c >= o.cv ? c + 1 : c;
+}
+// position after which the first head's (part 0) / all heads' (part 1) keys and values of this CTA are stored;
+// a qkv of one or two chunks is not reordered and reports once, at its end
+__device__ __forceinline__ int publish_pos(const ChunkOrder& o, int part) {
+    if (!o.qkv) return -1;
+    if (!o.reorder) return part == 0 ? -1 : o.n_chunks - 1;
+    return part == 0 ? 1 : o.n_kv - 1;
+}
 
 // Bounded wait on a barrier.  Once a wait has run out the CTA is aborting: later waits return at once and
 // the results are meaningless (the status word says so).
@@ -193,11 +221,11 @@ __device__ __forceinline__ uint32_t step_claim(Ctx& cx, uint32_t bytes) {
 //   the vector pack (bias, g, c1, c2) into the linear's pack buffer;
 //   LoRA shrink, if any slab is active: K/128 steps, each the [16 rows][64] boxes of A^T of all active slabs
 //   for two K boxes (the second K box's slabs 16 KB into the slot);
-//   for each chunk of 128 outputs, starting at first_chunk and wrapping round: K/128 steps of W^T, each two
+//   for each chunk of 128 outputs, in the order of chunk_at(): K/128 steps of W^T, each two
 //   K boxes of the chunk ([64 rows][64] boxes, two per K box of a full chunk), then the chunk's rows of
 //   the active slabs' B^T ([128 rows][16] boxes, four per step).
 __device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st, const ActiveSet& as, int rs, int slabs_max,
-                               int first_chunk) {
+                               int d, bool qkv) {
     const int N = lin->n_out, K = lin->k_in, k_boxes = K >> 6, n_chunks = (N + 127) >> 7, n_sl = st.n;
     const bool folded = lin->ln_g != nullptr;
     {
@@ -229,9 +257,9 @@ __device__ void produce_linear(Ctx& cx, const LatLinear* lin, const SlabTab& st,
             ring_advance(cx);
         }
     }
+    const ChunkOrder order = chunk_order(N, d, qkv);
     for (int ci = 0; ci < n_chunks; ++ci) {
-        int nc = first_chunk + ci;
-        if (nc >= n_chunks) nc -= n_chunks;
+        const int nc = chunk_at(order, ci);
         const int rows = min(128, N - nc * 128);
         for (int kb0 = 0; kb0 < k_boxes && !*cx.abort_flag; kb0 += 2) {
             const int nb = min(2, k_boxes - kb0);
@@ -288,17 +316,17 @@ __device__ __forceinline__ void acc_zero(float (&acc)[2][2][4]) {
 // The consumers' side of a linear's chunks: y[16, N] = A[16, K] W + t B.  A thread's eight values of a chunk
 // go to epi(n0, y) in one call -- y[q][0..1] = columns n0 + 8 q, n0 + 8 q + 1 of row g, y[q][2..3] the same
 // columns of row g + 8 -- so that the epilogue can fetch everything it needs before its first store.
-// After the chunk `publish_after` (if >= 0) each warp reports at the barrier on which the key/value producer
-// waits before it counts the CTA in at the frame's counter.
+// qkv: after the chunks at the two publish positions each warp reports at the barrier on which the key/value
+// producer waits before it counts the CTA in at the frame's counter.
 template <typename Epi>
-__device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl, int first_chunk, int publish_after,
+__device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl, int d, bool qkv,
                          Epi epi) {
     const int k_boxes = K >> 6, n_chunks = (N + 127) >> 7;
     const uint32_t a_base = s_u32(A) + ((cx.lane & 15) * lda + (cx.lane >> 4) * 8) * 2;
     const uint32_t t_row = s_u32(cx.sm + cx.L.tbuf) + ((cx.lane & 15) * cx.L.ldt + (cx.lane >> 4) * 8) * 2;
+    const ChunkOrder order = chunk_order(N, d, qkv);
     for (int ci = 0; ci < n_chunks; ++ci) {
-        int nc = first_chunk + ci;
-        if (nc >= n_chunks) nc -= n_chunks;
+        const int nc = chunk_at(order, ci);
         const int rows = min(128, N - nc * 128);
         const bool active = cx.warp * 16 < rows;
         float acc[2][2][4];
@@ -329,9 +357,13 @@ __device__ void linear16(Ctx& cx, const bf16* A, int lda, int K, int N, int n_sl
                 for (int e = 0; e < 4; ++e) y[q][e] = acc[q][0][e] + acc[q][1][e];
             epi(nc * 128 + cx.warp * 16 + 2 * cx.t, y);
         }
-        if (nc == publish_after) {       // this warp's keys and values of the block are stored: tell the key/value producer
+        // this warp's keys and values of the block (the first head's / all) are stored: tell the key/value producer
+        if (ci == publish_pos(order, 0) || ci == publish_pos(order, 1)) {
             __syncwarp();
-            if (cx.lane == 0) bar_arrive(kvdone_bar(cx));
+            if (cx.lane == 0) {
+                if (ci == publish_pos(order, 0)) bar_arrive(kvdone_bar(cx, 0));
+                if (ci == publish_pos(order, 1)) bar_arrive(kvdone_bar(cx, 1));
+            }
         }
     }
 }
@@ -447,7 +479,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         bar_init(kfull_bar(cx), 1); bar_init(kempty_bar(cx), LT_CWARPS);
         bar_init(vfull_bar(cx), 1); bar_init(vempty_bar(cx), LT_CWARPS);
         for (int b = 0; b < 2; ++b) { bar_init(cfull_bar(cx, b), 1); bar_init(cempty_bar(cx, b), LT_CWARPS); }
-        bar_init(kvdone_bar(cx), LT_CWARPS);
+        bar_init(kvdone_bar(cx, 0), LT_CWARPS); bar_init(kvdone_bar(cx, 1), LT_CWARPS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -497,20 +529,15 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         slabtab[threadIdx.x] = st;
     }
     __syncthreads();
-    // qkv: the chunks that hold key and value columns come first; after the last chunk the frame's other
-    // CTAs may fetch them, and the chunks of query columns alone follow
-    const int qkv_chunks = (3 * d + 127) >> 7;
-    const int qkv_first = qkv_chunks > 1 ? d >> 7 : 0, qkv_last = qkv_chunks - 1;
-
     // ---- the weight producer: one thread, the whole network's static operands in consumption order
     if (cx.warp == LT_CWARPS) {
         if (cx.lane != 0) return;
         SlabTab none;
         none.n = 0;
-        produce_linear(cx, args.lin + (size_t)args.layers * 4, none, *as, rs, args.slabs_max, 0);
+        produce_linear(cx, args.lin + (size_t)args.layers * 4, none, *as, rs, args.slabs_max, d, false);
         for (int l = 0; l < args.layers && !*abort_flag; ++l)
             for (int j = 0; j < 4; ++j)
-                produce_linear(cx, args.lin + (size_t)l * 4 + j, slabtab[l * 4 + j], *as, rs, args.slabs_max, j == 0 ? qkv_first : 0);
+                produce_linear(cx, args.lin + (size_t)l * 4 + j, slabtab[l * 4 + j], *as, rs, args.slabs_max, d, j == 0);
         return;
     }
     // ---- the key/value producer: per block, wait for the frame's CTAs, then one head after the other
@@ -518,34 +545,40 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         if (cx.lane != 0) return;
         uint32_t idx = 0;
         for (int l = 0; l < args.layers && !*abort_flag; ++l) {
-            // the consumer warps have stored this CTA's keys and values of block l (ordinary stores, fetched by
-            // TMA on the other side: order the two proxies as well as the scopes), so the CTA counts itself in:
-            // everything its threads stored up to there is visible to whoever sees the count
-            bar_wait(cx, kvdone_bar(cx), (uint32_t)l & 1u);
-            if (*abort_flag) break;
-            asm volatile("fence.proxy.async.global;" ::: "memory");
-            __threadfence();
-            atomicAdd(args.bar + f, 1u);
-            const unsigned int want = (unsigned int)args.tiles_pf * (unsigned int)(l + 1);
-            const long long t0 = clock64();
-            unsigned int seen;
-            do {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(args.bar + f) : "memory");
-                if (seen < want && (*abort_flag || clock64() - t0 > LT_WAIT_CYCLES)) {
-                    if (!*abort_flag) { *abort_flag = 1; atomicCAS(args.status, 0, (int)PM_ERR_TIMEOUT); }
-                    break;
-                }
-            } while (seen < want);
-            if (*abort_flag) break;
-            asm volatile("fence.proxy.async.global;" ::: "memory");
+            // Twice per block -- for the first head, then for the others -- : the consumer warps have stored this
+            // CTA's keys and values (ordinary stores, fetched by TMA on the other side: order the two proxies as
+            // well as the scopes), so the CTA counts itself in: everything its threads stored up to there is
+            // visible to whoever sees the count.  Then the heads' keys and values, one after the other.
             const int kv_row0 = ((l & 1) * args.n_frames + f) * T;
-            for (int h = 0; h < args.heads; ++h, ++idx) {
-                bar_wait(cx, kempty_bar(cx), (idx & 1u) ^ 1u);
-                bar_expect(kfull_bar(cx), (uint32_t)tpad * 128u);
-                tma_box(s_u32(smem + cx.L.kbuf), &args.tm_kv, h * LT_HD, kv_row0, kfull_bar(cx));
-                bar_wait(cx, vempty_bar(cx), (idx & 1u) ^ 1u);
-                bar_expect(vfull_bar(cx), (uint32_t)tpad * 128u);
-                tma_box(s_u32(smem + cx.L.vbuf), &args.tm_kv, d + h * LT_HD, kv_row0, vfull_bar(cx));
+            const bool two = chunk_order(3 * d, d, true).reorder;   // else: one count-in per block
+            for (int part = 0; part < (two ? 2 : 1) && !*abort_flag; ++part) {
+                bar_wait(cx, kvdone_bar(cx, two ? part : 1), (uint32_t)l & 1u);
+                if (*abort_flag) break;
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                atomicAdd(args.bar + f, 1u);
+                const unsigned int per = two ? 2u : 1u;
+                const unsigned int want = (unsigned int)args.tiles_pf * (per * (unsigned int)l + (unsigned int)part + 1u);
+                const long long t0 = clock64();
+                unsigned int seen;
+                do {
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(args.bar + f) : "memory");
+                    if (seen < want && (*abort_flag || clock64() - t0 > LT_WAIT_CYCLES)) {
+                        if (!*abort_flag) { *abort_flag = 1; atomicCAS(args.status, 0, (int)PM_ERR_TIMEOUT); }
+                        break;
+                    }
+                } while (seen < want);
+                if (*abort_flag) break;
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                const int h0 = !two ? 0 : part == 0 ? 0 : 1, h1 = !two ? args.heads : part == 0 ? 1 : args.heads;
+                for (int h = h0; h < h1; ++h, ++idx) {
+                    bar_wait(cx, kempty_bar(cx), (idx & 1u) ^ 1u);
+                    bar_expect(kfull_bar(cx), (uint32_t)tpad * 128u);
+                    tma_box(s_u32(smem + cx.L.kbuf), &args.tm_kv, h * LT_HD, kv_row0, kfull_bar(cx));
+                    bar_wait(cx, vempty_bar(cx), (idx & 1u) ^ 1u);
+                    bar_expect(vfull_bar(cx), (uint32_t)tpad * 128u);
+                    tma_box(s_u32(smem + cx.L.vbuf), &args.tm_kv, d + h * LT_HD, kv_row0, vfull_bar(cx));
+                }
             }
         }
         return;
@@ -585,7 +618,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
     // ---- patch projection + positions; the CLS row
     {
         const float* cv = pack_acquire();
-        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, 0, -1, [&](int n0, float (&y)[2][4]) {
+        linear16(cx, hbuf, cx.L.ldh, args.patch_dim, d, 0, d, false, [&](int n0, float (&y)[2][4]) {
 #pragma unroll
             for (int hi = 0; hi < 2; ++hi) {
                 const int r = cx.g + 8 * hi, tok = r0 + r;
@@ -655,7 +688,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             const float* cv = pack_acquire();
             shrink(st[0], abuf, cx.L.lda, d, 3 * d, true, cv);
             const float4 s_lo = stats[cx.g], s_hi = stats[cx.g + 8];
-            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, qkv_first, qkv_last, [&](int n0, float (&y)[2][4]) {
+            linear16(cx, abuf, cx.L.lda, d, 3 * d, st[0].n, d, true, [&](int n0, float (&y)[2][4]) {
                 float2 b[2], gs[2];
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
@@ -818,7 +851,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         {
             const float* cv = pack_acquire();
             shrink(st[1], abuf, cx.L.lda, d, d, false, cv);
-            linear16(cx, abuf, cx.L.lda, d, d, st[1].n, 0, -1, residual(cv));
+            linear16(cx, abuf, cx.L.lda, d, d, st[1].n, d, false, residual(cv));
             pack_release();
         }
         consumer_sync();
@@ -830,7 +863,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
             const int N = args.mlp;
             shrink(st[2], abuf, cx.L.lda, d, N, true, cv);
             const float4 s_lo = stats[cx.g], s_hi = stats[cx.g + 8];
-            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, 0, -1, [&](int n0, float (&y)[2][4]) {
+            linear16(cx, abuf, cx.L.lda, d, N, st[2].n, d, false, [&](int n0, float (&y)[2][4]) {
                 float2 b[2], gs[2];
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
@@ -852,7 +885,7 @@ __global__ void __launch_bounds__(LT_THREADS, 1) latency_forward_kernel(const __
         {
             const float* cv = pack_acquire();
             shrink(st[3], hbuf, cx.L.ldh, args.mlp, d, false, cv);
-            linear16(cx, hbuf, cx.L.ldh, args.mlp, d, st[3].n, 0, -1, residual(cv));
+            linear16(cx, hbuf, cx.L.ldh, args.mlp, d, st[3].n, d, false, residual(cv));
             pack_release();
         }
         consumer_sync();
