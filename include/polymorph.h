@@ -263,7 +263,7 @@ int pm_set_graphs(pm_handle h, int on);
  * the single-stream operating point of Sec. 4 -- run the whole forward (patch embedding, every block with
  * its unmerged LoRA terms of Sec. 3.1, heads, sigmoid, merge) as ONE kernel in which a CTA owns 16 token
  * rows from the first layer to the last.  pm_forward and pm_forward_device_sets use it for such batches
- * (same results within rounding as the layer-by-layer kernels; about 340 against 545 us per DeiT-tiny
+ * (same results within rounding as the layer-by-layer kernels; about 330 against 545 us per DeiT-tiny
  * frame and step on a B200); pm_set_small_batch_kernel(h, 0) sends them through the layer-by-layer kernels
  * instead.  Default on. */
 int pm_set_small_batch_kernel(pm_handle h, int on);
