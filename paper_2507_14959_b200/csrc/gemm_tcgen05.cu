@@ -751,14 +751,19 @@ struct ShrinkArgs {
     // stats_out for the GEMM that follows.  Every row tile is then visited, with or without slabs.
     float2* stats_out;
     float ln_eps;
+    int ring_bytes, max_stages;       // the stage ring of a CTA
 };
 
-constexpr int SHRINK_MAX_STAGES = 4;
+constexpr int SHRINK_MAX_STAGES = 8;
 constexpr int SHRINK_GROUP = 8;                       // slabs per pass over x: 128 accumulator columns
 constexpr int SHRINK_X_BYTES = BM * BK * 2;           // 16 KB
 constexpr int SHRINK_A_SLAB_BYTES = PM_SLAB * BK * 2; // 2 KB: 16 arena rows x 64 K-columns
-constexpr int SHRINK_RING_BYTES = 72 * 1024;          // 4 stages with one slab, 3 up to four, 2 up to eight
-constexpr int SHRINK_SMEM_BYTES = SHRINK_RING_BYTES + 256;
+// The ring of x / slab stages.  Full grids (three CTAs per SM): 72 KB, at most four stages -- 4 stages with one
+// slab, 3 up to four, 2 up to eight.  Grids of no more CTAs than SMs (a few frames): a CTA has its SM to
+// itself and nothing else hides the latency of its loads, so it takes 192 KB and up to eight stages.
+constexpr int SHRINK_RING_BYTES = 72 * 1024;
+constexpr int SHRINK_RING_BYTES_ALONE = 192 * 1024;
+constexpr int SHRINK_SMEM_MAX = SHRINK_RING_BYTES_ALONE + 256;
 
 __global__ void __launch_bounds__(SHRINK_THREADS)
 shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_at,
@@ -776,19 +781,19 @@ shrink_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
                                               // counts as having released the kernel's dependents)
     const int sg = min(ns, SHRINK_GROUP);
     const int stage_bytes = SHRINK_X_BYTES + sg * SHRINK_A_SLAB_BYTES;
-    const int STG = min(SHRINK_MAX_STAGES, SHRINK_RING_BYTES / stage_bytes);
+    const int STG = min(args.max_stages, args.ring_bytes / stage_bytes);
     // groups of slabs; in statistics mode a tile without slabs still makes one pass over x
     const int n_groups = ns == 0 ? 1 : (ns + SHRINK_GROUP - 1) / SHRINK_GROUP;
     uint32_t acc_cols = 32;                   // power of two >= 16 * sg
     while ((int)acc_cols < sg * PM_SLAB) acc_cols <<= 1;
 
-    const uint32_t bars = base + SHRINK_RING_BYTES;
+    const uint32_t bars = base + (uint32_t)args.ring_bytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (SHRINK_MAX_STAGES + s); };
     const uint32_t tfull_bar = bars + 8u * (2 * SHRINK_MAX_STAGES);
     const uint32_t tempty_bar = bars + 8u * (2 * SHRINK_MAX_STAGES + 1);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + SHRINK_RING_BYTES + 8 * (2 * SHRINK_MAX_STAGES + 2));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SHRINK_RING_BYTES + 8 * (2 * SHRINK_MAX_STAGES + 2) + 8);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + args.ring_bytes + 8 * (2 * SHRINK_MAX_STAGES + 2));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + args.ring_bytes + 8 * (2 * SHRINK_MAX_STAGES + 2) + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = args.k_in / BK;
@@ -1106,7 +1111,7 @@ bool tm_encode_3d(CUtensorMap* tm, const void* base, uint64_t d0, uint64_t d1, u
 }
 
 cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev& R,
-                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int /*n_sms*/,
+                          const CUtensorMap* tm_x, const bf16* /*x*/, int rows, bf16* tbuf, int n_sms,
                           const float2* ln_stats, float2* stats_out, float ln_eps) {
     if (R.n_tiles <= 0) return cudaSuccess;
     if (R.slab_cap <= 0) return stats_out ? cudaErrorInvalidValue : cudaSuccess;   // nothing to shrink
@@ -1123,9 +1128,12 @@ cudaError_t launch_shrink(const Launch& L, const LinearDev& lin, const RouteDev&
     // follows (which walks front to back)
     a.reverse = (size_t)rows * lin.k_in * sizeof(bf16) > ((size_t)96 << 20) ? 1 : 0;
     static SmemGrant grant;
-    if (cudaError_t e = grant.ensure(shrink_tc_kernel, SHRINK_SMEM_BYTES); e != cudaSuccess) return e;
+    if (cudaError_t e = grant.ensure(shrink_tc_kernel, SHRINK_SMEM_MAX); e != cudaSuccess) return e;
+    const bool alone = n_sms > 0 && a.n_tiles <= n_sms;
+    a.ring_bytes = alone ? SHRINK_RING_BYTES_ALONE : SHRINK_RING_BYTES;
+    a.max_stages = alone ? SHRINK_MAX_STAGES : 4;
     ProfScope ps(L, KC_SHRINK);
-    shrink_tc_kernel<<<a.n_tiles, SHRINK_THREADS, SHRINK_SMEM_BYTES, L.st>>>(*tm_x, lin.tm_at, a);
+    shrink_tc_kernel<<<a.n_tiles, SHRINK_THREADS, a.ring_bytes + 256, L.st>>>(*tm_x, lin.tm_at, a);
     BUMP(L);
     return cudaGetLastError();
 }
